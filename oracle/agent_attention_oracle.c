@@ -1,0 +1,230 @@
+/*
+ * Agent Attention forward pass: plain fp64 CPU oracle.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, dense, obviously-correct statement of
+ * what the method computes, written from the paper's equations.  It shares no code,
+ * header, table or helper with the CUDA library and must never be called from a product
+ * path; only tests, the smoke check and the benchmark's CPU-baseline leg use it.
+ *
+ * Everything is double precision.  Nothing is blocked, fused, split or padded: every
+ * softmax row is materialised in full and normalised by its plain definition.
+ *
+ * Layouts (dense, last index fastest), per slab = one (batch, head) pair:
+ *   Q, K, V : [N][d]   token t = y*W + x on an H x W grid (row-major, App. B reshape)
+ *   A       : [n][d]   agent a = ay*pw + ax
+ *   B1      : [n][N]   per head, shared over the batch          (Eq. 5)
+ *   B2      : [N][n]   per head, shared over the batch          (Eq. 5)
+ *   Wd      : [d][3][3] per head, one 3x3 filter per channel    (Eq. 6, k = 3 in Eq. 7)
+ *
+ * Parity pins live in tests/test_oracle_pins.py.  Unpinned: nothing in this file; the
+ * paper's trained-model numbers (accuracy, FID) are "parity unpinned" and not attempted.
+ */
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* ---------------------------------------------------------------------------------
+ * Agent tokens by pooling, A = Pooling(Q)  (Sec. 4.2, text under Eq. 6).
+ * Average pooling to a ph x pw grid.  Window of pooled cell (ay, ax): rows
+ * floor(ay*H/ph) .. ceil((ay+1)*H/ph)-1 and columns likewise; when ph divides H this is
+ * plain (H/ph) x (W/pw) block averaging.
+ * ------------------------------------------------------------------------------- */
+void aa_oracle_pool(const double* Q, int H, int W, int d, int ph, int pw, double* A)
+{
+    for (int ay = 0; ay < ph; ++ay) {
+        int y0 = (ay * H) / ph;
+        int y1 = ((ay + 1) * H + ph - 1) / ph;
+        for (int ax = 0; ax < pw; ++ax) {
+            int x0 = (ax * W) / pw;
+            int x1 = ((ax + 1) * W + pw - 1) / pw;
+            double* a = A + (size_t)(ay * pw + ax) * d;
+            for (int c = 0; c < d; ++c) a[c] = 0.0;
+            for (int y = y0; y < y1; ++y)
+                for (int x = x0; x < x1; ++x) {
+                    const double* q = Q + (size_t)(y * W + x) * d;
+                    for (int c = 0; c < d; ++c) a[c] += q[c];
+                }
+            double cnt = (double)(y1 - y0) * (double)(x1 - x0);
+            for (int c = 0; c < d; ++c) a[c] /= cnt;
+        }
+    }
+}
+
+/* ---------------------------------------------------------------------------------
+ * Softmax attention, Eq. 1 with Sim(q,k) = exp(q.k * scale) (Sec. 3.2), with the
+ * additive bias of Eq. 5 inside the exponent (the bias itself is not scaled):
+ *   out[i,:] = sum_j  exp(s_ij) / (sum_j' exp(s_ij'))  *  Vm[j,:],
+ *   s_ij = scale * <Qm[i,:], Km[j,:]> + bias[i,j].
+ * Qm [rows][d], Km [cols][d], Vm [cols][dv], bias [rows][cols] or NULL, out [rows][dv].
+ * If probs != NULL the row-stochastic matrix [rows][cols] is written there too.
+ * Both stages of Eq. 3 are calls of this one routine.
+ * ------------------------------------------------------------------------------- */
+void aa_oracle_softmax_attention(const double* Qm, const double* Km, const double* Vm,
+                                 const double* bias, int rows, int cols, int d, int dv,
+                                 double scale, double* out, double* probs)
+{
+    double* s = (double*)malloc(sizeof(double) * (size_t)cols);
+    for (int i = 0; i < rows; ++i) {
+        const double* q = Qm + (size_t)i * d;
+        double mx = -INFINITY;
+        for (int j = 0; j < cols; ++j) {
+            const double* k = Km + (size_t)j * d;
+            double dot = 0.0;
+            for (int c = 0; c < d; ++c) dot += q[c] * k[c];
+            double v = dot * scale;
+            if (bias) v += bias[(size_t)i * cols + j];
+            s[j] = v;
+            if (v > mx) mx = v;
+        }
+        double den = 0.0;
+        for (int j = 0; j < cols; ++j) { s[j] = exp(s[j] - mx); den += s[j]; }
+        for (int j = 0; j < cols; ++j) s[j] /= den;
+        if (probs) memcpy(probs + (size_t)i * cols, s, sizeof(double) * (size_t)cols);
+        double* o = out + (size_t)i * dv;
+        for (int c = 0; c < dv; ++c) o[c] = 0.0;
+        for (int j = 0; j < cols; ++j) {
+            const double* v = Vm + (size_t)j * dv;
+            double p = s[j];
+            for (int c = 0; c < dv; ++c) o[c] += p * v[c];
+        }
+    }
+    free(s);
+}
+
+/* ---------------------------------------------------------------------------------
+ * Diversity restoration term of Eq. 6: O += DWC(V), a depthwise 3x3 convolution over the
+ * token grid, stride 1, zero padding 1, cross-correlation indexing (no filter flip), no
+ * additive conv bias:
+ *   O[y,x,c] += sum_{u,v in 0..2} Wd[c][u][v] * V[y+u-1, x+v-1, c]   (terms outside the grid dropped)
+ * ------------------------------------------------------------------------------- */
+void aa_oracle_dwc_add(const double* V, const double* Wd, int H, int W, int d, double* O)
+{
+    for (int y = 0; y < H; ++y)
+        for (int x = 0; x < W; ++x) {
+            double* o = O + (size_t)(y * W + x) * d;
+            for (int u = 0; u < 3; ++u) {
+                int yy = y + u - 1;
+                if (yy < 0 || yy >= H) continue;
+                for (int v = 0; v < 3; ++v) {
+                    int xx = x + v - 1;
+                    if (xx < 0 || xx >= W) continue;
+                    const double* vin = V + (size_t)(yy * W + xx) * d;
+                    for (int c = 0; c < d; ++c) o[c] += Wd[(size_t)c * 9 + u * 3 + v] * vin[c];
+                }
+            }
+        }
+}
+
+/* ---------------------------------------------------------------------------------
+ * The module of Eq. 6,  O = s(Q A^T + B2) s(A K^T + B1) V + DWC(V),  evaluated as the two
+ * Softmax attentions of Eq. 3 (agent aggregation, then agent broadcast).
+ *
+ *   Q, K, V [B][heads][N][d];  A_in [B][heads][n][d] or NULL (then A = Pooling(Q) with a
+ *   ph x pw agent grid, n = ph*pw);  b1 [heads][n][N] / b2 [heads][N][n] or NULL;
+ *   wd [heads][d][3][3] or NULL;  O [B][heads][N][d].
+ *   A_out, VA_out: optional [B][heads][n][d] copies of the agents and agent features.
+ *   threads: slabs are independent and are spread over this many OpenMP threads.
+ * Returns the number of threads actually used, or -1 on bad arguments.
+ * ------------------------------------------------------------------------------- */
+int aa_oracle_forward(const double* Q, const double* K, const double* V, const double* A_in,
+                      int B, int heads, int H, int W, int d, int n, int ph, int pw,
+                      const double* b1, const double* b2, const double* wd,
+                      double scale1, double scale2,
+                      double* O, double* A_out, double* VA_out, int threads)
+{
+    if (!Q || !K || !V || !O || B <= 0 || heads <= 0 || H <= 0 || W <= 0 || d <= 0 || n <= 0)
+        return -1;
+    if (!A_in && (ph <= 0 || pw <= 0 || ph * pw != n || ph > H || pw > W)) return -1;
+    const int N = H * W;
+    const int slabs = B * heads;
+    int used = 1;
+    if (threads < 1) threads = 1;
+#ifdef _OPENMP
+    if (threads > slabs) threads = slabs;
+    used = threads;
+    #pragma omp parallel for num_threads(threads) schedule(dynamic, 1)
+#endif
+    for (int s = 0; s < slabs; ++s) {
+        const int head = s % heads;
+        const size_t off = (size_t)s * N * d;
+        const double* q = Q + off;
+        const double* k = K + off;
+        const double* v = V + off;
+        double* o = O + off;
+        double* a  = (double*)malloc(sizeof(double) * (size_t)n * d);
+        double* va = (double*)malloc(sizeof(double) * (size_t)n * d);
+        if (A_in) memcpy(a, A_in + (size_t)s * n * d, sizeof(double) * (size_t)n * d);
+        else      aa_oracle_pool(q, H, W, d, ph, pw, a);
+        /* agent aggregation  V_A = Attn^S(A, K, V)  with B1 */
+        aa_oracle_softmax_attention(a, k, v, b1 ? b1 + (size_t)head * n * N : NULL,
+                                    n, N, d, d, scale1, va, NULL);
+        /* agent broadcast  O = Attn^S(Q, A, V_A)  with B2 */
+        aa_oracle_softmax_attention(q, a, va, b2 ? b2 + (size_t)head * N * n : NULL,
+                                    N, n, d, d, scale2, o, NULL);
+        if (wd) aa_oracle_dwc_add(v, wd + (size_t)head * d * 9, H, W, d, o);
+        if (A_out)  memcpy(A_out  + (size_t)s * n * d, a,  sizeof(double) * (size_t)n * d);
+        if (VA_out) memcpy(VA_out + (size_t)s * n * d, va, sizeof(double) * (size_t)n * d);
+        free(a);
+        free(va);
+    }
+    return used;
+}
+
+/* ---------------------------------------------------------------------------------
+ * Generalized-linear-attention form, Eq. 4 (with the biases of Eq. 5): for one slab form
+ * the explicit N x N matrix  M = s(Q A^T + B2) . s(A K^T + B1)  and  O = M V.
+ * Tiny inputs only (O(N^2) memory).  M [N][N], O [N][d].
+ * ------------------------------------------------------------------------------- */
+void aa_oracle_explicit(const double* Q, const double* A, const double* K, const double* V,
+                        const double* b1, const double* b2, int N, int n, int d,
+                        double scale1, double scale2, double* M, double* O)
+{
+    double* phiq = (double*)malloc(sizeof(double) * (size_t)N * n);   /* s(Q A^T + B2) */
+    double* phik = (double*)malloc(sizeof(double) * (size_t)n * N);   /* s(A K^T + B1) */
+    double* dump = (double*)malloc(sizeof(double) * (size_t)(N > n ? N : n) * d);
+    aa_oracle_softmax_attention(Q, A, A, b2, N, n, d, d, scale2, dump, phiq);
+    aa_oracle_softmax_attention(A, K, K, b1, n, N, d, d, scale1, dump, phik);
+    for (int i = 0; i < N; ++i)
+        for (int j = 0; j < N; ++j) {
+            double acc = 0.0;
+            for (int a = 0; a < n; ++a) acc += phiq[(size_t)i * n + a] * phik[(size_t)a * N + j];
+            M[(size_t)i * N + j] = acc;
+        }
+    for (int i = 0; i < N; ++i)
+        for (int c = 0; c < d; ++c) {
+            double acc = 0.0;
+            for (int j = 0; j < N; ++j) acc += M[(size_t)i * N + j] * V[(size_t)j * d + c];
+            O[(size_t)i * d + c] = acc;
+        }
+    free(phiq); free(phik); free(dump);
+}
+
+/* ---------------------------------------------------------------------------------
+ * Module complexity, Eq. 7, in multiply-accumulates for N tokens, C channels (all heads),
+ * n agents, DWC kernel size k:
+ *   parts = { 4NC^2 (projections), NC (agents), 2nNC (aggregation: logits and weighted
+ *   sum), 2NnC (broadcast), k^2 NC (DWC) };  returns their sum.
+ * ------------------------------------------------------------------------------- */
+long long aa_oracle_macs(long long N, long long C, long long n, long long k, long long* parts)
+{
+    long long p[5];
+    p[0] = 4 * N * C * C;
+    p[1] = N * C;
+    p[2] = 2 * n * N * C;
+    p[3] = 2 * N * n * C;
+    p[4] = k * k * N * C;
+    if (parts) memcpy(parts, p, sizeof(p));
+    return p[0] + p[1] + p[2] + p[3] + p[4];
+}
+
+int aa_oracle_max_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
