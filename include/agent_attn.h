@@ -1,0 +1,163 @@
+/*
+ * agent_attn.h - C ABI of the Agent Attention forward pass for NVIDIA B200 (sm_100a).
+ *
+ * The library evaluates, per (batch, head) pair ("slab") of N = grid_h * grid_w tokens laid
+ * out row-major on a 2-D grid (token t = y * grid_w + x), the module of Eq. 6 of
+ * "Agent Attention: On the Integration of Softmax and Linear Attention":
+ *
+ *     A   = Pooling(Q)                                   (n agents, text under Eq. 6)
+ *     V_A = softmax(scale1 * A K^T + B1) V               (agent aggregation, Eq. 3 / Eq. 5)
+ *     O   = softmax(scale2 * Q A^T + B2) V_A + DWC(V)    (agent broadcast,  Eq. 3 / Eq. 5 / Eq. 6)
+ *
+ * with scale = 1/sqrt(d) by default (Sec. 3.2), dense additive agent biases B1 [n x N] and
+ * B2 [N x n] per head (Eq. 5; not multiplied by the scale), and DWC a depthwise 3x3
+ * cross-correlation over the token grid with zero padding and no additive bias (Eq. 6, k = 3
+ * in Eq. 7).
+ *
+ * General rules
+ *  - Every pointer named "device" must be device memory of the handle's GPU, 16-byte aligned,
+ *    dense with the stated shape (last index fastest).  The caller owns all buffers; the
+ *    library allocates no device memory in any call below except agent_attn_create (one small
+ *    status word).  Nothing may alias `out`.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  All device
+ *    work is enqueued on it; calls return without synchronising unless stated otherwise.
+ *  - Every int-returning function returns an aa_status.  On failure nothing was launched (or,
+ *    for AA_ERR_CUDA, the launch failed) and agent_attn_last_error() describes the reason.
+ *    No call throws, aborts or traps.
+ *  - Results are bit-identical from run to run for the same inputs, handle configuration and
+ *    device.
+ */
+#ifndef AGENT_ATTN_H_
+#define AGENT_ATTN_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct agent_attn_handle agent_attn_handle;   /* opaque; host memory owned by the library */
+
+typedef enum { AA_F32 = 0, AA_BF16 = 1, AA_F16 = 2 } aa_dtype;
+
+typedef enum {
+    AA_OK = 0,
+    AA_ERR_INVALID_ARG = 1,   /* null pointer, bad shape, misaligned pointer, aliasing */
+    AA_ERR_UNSUPPORTED = 2,   /* head_dim > 128, n_agents > 256, unknown dtype, ... */
+    AA_ERR_WORKSPACE   = 3,   /* workspace (or staging) buffer too small */
+    AA_ERR_CUDA        = 4,   /* a CUDA runtime call failed (no usable GPU included) */
+    AA_ERR_TIMEOUT     = 5    /* a bounded device-side wait gave up (see query_status) */
+} aa_status;
+
+typedef enum {
+    AA_PATH_AUTO = 0,         /* tensor-core kernels for bf16/f16, fp32 FMA kernels for f32 */
+    AA_PATH_SIMT = 1          /* fp32 FMA kernels for every dtype (slow; for cross-checks) */
+} aa_path;
+
+typedef struct {
+    int   batch;              /* B: batch entries per call                                  */
+    int   heads;              /* h: heads per batch entry; slab index = b * heads + head    */
+    int   head_dim;           /* d: 8..128, head_dim * sizeof(element) a multiple of 16     */
+    int   max_tokens;         /* largest N = grid_h * grid_w any call will use              */
+    int   max_agents;         /* largest n any call will use (<= 256)                       */
+    int   dtype;              /* aa_dtype: element type of Q, K, V, A, B1, B2, Wd and out   */
+    float scale1;             /* logit scale of the aggregation; 0 selects 1/sqrt(d)        */
+    float scale2;             /* logit scale of the broadcast;   0 selects 1/sqrt(d)        */
+    int   device;             /* CUDA device ordinal                                        */
+    int   path;               /* aa_path                                                    */
+} agent_attn_config;
+
+/* Dense agent biases of Eq. 5, already composed (App. B); either member may be NULL. */
+typedef struct {
+    const void* b1;           /* device [heads][n][N]: added to scale1 * A K^T              */
+    const void* b2;           /* device [heads][N][n]: added to scale2 * Q A^T              */
+} agent_attn_bias;
+
+/* Creates a handle for one configuration.  Makes cfg->device current for the duration of the
+ * call, allocates one 4-byte device status word, and keeps only host-side plan data.
+ * Errors: AA_ERR_INVALID_ARG (null, non-positive sizes), AA_ERR_UNSUPPORTED (limits above),
+ * AA_ERR_CUDA (no such device, or the device is not compute capability 10.x). */
+int agent_attn_create(agent_attn_handle** out, const agent_attn_config* cfg);
+
+/* Frees the handle and its status word.  NULL is accepted. */
+int agent_attn_destroy(agent_attn_handle* h);
+
+/* Text of the most recent failure on this handle ("" if none); valid until the next call on
+ * the handle.  NULL handle returns a static string. */
+const char* agent_attn_last_error(const agent_attn_handle* h);
+
+/* Bytes of device workspace that agent_attn_forward / agent_attn_aggregate need for this
+ * grid and agent count (holds A, V_A, the per-split online-softmax partials (max, sum, acc)
+ * and one arrival counter per slab).  Returns 0 on invalid arguments.  Its contents need
+ * no initialisation and carry nothing from call to call; it may be reused by any number of
+ * calls that do not overlap on the GPU. */
+size_t agent_attn_workspace_bytes(const agent_attn_handle* h, int grid_h, int grid_w, int n_agents);
+
+/* The whole module, Eq. 6.
+ *   Q, K, V     device [B][heads][N][d]
+ *   A           device [B][heads][n][d] agent tokens, or NULL: A = average pooling of Q over the
+ *               grid to a p x p agent grid with n = p * p (window of cell (ay, ax): rows
+ *               floor(ay*H/p) .. ceil((ay+1)*H/p) - 1, columns likewise); then n_agents must be a
+ *               perfect square with p <= min(grid_h, grid_w)
+ *   bias        NULL, or biases of Eq. 5 (members may be NULL individually)
+ *   dwc_weight  device [heads][d][3][3] or NULL (no DWC term).  tap (u, v) multiplies
+ *               V[y + u - 1][x + v - 1]; taps outside the grid contribute zero
+ *   out         device [B][heads][N][d]
+ *   workspace   device, >= agent_attn_workspace_bytes(...)
+ * Errors: AA_ERR_INVALID_ARG, AA_ERR_UNSUPPORTED (N > max_tokens, n > max_agents),
+ * AA_ERR_WORKSPACE, AA_ERR_CUDA.  Performs no host synchronisation and no allocation. */
+int agent_attn_forward(agent_attn_handle* h,
+                       const void* Q, const void* K, const void* V, const void* A,
+                       int grid_h, int grid_w, int n_agents,
+                       const agent_attn_bias* bias, const void* dwc_weight,
+                       void* out, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Step 1 alone: agent tokens by pooling (text under Eq. 6).  Q device [B][heads][N][d] ->
+ * A_out device [B][heads][n][d], n = pool_h * pool_w, windows as described above. */
+int agent_attn_pool(agent_attn_handle* h, const void* Q, int grid_h, int grid_w,
+                    int pool_h, int pool_w, void* A_out, void* stream);
+
+/* Step 2 alone: agent aggregation V_A = softmax(scale1 * A K^T + B1) V (Eq. 3, Eq. 5).
+ * A device [B][heads][n][d]; K, V device [B][heads][N][d]; b1 device [heads][n][N] or NULL;
+ * VA_out device [B][heads][n][d].  The N keys of a slab are split over thread blocks; the
+ * workspace (>= agent_attn_workspace_bytes for any grid with grid_h * grid_w = n_tokens)
+ * receives their partial (max, sum, acc) states, which the last block to finish merges in a
+ * fixed order. */
+int agent_attn_aggregate(agent_attn_handle* h, const void* A, const void* K, const void* V,
+                         const void* b1, int n_tokens, int n_agents, void* VA_out,
+                         void* workspace, size_t workspace_bytes, void* stream);
+
+/* Step 3 alone: agent broadcast plus the DWC term, O = softmax(scale2 * Q A^T + B2) V_A + DWC(V)
+ * (Eq. 3, Eq. 5, Eq. 6).  Q, V device [B][heads][N][d]; A, VA device [B][heads][n][d];
+ * b2 device [heads][N][n] or NULL; dwc_weight device [heads][d][3][3] or NULL (V is then
+ * unused and may be NULL). */
+int agent_attn_broadcast(agent_attn_handle* h, const void* Q, const void* A, const void* VA,
+                         const void* V, const void* b2, const void* dwc_weight,
+                         int grid_h, int grid_w, int n_agents, void* out, void* stream);
+
+/* Bytes of device staging memory that agent_attn_forward_host needs (room for Q, K, V, A, B1,
+ * B2, Wd, out and the workspace, each 256-byte aligned).  0 on invalid arguments. */
+size_t agent_attn_staging_bytes(const agent_attn_handle* h, int grid_h, int grid_w, int n_agents);
+
+/* Eq. 6 on HOST buffers: same arguments as agent_attn_forward, but Q, K, V, A, the bias
+ * members, dwc_weight and out are host pointers (pinned memory makes the copies asynchronous).
+ * `staging` is device memory of >= agent_attn_staging_bytes(...) owned by the caller.
+ * Enqueues host-to-device copies of every input, the forward pass and the device-to-host copy
+ * of out on `stream`; the caller synchronises the stream before reading `out`. */
+int agent_attn_forward_host(agent_attn_handle* h,
+                            const void* Q, const void* K, const void* V, const void* A,
+                            int grid_h, int grid_w, int n_agents,
+                            const agent_attn_bias* bias, const void* dwc_weight,
+                            void* out, void* staging, size_t staging_bytes, void* stream);
+
+/* Synchronises `stream`, then returns the device-side status word: AA_OK, or AA_ERR_TIMEOUT if
+ * a kernel's bounded wait expired since the last query (the word is cleared). */
+int agent_attn_query_status(agent_attn_handle* h, void* stream);
+
+/* Number of kernels the most recent successful call on this handle enqueued. */
+int agent_attn_last_launch_count(const agent_attn_handle* h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* AGENT_ATTN_H_ */
