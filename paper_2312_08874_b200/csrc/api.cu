@@ -1,0 +1,376 @@
+// C ABI of the agent-attention library: argument checks, workspace carving and kernel launches.
+// Every step of the path runs in the CUDA kernels of this directory; there is no CPU fallback.
+#include "../../include/agent_attn.h"
+#include "kernels.h"
+
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+using namespace aa;
+
+struct agent_attn_handle {
+    agent_attn_config cfg;
+    float scale1, scale2;
+    int sm_count;
+    int elem_bytes;
+    int* d_status;          // one device word: bounded waits report here (none of the current kernels wait)
+    int launches;
+    char err[512];
+};
+
+namespace {
+
+const char* kNullHandleMsg = "agent_attn: null handle";
+
+int fail(agent_attn_handle* h, int code, const char* fmt, ...) {
+    if (h) {
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(h->err, sizeof(h->err), fmt, ap);
+        va_end(ap);
+    }
+    return code;
+}
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+
+bool use_simt(const agent_attn_handle* h) {
+    return h->cfg.dtype == AA_F32 || h->cfg.path == AA_PATH_SIMT;
+}
+
+AggPlan plan_for(const agent_attn_handle* h, int n_tokens, int n_agents) {
+    const int slabs = h->cfg.batch * h->cfg.heads;
+    return use_simt(h) ? plan_aggregate_simt(slabs, n_agents, n_tokens, h->cfg.head_dim, h->sm_count)
+                       : plan_aggregate_mma(slabs, n_agents, n_tokens, h->cfg.head_dim, h->sm_count);
+}
+
+// Workspace layout: [A | V_A | partials | tickets], each region 256-byte aligned.
+struct WsLayout {
+    size_t a_off, va_off, part_off, ticket_off, total;
+};
+WsLayout ws_layout(const agent_attn_handle* h, int n_tokens, int n_agents) {
+    const size_t slabs = (size_t)h->cfg.batch * h->cfg.heads;
+    const AggPlan pl = plan_for(h, n_tokens, n_agents);
+    const size_t av = align_up(slabs * n_agents * h->cfg.head_dim * h->elem_bytes, 256);
+    WsLayout w;
+    w.a_off = 0;
+    w.va_off = av;
+    w.part_off = 2 * av;
+    w.ticket_off = w.part_off + align_up(slabs * pl.parts * partial_floats(pl.rows_pad, pl.dpad) * sizeof(float), 256);
+    w.total = w.ticket_off + align_up(slabs * sizeof(unsigned), 256);
+    return w;
+}
+
+int check_shape(agent_attn_handle* h, int n_tokens, int n_agents) {
+    if (n_tokens <= 0 || n_agents <= 0)
+        return fail(h, AA_ERR_INVALID_ARG, "token and agent counts must be positive (N=%d, n=%d)", n_tokens, n_agents);
+    if (n_tokens > h->cfg.max_tokens)
+        return fail(h, AA_ERR_UNSUPPORTED, "N=%d exceeds the handle's max_tokens=%d", n_tokens, h->cfg.max_tokens);
+    if (n_agents > h->cfg.max_agents)
+        return fail(h, AA_ERR_UNSUPPORTED, "n=%d exceeds the handle's max_agents=%d", n_agents, h->cfg.max_agents);
+    return AA_OK;
+}
+
+int isqrt_exact(int n) {
+    int p = (int)std::lround(std::sqrt((double)n));
+    return (p * p == n) ? p : -1;
+}
+
+int do_pool(agent_attn_handle* h, const void* Q, int gh, int gw, int ph, int pw, void* A, cudaStream_t st) {
+    PoolArgs pa;
+    pa.q = Q; pa.a = A;
+    pa.slabs = h->cfg.batch * h->cfg.heads;
+    pa.H = gh; pa.W = gw; pa.d = h->cfg.head_dim; pa.ph = ph; pa.pw = pw;
+    cudaError_t e = launch_pool(h->cfg.dtype, pa, st);
+    if (e != cudaSuccess) return fail(h, AA_ERR_CUDA, "pool launch failed: %s", cudaGetErrorString(e));
+    h->launches++;
+    return AA_OK;
+}
+
+int do_aggregate(agent_attn_handle* h, const void* A, const void* K, const void* V, const void* b1,
+                 int N, int n, void* VA, float* partials, unsigned* tickets, cudaStream_t st) {
+    const AggPlan pl = plan_for(h, N, n);
+    cudaError_t e = cudaMemsetAsync(tickets, 0, (size_t)h->cfg.batch * h->cfg.heads * sizeof(unsigned), st);
+    if (e != cudaSuccess) return fail(h, AA_ERR_CUDA, "ticket reset failed: %s", cudaGetErrorString(e));
+    AttnArgs a;
+    memset(&a, 0, sizeof(a));
+    a.qm = A; a.km = K; a.vm = V; a.bias = b1; a.out = VA;
+    a.partials = partials; a.tickets = tickets;
+    a.slabs = h->cfg.batch * h->cfg.heads; a.heads = h->cfg.heads;
+    a.rows = n; a.cols = N; a.d = h->cfg.head_dim;
+    a.scale = h->scale1; a.splits = pl.splits;
+    e = use_simt(h) ? launch_aggregate_simt(h->cfg.dtype, a, pl, st)
+                    : launch_aggregate_mma(h->cfg.dtype, a, pl, st);
+    if (e != cudaSuccess) return fail(h, AA_ERR_CUDA, "aggregation launch failed: %s", cudaGetErrorString(e));
+    h->launches++;
+    return AA_OK;
+}
+
+int do_broadcast(agent_attn_handle* h, const void* Q, const void* A, const void* VA, const void* V,
+                 const void* b2, const void* wd, int gh, int gw, int n, void* out, cudaStream_t st) {
+    AttnArgs a;
+    memset(&a, 0, sizeof(a));
+    a.qm = Q; a.km = A; a.vm = VA; a.bias = b2; a.out = out;
+    a.slabs = h->cfg.batch * h->cfg.heads; a.heads = h->cfg.heads;
+    a.rows = gh * gw; a.cols = n; a.d = h->cfg.head_dim;
+    a.scale = h->scale2; a.splits = 1;
+    a.dwc_v = wd ? V : nullptr; a.dwc_w = wd; a.H = gh; a.W = gw;
+    cudaError_t e = use_simt(h) ? launch_broadcast_simt(h->cfg.dtype, a, st)
+                                : launch_broadcast_mma(h->cfg.dtype, a, st);
+    if (e != cudaSuccess) return fail(h, AA_ERR_CUDA, "broadcast launch failed: %s", cudaGetErrorString(e));
+    h->launches++;
+    return AA_OK;
+}
+
+// Device guard: the handle's device is current inside every call and restored on exit.
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; prev = -1; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    }
+    ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+}  // namespace
+
+extern "C" {
+
+int agent_attn_create(agent_attn_handle** out, const agent_attn_config* cfg) {
+    if (!out || !cfg) return AA_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (cfg->batch <= 0 || cfg->heads <= 0 || cfg->head_dim <= 0 || cfg->max_tokens <= 0 ||
+        cfg->max_agents <= 0 || cfg->scale1 < 0.f || cfg->scale2 < 0.f)
+        return AA_ERR_INVALID_ARG;
+    if (cfg->dtype != AA_F32 && cfg->dtype != AA_BF16 && cfg->dtype != AA_F16) return AA_ERR_UNSUPPORTED;
+    if (cfg->path != AA_PATH_AUTO && cfg->path != AA_PATH_SIMT) return AA_ERR_UNSUPPORTED;
+    const int es = cfg->dtype == AA_F32 ? 4 : 2;
+    if (cfg->head_dim > 128 || cfg->head_dim < 8 || (cfg->head_dim * es) % 16 != 0) return AA_ERR_UNSUPPORTED;
+    if (cfg->max_agents > 256) return AA_ERR_UNSUPPORTED;
+    if ((long long)cfg->batch * cfg->heads > 65535) return AA_ERR_UNSUPPORTED;
+
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || cfg->device < 0 || cfg->device >= count) {
+        cudaGetLastError();
+        return AA_ERR_CUDA;
+    }
+    DeviceGuard guard(cfg->device);
+    if (!guard.ok) return AA_ERR_CUDA;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, cfg->device) != cudaSuccess) return AA_ERR_CUDA;
+    if (prop.major != 10) return AA_ERR_CUDA;       // the kernels are built for sm_100a only
+
+    agent_attn_handle* h = new (std::nothrow) agent_attn_handle;
+    if (!h) return AA_ERR_INVALID_ARG;
+    memset(h, 0, sizeof(*h));
+    h->cfg = *cfg;
+    h->elem_bytes = es;
+    h->sm_count = prop.multiProcessorCount;
+    const float def = 1.0f / std::sqrt((float)cfg->head_dim);
+    h->scale1 = cfg->scale1 > 0.f ? cfg->scale1 : def;
+    h->scale2 = cfg->scale2 > 0.f ? cfg->scale2 : def;
+    if (cudaMalloc(&h->d_status, sizeof(int)) != cudaSuccess || cudaMemset(h->d_status, 0, sizeof(int)) != cudaSuccess) {
+        delete h;
+        return AA_ERR_CUDA;
+    }
+    *out = h;
+    return AA_OK;
+}
+
+int agent_attn_destroy(agent_attn_handle* h) {
+    if (!h) return AA_OK;
+    {
+        DeviceGuard guard(h->cfg.device);
+        if (h->d_status) cudaFree(h->d_status);
+    }
+    delete h;
+    return AA_OK;
+}
+
+const char* agent_attn_last_error(const agent_attn_handle* h) { return h ? h->err : kNullHandleMsg; }
+
+int agent_attn_last_launch_count(const agent_attn_handle* h) { return h ? h->launches : 0; }
+
+size_t agent_attn_workspace_bytes(const agent_attn_handle* h, int grid_h, int grid_w, int n_agents) {
+    if (!h || grid_h <= 0 || grid_w <= 0 || n_agents <= 0) return 0;
+    if ((long long)grid_h * grid_w > h->cfg.max_tokens || n_agents > h->cfg.max_agents) return 0;
+    return ws_layout(h, grid_h * grid_w, n_agents).total;
+}
+
+int agent_attn_pool(agent_attn_handle* h, const void* Q, int grid_h, int grid_w, int pool_h, int pool_w,
+                    void* A_out, void* stream) {
+    if (!h) return AA_ERR_INVALID_ARG;
+    h->err[0] = 0;
+    if (!Q || !A_out) return fail(h, AA_ERR_INVALID_ARG, "null pointer");
+    if (grid_h <= 0 || grid_w <= 0 || pool_h <= 0 || pool_w <= 0 || pool_h > grid_h || pool_w > grid_w)
+        return fail(h, AA_ERR_INVALID_ARG, "pool grid %dx%d does not fit token grid %dx%d", pool_h, pool_w, grid_h, grid_w);
+    if (int rc = check_shape(h, grid_h * grid_w, pool_h * pool_w)) return rc;
+    if (misaligned(Q) || misaligned(A_out)) return fail(h, AA_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
+    DeviceGuard guard(h->cfg.device);
+    if (!guard.ok) return fail(h, AA_ERR_CUDA, "cannot select device %d", h->cfg.device);
+    h->launches = 0;
+    return do_pool(h, Q, grid_h, grid_w, pool_h, pool_w, A_out, (cudaStream_t)stream);
+}
+
+int agent_attn_aggregate(agent_attn_handle* h, const void* A, const void* K, const void* V, const void* b1,
+                         int n_tokens, int n_agents, void* VA_out, void* workspace, size_t workspace_bytes,
+                         void* stream) {
+    if (!h) return AA_ERR_INVALID_ARG;
+    h->err[0] = 0;
+    if (!A || !K || !V || !VA_out || !workspace) return fail(h, AA_ERR_INVALID_ARG, "null pointer");
+    if (int rc = check_shape(h, n_tokens, n_agents)) return rc;
+    if (misaligned(A) || misaligned(K) || misaligned(V) || misaligned(VA_out) || misaligned(workspace) ||
+        (b1 && misaligned(b1)))
+        return fail(h, AA_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
+    const WsLayout w = ws_layout(h, n_tokens, n_agents);
+    if (workspace_bytes < w.total)
+        return fail(h, AA_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", workspace_bytes, w.total);
+    DeviceGuard guard(h->cfg.device);
+    if (!guard.ok) return fail(h, AA_ERR_CUDA, "cannot select device %d", h->cfg.device);
+    h->launches = 0;
+    char* ws = static_cast<char*>(workspace);
+    return do_aggregate(h, A, K, V, b1, n_tokens, n_agents, VA_out, reinterpret_cast<float*>(ws + w.part_off),
+                        reinterpret_cast<unsigned*>(ws + w.ticket_off), (cudaStream_t)stream);
+}
+
+int agent_attn_broadcast(agent_attn_handle* h, const void* Q, const void* A, const void* VA, const void* V,
+                         const void* b2, const void* dwc_weight, int grid_h, int grid_w, int n_agents,
+                         void* out, void* stream) {
+    if (!h) return AA_ERR_INVALID_ARG;
+    h->err[0] = 0;
+    if (!Q || !A || !VA || !out || (dwc_weight && !V)) return fail(h, AA_ERR_INVALID_ARG, "null pointer");
+    if (grid_h <= 0 || grid_w <= 0) return fail(h, AA_ERR_INVALID_ARG, "grid must be positive");
+    if (int rc = check_shape(h, grid_h * grid_w, n_agents)) return rc;
+    if (misaligned(Q) || misaligned(A) || misaligned(VA) || misaligned(out) || (V && misaligned(V)) ||
+        (b2 && misaligned(b2)) || (dwc_weight && misaligned(dwc_weight)))
+        return fail(h, AA_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
+    if (out == Q || out == V || out == A || out == VA) return fail(h, AA_ERR_INVALID_ARG, "out must not alias an input");
+    DeviceGuard guard(h->cfg.device);
+    if (!guard.ok) return fail(h, AA_ERR_CUDA, "cannot select device %d", h->cfg.device);
+    h->launches = 0;
+    return do_broadcast(h, Q, A, VA, V, b2, dwc_weight, grid_h, grid_w, n_agents, out, (cudaStream_t)stream);
+}
+
+int agent_attn_forward(agent_attn_handle* h, const void* Q, const void* K, const void* V, const void* A,
+                       int grid_h, int grid_w, int n_agents, const agent_attn_bias* bias, const void* dwc_weight,
+                       void* out, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!h) return AA_ERR_INVALID_ARG;
+    h->err[0] = 0;
+    if (!Q || !K || !V || !out || !workspace) return fail(h, AA_ERR_INVALID_ARG, "null pointer");
+    if (grid_h <= 0 || grid_w <= 0) return fail(h, AA_ERR_INVALID_ARG, "grid must be positive");
+    if ((long long)grid_h * grid_w > 0x7fffffffLL) return fail(h, AA_ERR_INVALID_ARG, "grid too large");
+    const int N = grid_h * grid_w;
+    if (int rc = check_shape(h, N, n_agents)) return rc;
+    int p = 0;
+    if (!A) {
+        p = isqrt_exact(n_agents);
+        if (p < 0 || p > grid_h || p > grid_w)
+            return fail(h, AA_ERR_INVALID_ARG,
+                        "pooled agents need n = p*p with p <= min(grid_h, grid_w); got n=%d on %dx%d",
+                        n_agents, grid_h, grid_w);
+    }
+    const void* b1 = bias ? bias->b1 : nullptr;
+    const void* b2 = bias ? bias->b2 : nullptr;
+    if (misaligned(Q) || misaligned(K) || misaligned(V) || misaligned(out) || misaligned(workspace) ||
+        (A && misaligned(A)) || (b1 && misaligned(b1)) || (b2 && misaligned(b2)) ||
+        (dwc_weight && misaligned(dwc_weight)))
+        return fail(h, AA_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
+    if (out == Q || out == K || out == V) return fail(h, AA_ERR_INVALID_ARG, "out must not alias an input");
+    const WsLayout w = ws_layout(h, N, n_agents);
+    if (workspace_bytes < w.total)
+        return fail(h, AA_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", workspace_bytes, w.total);
+    DeviceGuard guard(h->cfg.device);
+    if (!guard.ok) return fail(h, AA_ERR_CUDA, "cannot select device %d", h->cfg.device);
+    h->launches = 0;
+    cudaStream_t st = (cudaStream_t)stream;
+    char* ws = static_cast<char*>(workspace);
+    const void* agents = A;
+    if (!A) {
+        if (int rc = do_pool(h, Q, grid_h, grid_w, p, p, ws + w.a_off, st)) return rc;
+        agents = ws + w.a_off;
+    }
+    void* va = ws + w.va_off;
+    if (int rc = do_aggregate(h, agents, K, V, b1, N, n_agents, va, reinterpret_cast<float*>(ws + w.part_off),
+                              reinterpret_cast<unsigned*>(ws + w.ticket_off), st))
+        return rc;
+    return do_broadcast(h, Q, agents, va, V, b2, dwc_weight, grid_h, grid_w, n_agents, out, st);
+}
+
+size_t agent_attn_staging_bytes(const agent_attn_handle* h, int grid_h, int grid_w, int n_agents) {
+    const size_t ws = agent_attn_workspace_bytes(h, grid_h, grid_w, n_agents);
+    if (!ws) return 0;
+    const size_t es = h->elem_bytes, slabs = (size_t)h->cfg.batch * h->cfg.heads;
+    const size_t N = (size_t)grid_h * grid_w, d = h->cfg.head_dim, n = n_agents, heads = h->cfg.heads;
+    const size_t qkv = align_up(slabs * N * d * es, 256);
+    return 4 * qkv + align_up(slabs * n * d * es, 256) + 2 * align_up(heads * n * N * es, 256) +
+           align_up(heads * d * 9 * es, 256) + align_up(ws, 256);
+}
+
+int agent_attn_forward_host(agent_attn_handle* h, const void* Q, const void* K, const void* V, const void* A,
+                            int grid_h, int grid_w, int n_agents, const agent_attn_bias* bias,
+                            const void* dwc_weight, void* out, void* staging, size_t staging_bytes, void* stream) {
+    if (!h) return AA_ERR_INVALID_ARG;
+    h->err[0] = 0;
+    if (!Q || !K || !V || !out || !staging) return fail(h, AA_ERR_INVALID_ARG, "null pointer");
+    const size_t need = agent_attn_staging_bytes(h, grid_h, grid_w, n_agents);
+    if (!need) return fail(h, AA_ERR_INVALID_ARG, "bad grid or agent count for this handle");
+    if (staging_bytes < need) return fail(h, AA_ERR_WORKSPACE, "staging has %zu bytes, %zu needed", staging_bytes, need);
+    if (misaligned(staging)) return fail(h, AA_ERR_INVALID_ARG, "staging must be 16-byte aligned");
+    DeviceGuard guard(h->cfg.device);
+    if (!guard.ok) return fail(h, AA_ERR_CUDA, "cannot select device %d", h->cfg.device);
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t es = h->elem_bytes, slabs = (size_t)h->cfg.batch * h->cfg.heads;
+    const size_t N = (size_t)grid_h * grid_w, d = h->cfg.head_dim, n = n_agents, heads = h->cfg.heads;
+    const size_t qkv_b = slabs * N * d * es, a_b = slabs * n * d * es, bias_b = heads * n * N * es, w_b = heads * d * 9 * es;
+    char* s = static_cast<char*>(staging);
+    char* dQ = s;                       s += align_up(qkv_b, 256);
+    char* dK = s;                       s += align_up(qkv_b, 256);
+    char* dV = s;                       s += align_up(qkv_b, 256);
+    char* dO = s;                       s += align_up(qkv_b, 256);
+    char* dA = s;                       s += align_up(a_b, 256);
+    char* dB1 = s;                      s += align_up(bias_b, 256);
+    char* dB2 = s;                      s += align_up(bias_b, 256);
+    char* dW = s;                       s += align_up(w_b, 256);
+    char* dWs = s;
+    const size_t ws_bytes = agent_attn_workspace_bytes(h, grid_h, grid_w, n_agents);
+    struct Cp { void* dst; const void* src; size_t bytes; } cps[] = {
+        {dQ, Q, qkv_b}, {dK, K, qkv_b}, {dV, V, qkv_b}, {dA, A, a_b},
+        {dB1, bias ? bias->b1 : nullptr, bias_b}, {dB2, bias ? bias->b2 : nullptr, bias_b}, {dW, dwc_weight, w_b}};
+    for (const Cp& c : cps) {
+        if (!c.src) continue;
+        cudaError_t e = cudaMemcpyAsync(c.dst, c.src, c.bytes, cudaMemcpyHostToDevice, st);
+        if (e != cudaSuccess) return fail(h, AA_ERR_CUDA, "host-to-device copy failed: %s", cudaGetErrorString(e));
+    }
+    agent_attn_bias db;
+    db.b1 = (bias && bias->b1) ? dB1 : nullptr;
+    db.b2 = (bias && bias->b2) ? dB2 : nullptr;
+    int rc = agent_attn_forward(h, dQ, dK, dV, A ? dA : nullptr, grid_h, grid_w, n_agents, bias ? &db : nullptr,
+                                dwc_weight ? dW : nullptr, dO, dWs, ws_bytes, stream);
+    if (rc) return rc;
+    cudaError_t e = cudaMemcpyAsync(out, dO, qkv_b, cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) return fail(h, AA_ERR_CUDA, "device-to-host copy failed: %s", cudaGetErrorString(e));
+    return AA_OK;
+}
+
+int agent_attn_query_status(agent_attn_handle* h, void* stream) {
+    if (!h) return AA_ERR_INVALID_ARG;
+    DeviceGuard guard(h->cfg.device);
+    if (!guard.ok) return fail(h, AA_ERR_CUDA, "cannot select device %d", h->cfg.device);
+    cudaStream_t st = (cudaStream_t)stream;
+    int word = 0;
+    cudaError_t e = cudaStreamSynchronize(st);
+    if (e == cudaSuccess) e = cudaMemcpy(&word, h->d_status, sizeof(int), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return fail(h, AA_ERR_CUDA, "status query failed: %s", cudaGetErrorString(e));
+    if (word != 0) {
+        cudaMemset(h->d_status, 0, sizeof(int));
+        return fail(h, AA_ERR_TIMEOUT, "a device-side bounded wait expired (code %d)", word);
+    }
+    return AA_OK;
+}
+
+}  // extern "C"

@@ -152,11 +152,4 @@ __device__ __forceinline__ void mma16816<__half>(float* c, const uint32_t* a, ui
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-// ------------------------------------------------------------------ split-partial layout
-// One partial per (slab, part): m[rows_pad], l[rows_pad], acc[rows_pad][dpad], all fp32, with m
-// and the logits in log2 units (logit * log2(e)), so weights are exp2(m_j - m).
-__host__ __device__ inline size_t partial_floats(int rows_pad, int dpad) {
-    return (size_t)rows_pad * (size_t)(dpad + 2);
-}
-
 }  // namespace aa

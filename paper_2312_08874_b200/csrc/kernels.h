@@ -9,6 +9,13 @@ namespace aa {
 
 enum DType { kF32 = 0, kBF16 = 1, kF16 = 2 };
 
+// Split-partial layout.  One partial per (slab, part): m[rows_pad], l[rows_pad],
+// acc[rows_pad][dpad], all fp32, with m and the logits in log2 units (logit * log2(e)), so the
+// merge weights are exp2(m_j - m).
+__host__ __device__ inline size_t partial_floats(int rows_pad, int dpad) {
+    return (size_t)rows_pad * (size_t)(dpad + 2);
+}
+
 // Agent pooling: A[slab][ay*pw+ax][:] = mean of Q over the window of pooled cell (ay, ax).
 struct PoolArgs {
     const void* q;      // [slabs][H*W][d]

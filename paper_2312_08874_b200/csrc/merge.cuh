@@ -1,6 +1,7 @@
 // Merge of split online-softmax partial states into V_A (Eq. 3, agent aggregation).
 #pragma once
 #include "common.cuh"
+#include "kernels.h"
 
 namespace aa {
 
