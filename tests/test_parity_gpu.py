@@ -1,0 +1,212 @@
+"""GPU-vs-oracle parity through the C ABI, element by element on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import agent_attention_oracle as orc
+from paper_2312_08874_b200 import AA_PATH_AUTO, AA_PATH_SIMT, WORKLOADS, AgentAttention, Workload, make_inputs
+from tests.parity_util import (assert_close, errors, gpu_forward, make_module, oracle_forward, to_dev, to_np)
+
+pytestmark = pytest.mark.gpu
+
+
+# ------------------------------------------------------------------ the five configurations
+@pytest.mark.parametrize("name", ["cfg1_deit_f32", "cfg2_deit_bf16", "cfg3_pvt_bf16", "cfg4_sd_f16",
+                                  "cfg5a_hires_bf16"])
+def test_full_size_configs_match_oracle(name):
+    w = WORKLOADS[name]
+    inp = make_inputs(w)
+    mod = make_module(w)
+    out = gpu_forward(mod, w, inp)
+    ref, a_ref, va_ref = oracle_forward(w, inp, return_intermediates=True)
+    assert_close(out, ref, w.dtype, name)
+    # intermediates through the step entry points
+    a = mod.pool(to_dev(inp["q"]), w.grid_h, w.grid_w, w.pool, w.pool)
+    assert_close(a, a_ref, w.dtype, name + " agents")
+    va = mod.aggregate(a, to_dev(inp["k"]), to_dev(inp["v"]), b1=to_dev(inp["b1"]))
+    torch.cuda.synchronize()
+    assert_close(va, va_ref, w.dtype, name + " agent features")
+
+
+def test_largest_config_matches_oracle_on_sampled_slabs():
+    w = WORKLOADS["cfg5b_hires_bf16"]
+    inp = make_inputs(w)
+    mod = make_module(w)
+    out = gpu_forward(mod, w, inp)
+    assert torch.isfinite(out.float()).all()
+    slabs = [(0, 0), (1, 5)]
+    for (b, h), ref in zip(slabs, oracle_forward(w, inp, slabs=slabs)):
+        assert_close(out[b:b + 1, h:h + 1], ref, w.dtype, f"cfg5b slab {(b, h)}")
+
+
+# ------------------------------------------------------- attention term must not hide under DWC
+@pytest.mark.parametrize("name", ["cfg3_pvt_bf16", "cfg5a_hires_bf16"])
+@pytest.mark.parametrize("variant", ["no_dwc", "shifted_v"])
+def test_attention_term_alone_and_with_nonzero_mean_values(name, variant):
+    w = WORKLOADS[name].scaled(batch=2)
+    inp = make_inputs(w)
+    if variant == "no_dwc":
+        inp["dwc"] = None
+    else:
+        inp["v"] = (inp["v"].float() + 1.0).to(inp["v"].dtype)
+    mod = make_module(w)
+    out = gpu_forward(mod, w, inp)
+    assert_close(out, oracle_forward(w, inp), w.dtype, f"{name} {variant}")
+
+
+# ------------------------------------------------------------------------------ shape sweep
+SWEEP = [
+    # batch heads H  W   d   pool dtype  bias  dwc
+    (2, 2, 7, 9, 8, 2, "f32", True, True),
+    (1, 3, 10, 10, 40, 4, "f32", True, True),
+    (2, 1, 5, 5, 128, 5, "f32", False, True),
+    (1, 2, 33, 17, 16, 3, "f32", True, False),
+    (3, 2, 14, 14, 64, 7, "bf16", True, True),
+    (2, 2, 9, 11, 40, 3, "f16", True, True),
+    (1, 2, 20, 20, 32, 5, "bf16", True, True),
+    (2, 1, 31, 29, 64, 6, "bf16", True, True),      # odd N: bias rows unaligned
+    (1, 1, 40, 40, 128, 9, "f16", True, True),
+    (1, 2, 36, 36, 96, 10, "bf16", False, True),
+    (1, 2, 48, 48, 8, 12, "bf16", True, True),
+    (1, 1, 64, 64, 24, 16, "f16", True, False),
+    (2, 1, 3, 3, 16, 1, "bf16", True, True),        # one agent, nine tokens
+    (1, 1, 1, 1, 64, 1, "bf16", True, True),        # a single token
+]
+
+
+@pytest.mark.parametrize("path", [AA_PATH_AUTO, AA_PATH_SIMT], ids=["auto", "simt"])
+@pytest.mark.parametrize("case", SWEEP, ids=[f"B{c[0]}h{c[1]}_{c[2]}x{c[3]}_d{c[4]}_p{c[5]}_{c[6]}" for c in SWEEP])
+def test_shape_sweep(case, path):
+    B, heads, H, W, d, pool, dtype, bias, dwc = case
+    w = Workload("sweep", B, heads, H, W, d, pool, dtype, bias, dwc, 1.0, seed=100 + H * W + d)
+    inp = make_inputs(w, bias_std=0.5, dwc_std=0.2)
+    mod = make_module(w, path=path)
+    out = gpu_forward(mod, w, inp)
+    ref, a_ref, va_ref = oracle_forward(w, inp, return_intermediates=True)
+    assert_close(out, ref, dtype, f"{case}")
+    a = mod.pool(to_dev(inp["q"]), H, W, pool, pool)
+    assert_close(a, a_ref, dtype, "agents")
+    va = mod.aggregate(a, to_dev(inp["k"]), to_dev(inp["v"]), b1=to_dev(inp["b1"]))
+    torch.cuda.synchronize()
+    assert_close(va, va_ref, dtype, "agent features")
+
+
+# ------------------------------------------------------------------- method-level properties
+def test_user_supplied_agents_non_square_count():
+    w = Workload("user_a", 2, 2, 12, 10, 64, 1, "bf16", True, True, 1.0, seed=7)
+    n = 23
+    inp = make_inputs(w)
+    g = torch.Generator().manual_seed(8)
+    agents = torch.randn((2, 2, n, 64), generator=g).to(torch.bfloat16)
+    b1 = (torch.randn((2, n, w.tokens), generator=g) * 0.3).to(torch.bfloat16)
+    b2 = (torch.randn((2, w.tokens, n), generator=g) * 0.3).to(torch.bfloat16)
+    mod = make_module(w, max_agents=n)
+    out = mod.forward(to_dev(inp["q"]), to_dev(inp["k"]), to_dev(inp["v"]), 12, 10, n, agents=agents.cuda(),
+                      b1=b1.cuda(), b2=b2.cuda(), dwc_weight=to_dev(inp["dwc"]))
+    torch.cuda.synchronize()
+    ref = orc.forward(to_np(inp["q"]), to_np(inp["k"]), to_np(inp["v"]), 12, 10, agents=to_np(agents),
+                      b1=to_np(b1), b2=to_np(b2), dwc_weight=to_np(inp["dwc"]), threads=4)
+    assert_close(out, ref, "bf16", "user agents")
+
+
+def test_separate_scales_follow_the_stable_diffusion_variant():
+    # App. C.1: larger scale in the broadcast only, shortcut k*V = centre-tap filter.
+    w = Workload("sd", 1, 2, 16, 16, 40, 4, "f16", False, True, 1.0 / np.sqrt(40.0), seed=9)
+    inp = make_inputs(w)
+    wd = torch.zeros((2, 40, 3, 3), dtype=torch.float16)
+    wd[:, :, 1, 1] = 0.075
+    inp["dwc"] = wd
+    s2 = 40.0 ** -0.15
+    mod = make_module(w, scale2=s2)
+    out = gpu_forward(mod, w, inp)
+    ref = oracle_forward(w, inp, scale2=s2)
+    assert_close(out, ref, "f16", "sd variant")
+    ref_default = oracle_forward(w, inp)
+    assert errors(out, ref_default)["rel_l2"] > 1e-2      # the scale really is used
+
+
+def test_constant_values_are_reproduced_and_single_agent_rows_are_identical():
+    w = Workload("const_v", 1, 1, 16, 16, 64, 4, "bf16", True, False, 1.0, seed=10)
+    inp = make_inputs(w)
+    const = (torch.arange(64, dtype=torch.float32) / 16.0 - 2.0).to(torch.bfloat16)
+    inp["v"] = const.expand(1, 1, 256, 64).contiguous()
+    out = gpu_forward(make_module(w), w, inp)
+    assert_close(out, to_np(inp["v"]), "bf16", "constant V", scale=0.5)
+    w1 = Workload("one_agent", 1, 2, 8, 8, 32, 1, "f16", False, False, 1.0, seed=11)
+    inp1 = make_inputs(w1)
+    out1 = gpu_forward(make_module(w1), w1, inp1)
+    assert torch.equal(out1, out1[:, :, :1].expand_as(out1))
+
+
+def test_key_value_permutation_changes_split_boundaries_not_the_result():
+    w = WORKLOADS["cfg3_pvt_bf16"].scaled(batch=1, bias=False, dwc=False)
+    inp = make_inputs(w)
+    mod = make_module(w)
+    out1 = gpu_forward(mod, w, inp).float()
+    perm = torch.randperm(w.tokens, generator=torch.Generator().manual_seed(3))
+    inp2 = dict(inp, k=inp["k"][:, :, perm].contiguous(), v=inp["v"][:, :, perm].contiguous())
+    out2 = gpu_forward(mod, w, inp2).float()
+    ref = oracle_forward(w, inp)
+    assert_close(out1, ref, "bf16", "original order")
+    assert_close(out2, ref, "bf16", "permuted keys")
+
+
+def test_zero_bias_tensors_equal_null_bias_and_runs_are_bitwise_repeatable():
+    w = WORKLOADS["cfg2_deit_bf16"].scaled(batch=4, bias=False)
+    inp = make_inputs(w)
+    mod = make_module(w)
+    out_null = gpu_forward(mod, w, inp).clone()
+    again = gpu_forward(mod, w, inp).clone()
+    assert torch.equal(out_null, again)
+    inp0 = dict(inp, b1=torch.zeros((w.heads, w.agents, w.tokens), dtype=torch.bfloat16),
+                b2=torch.zeros((w.heads, w.tokens, w.agents), dtype=torch.bfloat16))
+    out_zero = gpu_forward(mod, w, inp0)
+    assert torch.equal(out_null, out_zero)
+
+
+def test_large_logits_stay_finite():
+    w = Workload("hot", 1, 1, 16, 16, 64, 4, "bf16", False, False, 6.0, seed=12)
+    inp = make_inputs(w)
+    out = gpu_forward(make_module(w), w, inp)
+    ref = oracle_forward(w, inp)
+    assert torch.isfinite(out.float()).all()
+    assert_close(out, ref, "bf16", "large logits", scale=4.0)
+
+
+def test_forward_host_matches_forward():
+    w = WORKLOADS["cfg2_deit_bf16"].scaled(batch=3)
+    inp = make_inputs(w)
+    mod = make_module(w)
+    out_dev = gpu_forward(mod, w, inp).cpu()
+    pin = {k: (None if v is None else v.pin_memory()) for k, v in inp.items()}
+    out_host = mod.forward_host(pin["q"], pin["k"], pin["v"], w.grid_h, w.grid_w, w.agents, b1=pin["b1"],
+                                b2=pin["b2"], dwc_weight=pin["dwc"])
+    assert torch.equal(out_dev, out_host)
+    assert mod.last_launch_count() == 3
+    assert mod.query_status() == 0
+
+
+# --------------------------------------------------------------------------------- error paths
+def test_invalid_arguments_are_rejected_without_launching():
+    from paper_2312_08874_b200 import AgentAttnError
+    w = WORKLOADS["cfg1_deit_f32"]
+    inp = make_inputs(w)
+    mod = make_module(w)
+    q, k, v = to_dev(inp["q"]), to_dev(inp["k"]), to_dev(inp["v"])
+    with pytest.raises(AgentAttnError) as e:                # n not a square when pooling
+        mod.forward(q, k, v, 14, 14, 48)
+    assert e.value.status == 1
+    with pytest.raises(AgentAttnError) as e:                # more agents than the handle allows
+        mod.forward(q, k, v, 14, 14, 64)
+    assert e.value.status in (1, 2)
+    with pytest.raises(AgentAttnError) as e:                # workspace too small
+        mod.forward(q, k, v, 14, 14, 49, workspace=torch.empty(64, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == 3
+    with pytest.raises(AgentAttnError) as e:                # out aliases an input
+        mod.forward(q, k, v, 14, 14, 49, out=q)
+    assert e.value.status == 1
+    with pytest.raises(AgentAttnError):                     # unsupported head dim
+        AgentAttention(1, 1, 136, 64, 16, torch.bfloat16)
+    with pytest.raises(AgentAttnError):
+        AgentAttention(1, 1, 64, 64, 257, torch.bfloat16)
+    torch.cuda.synchronize()
