@@ -1,0 +1,315 @@
+#!/usr/bin/env python
+"""Benchmark of the Agent Attention forward pass (one JSON line on stdout, printed by rank 0).
+
+A step is one forward pass of the whole module (pool -> aggregation -> broadcast + DWC) over one
+batch of synthetic input of the headline shape (N = 3136 tokens on a 56x56 grid, n = 49 agents,
+d = 64, bf16, batch 64).  Inputs are resident in HBM before the timed region; the buffer sets
+rotate so that no step finds its inputs in L2.  `--impl reference` times the fp64 CPU oracle on
+the host cores instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2312_08874_b200 import WORKLOADS, make_inputs  # noqa: E402
+from paper_2312_08874_b200 import dist as pdist  # noqa: E402
+from paper_2312_08874_b200.workloads import TORCH_DTYPE  # noqa: E402
+
+METRIC = "agent-attention fwd tokens/s and % of HBM roofline at N=3136,n=49,d=64"
+UNIT = "tokens/s"
+DEFAULT_WORKLOAD = "cfg3_pvt_bf16"
+L2_BYTES = 126 * 1024 * 1024
+
+
+def measured_peaks():
+    """(HBM GB/s, source) from the generated peaks file, else the machine's fallback figure."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML (read-only) while a region runs."""
+
+    def __init__(self, index: int):
+        super().__init__(daemon=True)
+        self.index, self.samples, self.reasons, self.max_mhz = index, [], set(), None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+            getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+        }
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    bits = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    bits = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, nm in names.items():
+                    if bits & bit:
+                        self.reasons.add(nm)
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def stop(self):
+        self._stop_evt.set()
+        self.join(timeout=2.0)
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def flops_of(w) -> int:
+    """2 x the multiply-accumulates of Eq. 7 without the projections, per forward pass."""
+    per_slab = 8 * w.tokens * w.agents * w.head_dim + w.tokens * w.head_dim
+    if w.dwc:
+        per_slab += 18 * w.tokens * w.head_dim
+    return w.slabs * per_slab
+
+
+def oracle_sample_run(w, inp_np, threads):
+    from oracle import agent_attention_oracle as orc
+    t0 = time.perf_counter()
+    orc.forward(inp_np["q"], inp_np["k"], inp_np["v"], w.grid_h, w.grid_w, pool_hw=(w.pool, w.pool),
+                b1=inp_np["b1"], b2=inp_np["b2"], dwc_weight=inp_np["dwc"], threads=threads)
+    return time.perf_counter() - t0, orc.forward.last_threads
+
+
+def oracle_inputs(w):
+    inp = make_inputs(w)
+    return {k: (None if v is None else v.double().numpy()) for k, v in inp.items()}
+
+
+def run_reference(args, w):
+    """The oracle as it stands on the host cores; each step is one pass over a bounded sample."""
+    rank, _, world = pdist.env_rank()
+    if rank != 0:
+        return
+    from oracle import agent_attention_oracle as orc
+    threads = orc.max_threads()
+    # sample: as many whole batch entries as there are host threads, capped at the workload's batch
+    sample_batch = max(1, min(w.batch, threads // max(1, w.heads)))
+    ws = w.scaled(batch=sample_batch)
+    inp = oracle_inputs(ws)
+    for _ in range(args.warmup):
+        oracle_sample_run(ws, inp, threads)
+    t0 = time.perf_counter()
+    used = 1
+    for _ in range(args.steps):
+        _, used = oracle_sample_run(ws, inp, threads)
+    total = time.perf_counter() - t0
+    value = args.steps * ws.batch * ws.tokens / total
+    sample = f"{ws.batch} of {w.batch} batch entries ({ws.slabs} slabs) of {w.name} per step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": used, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=50)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
+    ap.add_argument("--e2e-steps", type=int, default=10)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--min-warmup-seconds", type=float, default=0.2)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    w = WORKLOADS[args.workload]
+
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    from paper_2312_08874_b200 import AgentAttention
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the forward pass has no CPU path")
+    rank, local_rank, world = pdist.init()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dt = TORCH_DTYPE[w.dtype]
+
+    # Rotating buffer sets: together more than 4x the L2, so no step re-reads a resident set.
+    set_bytes = w.algorithmic_bytes()
+    n_sets = max(2, -(-4 * L2_BYTES // set_bytes))
+    host = make_inputs(w, seed=w.seed + 1000 * rank)
+    sets = []
+    for s in range(n_sets):
+        g = torch.Generator(device="cpu").manual_seed(17 + s)
+        roll = int(torch.randint(1, w.tokens, (1,), generator=g))
+        d = {k: (None if v is None else v.to(dev)) for k, v in host.items()}
+        if s:  # distinct contents per set, same distribution (a roll along the token axis)
+            for k in ("q", "k", "v"):
+                d[k] = torch.roll(d[k], roll, dims=2).contiguous()
+        d["out"] = torch.empty_like(d["q"])
+        sets.append(d)
+    mod = AgentAttention(w.batch, w.heads, w.head_dim, w.tokens, w.agents, dt, device=local_rank)
+    ws = mod.workspace(w.grid_h, w.grid_w, w.agents)
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        d = sets[i % n_sets]
+        mod.forward(d["q"], d["k"], d["v"], w.grid_h, w.grid_w, w.agents, b1=d["b1"], b2=d["b2"],
+                    dwc_weight=d["dwc"], out=d["out"], workspace=ws, stream=stream)
+
+    # warm-up: W steps, and at least 0.2 s so that clocks have ramped
+    t_w = time.perf_counter()
+    i = 0
+    while i < args.warmup or time.perf_counter() - t_w < args.min_warmup_seconds:
+        step(i)
+        i += 1
+        if i % 64 == 0:
+            torch.cuda.synchronize()
+    torch.cuda.synchronize()
+    launches_per_step = mod.last_launch_count()
+
+    sampler = ClockSampler(local_rank)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    pdist.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    e0.record(stream)
+    for i in range(args.steps):
+        step(i)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    pdist.barrier()
+    clocks = sampler.stop()
+    ms_total = pdist.max_over_ranks(e0.elapsed_time(e1))
+    ms_step = ms_total / args.steps
+    tokens_per_step = world * w.batch * w.tokens
+    value = tokens_per_step / (ms_step * 1e-3)
+
+    # per-kernel durations: the same steps issued through the step-level entry points with an
+    # event between kernels (on the launching stream)
+    kb_steps = min(args.steps, 200)
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(kb_steps)]
+    a_buf = torch.empty((w.batch, w.heads, w.agents, w.head_dim), dtype=dt, device=dev)
+    va_buf = torch.empty_like(a_buf)
+    torch.cuda.synchronize()
+    for i in range(kb_steps):
+        d = sets[i % n_sets]
+        evs[i][0].record(stream)
+        mod.pool(d["q"], w.grid_h, w.grid_w, w.pool, w.pool, out=a_buf, stream=stream)
+        evs[i][1].record(stream)
+        mod.aggregate(a_buf, d["k"], d["v"], b1=d["b1"], out=va_buf, workspace=ws, stream=stream)
+        evs[i][2].record(stream)
+        mod.broadcast(d["q"], a_buf, va_buf, d["v"], w.grid_h, w.grid_w, b2=d["b2"], dwc_weight=d["dwc"],
+                      out=d["out"], stream=stream)
+        evs[i][3].record(stream)
+    torch.cuda.synchronize()
+    kern_ms = {nm: statistics.mean(evs[i][j].elapsed_time(evs[i][j + 1]) for i in range(kb_steps))
+               for j, nm in enumerate(("pool", "aggregate", "broadcast_dwc"))}
+    s = w.elem_bytes
+    unit = w.slabs * w.tokens * w.head_dim * s                       # one [B,h,N,d] tensor
+    bias_b = w.heads * w.agents * w.tokens * s if w.bias else 0
+    kern_bytes = {"pool": unit, "aggregate": 2 * unit + bias_b,
+                  "broadcast_dwc": unit + bias_b + (9 * w.heads * w.head_dim * s if w.dwc else 0)}
+    dominant = max(kern_ms, key=kern_ms.get)
+    peak, peak_src = measured_peaks()
+    dom_gbs = kern_bytes[dominant] / (kern_ms[dominant] * 1e-3) / 1e9
+    path_gbs = set_bytes / (ms_step * 1e-3) / 1e9
+    roofline = {
+        "bound": "hbm", "kernel": dominant, "achieved": dom_gbs, "peak": peak, "unit": "GB/s",
+        "frac": dom_gbs / peak, "traffic": None, "peak_source": peak_src,
+        "kernel_ms": kern_ms, "kernel_algorithmic_bytes": kern_bytes,
+        "path_achieved": path_gbs, "path_frac": path_gbs / peak, "path_frac_nominal_8TBs": path_gbs / 8000.0,
+        "path_algorithmic_bytes": set_bytes, "path_tflops": flops_of(w) / (ms_step * 1e-3) / 1e12,
+    }
+
+    # end to end through the host-buffer entry point: pinned inputs in, result out, every step
+    e2e = None
+    if args.e2e_steps > 0:
+        pin = {k: (None if v is None else v.pin_memory()) for k, v in host.items()}
+        out_h = torch.empty_like(pin["q"]).pin_memory()
+        for _ in range(2):
+            mod.forward_host(pin["q"], pin["k"], pin["v"], w.grid_h, w.grid_w, w.agents, b1=pin["b1"],
+                             b2=pin["b2"], dwc_weight=pin["dwc"], out=out_h, stream=stream)
+        pdist.barrier()
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for _ in range(args.e2e_steps):
+            mod.forward_host(pin["q"], pin["k"], pin["v"], w.grid_h, w.grid_w, w.agents, b1=pin["b1"],
+                             b2=pin["b2"], dwc_weight=pin["dwc"], out=out_h, stream=stream, synchronize=False)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        ms_e2e = pdist.max_over_ranks(e0.elapsed_time(e1)) / args.e2e_steps
+        h2d = sum(v.numel() * v.element_size() for v in pin.values() if v is not None)
+        e2e = {"value": tokens_per_step / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": out_h.numel() * out_h.element_size(), "ms_per_step": ms_e2e,
+               "steps": args.e2e_steps}
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        from oracle import agent_attention_oracle as orc
+        threads = orc.max_threads()
+        inp_np = {k: (None if v is None else v.double().numpy()) for k, v in host.items()}
+        best, used, reps, spent = None, 1, 0, 0.0
+        while reps < 3 or (spent < 2.0 and reps < 20):
+            t, used = oracle_sample_run(w, inp_np, threads)
+            best = t if best is None else min(best, t)
+            spent += t
+            reps += 1
+        cpu_baseline = {"value": w.batch * w.tokens / best, "unit": UNIT, "cores": used, "kind": "oracle",
+                        "sample": f"the full {w.name} batch ({w.slabs} slabs), best of {reps} passes, "
+                                  f"{spent * used:.0f} core-seconds in total"}
+
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
+            "config": {"workload": w.name, "batch_per_gpu": w.batch, "heads": w.heads, "tokens": w.tokens,
+                       "grid": [w.grid_h, w.grid_w], "head_dim": w.head_dim, "agents": w.agents,
+                       "bias": w.bias, "dwc": w.dwc,
+                       "l2": f"{n_sets} rotating buffer sets of {set_bytes / 1e6:.1f} MB (> 4x the 126 MB L2)",
+                       "parallelism": f"batch-sharded x{world}, no collective"},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
+            "roofline": roofline, "cpu_baseline": cpu_baseline,
+        }))
+    pdist.shutdown()
+
+
+if __name__ == "__main__":
+    main()
