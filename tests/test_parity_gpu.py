@@ -111,7 +111,7 @@ def test_user_supplied_agents_non_square_count():
 
 def test_separate_scales_follow_the_stable_diffusion_variant():
     # App. C.1: larger scale in the broadcast only, shortcut k*V = centre-tap filter.
-    w = Workload("sd", 1, 2, 16, 16, 40, 4, "f16", False, True, 1.0 / np.sqrt(40.0), seed=9)
+    w = Workload("sd", 1, 2, 16, 16, 40, 4, "f16", False, True, 1.0, seed=9)
     inp = make_inputs(w)
     wd = torch.zeros((2, 40, 3, 3), dtype=torch.float16)
     wd[:, :, 1, 1] = 0.075
@@ -122,7 +122,7 @@ def test_separate_scales_follow_the_stable_diffusion_variant():
     ref = oracle_forward(w, inp, scale2=s2)
     assert_close(out, ref, "f16", "sd variant")
     ref_default = oracle_forward(w, inp)
-    assert errors(out, ref_default)["rel_l2"] > 1e-2      # the scale really is used
+    assert errors(out, ref_default)["rel_l2"] > 2e-2      # the larger broadcast scale really is used
 
 
 def test_constant_values_are_reproduced_and_single_agent_rows_are_identical():
