@@ -157,6 +157,33 @@ int agent_attn_query_status(agent_attn_handle* h, void* stream);
 /* Number of kernels the most recent successful call on this handle enqueued. */
 int agent_attn_last_launch_count(const agent_attn_handle* h);
 
+/* Agent aggregation without any caller- or library-side allocation (the paper has no counterpart
+ * of this call; it computes exactly what agent_attn_aggregate computes).
+ *
+ * Who it is for: code that must not, or cannot, call cudaMalloc at the point where it needs the
+ * aggregation - for example a plugin running inside a host application that owns the memory pool,
+ * a real-time loop with a fixed memory budget, or a caller that only holds its input and output
+ * buffers and has nowhere to put a workspace.  agent_attn_aggregate needs a caller-provided
+ * workspace for the per-split partial softmax states; this variant keeps them in a fixed array
+ * inside the library image instead (agent_attn_static_scratch_bytes() = 32 MiB, resident on every
+ * GPU that loads the library until the process exits).
+ *
+ * Arguments as agent_attn_aggregate, minus the workspace.  Shapes whose partial states do not fit
+ * the fixed array are rejected with AA_ERR_WORKSPACE and a message that states both sizes.
+ * The first call on each device looks up the array's device address (cudaGetSymbolAddress) and
+ * caches it; make that first call outside any stream capture.  The call performs no cudaMalloc,
+ * cudaFree or other allocating routine.  All calls (all handles, all streams) share the one
+ * array: the arrival counters are cleared on `stream` at the start of each call and the partial
+ * states are fully rewritten, so nothing is carried over from the previous call, but two calls
+ * that overlap on the GPU (different streams, or different threads without ordering) race on it
+ * and must be serialised by the caller. */
+int agent_attn_aggregate_static(agent_attn_handle* h, const void* A, const void* K, const void* V,
+                                const void* b1, int n_tokens, int n_agents, void* VA_out,
+                                void* stream);
+
+/* Size in bytes of the fixed scratch array used by agent_attn_aggregate_static. */
+size_t agent_attn_static_scratch_bytes(void);
+
 #ifdef __cplusplus
 }
 #endif

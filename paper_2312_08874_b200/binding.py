@@ -24,7 +24,7 @@ EXPORTS = [
     "agent_attn_create", "agent_attn_destroy", "agent_attn_last_error", "agent_attn_workspace_bytes",
     "agent_attn_forward", "agent_attn_pool", "agent_attn_aggregate", "agent_attn_broadcast",
     "agent_attn_staging_bytes", "agent_attn_forward_host", "agent_attn_query_status",
-    "agent_attn_last_launch_count",
+    "agent_attn_last_launch_count", "agent_attn_aggregate_static", "agent_attn_static_scratch_bytes",
 ]
 
 
@@ -89,6 +89,10 @@ def load_library(build_if_missing: bool = True) -> ctypes.CDLL:
     lib.agent_attn_query_status.restype = ci
     lib.agent_attn_last_launch_count.argtypes = [vp]
     lib.agent_attn_last_launch_count.restype = ci
+    lib.agent_attn_aggregate_static.argtypes = [vp, vp, vp, vp, vp, ci, ci, vp, vp]
+    lib.agent_attn_aggregate_static.restype = ci
+    lib.agent_attn_static_scratch_bytes.argtypes = []
+    lib.agent_attn_static_scratch_bytes.restype = sz
     _lib = lib
     return lib
 
@@ -204,6 +208,25 @@ class AgentAttention:
         ws = self.workspace(1, N, n) if workspace is None else workspace
         self._check(self.lib.agent_attn_aggregate(self._h, _ptr(agents), _ptr(k), _ptr(v), _ptr(b1), N, n,
                                                   _ptr(out), _ptr(ws), ws.numel(), _stream_ptr(stream)))
+        return out
+
+    def aggregate_static(self, agents, k, v, b1=None, out=None, stream=None):
+        """`agent_attn_aggregate_static`: the aggregation for callers that cannot allocate.
+
+        Same result as `aggregate`, but the split partials live in the library's fixed 32 MiB
+        array instead of a workspace, so this call allocates nothing when `out` is given.
+        Calls that overlap on the GPU share that array and must be serialised.
+        """
+        B, h, d = self.batch, self.heads, self.head_dim
+        n, N = agents.shape[2], k.shape[2]
+        self._chk_tensor(agents, (B, h, n, d), "agents")
+        self._chk_tensor(k, (B, h, N, d), "k")
+        self._chk_tensor(v, (B, h, N, d), "v")
+        self._chk_tensor(b1, (h, n, N), "b1")
+        if out is None:
+            out = torch.empty_like(agents)
+        self._check(self.lib.agent_attn_aggregate_static(self._h, _ptr(agents), _ptr(k), _ptr(v), _ptr(b1),
+                                                         N, n, _ptr(out), _stream_ptr(stream)))
         return out
 
     def broadcast(self, q, agents, va, v, grid_h: int, grid_w: int, b2=None, dwc_weight=None, out=None,

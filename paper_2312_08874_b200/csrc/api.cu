@@ -7,6 +7,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 using namespace aa;
@@ -374,3 +375,69 @@ int agent_attn_query_status(agent_attn_handle* h, void* stream) {
 }
 
 }  // extern "C"
+
+// --------------------------------------------------------------------------------------------
+// Aggregation for callers that cannot allocate device memory.
+//
+// The split partials and arrival counters of the aggregation live in this fixed array, which is
+// part of the library image: every GPU that loads the library holds it until the process exits.
+// In host code `g_static_scratch` is only a stand-in symbol, not a device address; the address a
+// kernel may use is obtained once per device with cudaGetSymbolAddress (device current) below.
+#define AA_STATIC_SCRATCH_BYTES (32u * 1024u * 1024u)
+static __device__ __align__(256) unsigned char g_static_scratch[AA_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mu;
+void* g_static_ptr[kMaxDevices] = {nullptr};
+
+// Device address of the static scratch on the current device (looked up on first use).
+cudaError_t static_scratch_address(int device, void** out) {
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    if (device < 0 || device >= kMaxDevices) return cudaErrorInvalidDevice;
+    if (!g_static_ptr[device]) {
+        void* ptr = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+        if (e != cudaSuccess) return e;
+        g_static_ptr[device] = ptr;
+    }
+    *out = g_static_ptr[device];
+    return cudaSuccess;
+}
+}  // namespace
+
+extern "C" size_t agent_attn_static_scratch_bytes(void) { return AA_STATIC_SCRATCH_BYTES; }
+
+extern "C" int agent_attn_aggregate_static(agent_attn_handle* h, const void* A, const void* K, const void* V,
+                                           const void* b1, int n_tokens, int n_agents, void* VA_out,
+                                           void* stream) {
+    if (!h) return AA_ERR_INVALID_ARG;
+    h->err[0] = 0;
+    if (!A || !K || !V || !VA_out) return fail(h, AA_ERR_INVALID_ARG, "null pointer");
+    if (int rc = check_shape(h, n_tokens, n_agents)) return rc;
+    if (misaligned(A) || misaligned(K) || misaligned(V) || misaligned(VA_out) || (b1 && misaligned(b1)))
+        return fail(h, AA_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
+    // scratch layout: [partials | arrival counters], each 256-byte aligned
+    const size_t slabs = (size_t)h->cfg.batch * h->cfg.heads;
+    const AggPlan pl = plan_for(h, n_tokens, n_agents);
+    const size_t part_bytes = align_up(slabs * pl.parts * partial_floats(pl.rows_pad, pl.dpad) * sizeof(float), 256);
+    const size_t need = part_bytes + align_up(slabs * sizeof(unsigned), 256);
+    if (need > AA_STATIC_SCRATCH_BYTES)
+        return fail(h, AA_ERR_WORKSPACE,
+                    "this shape needs %zu bytes of scratch but the built-in scratch holds %u bytes; "
+                    "use agent_attn_aggregate with a caller-provided workspace",
+                    need, (unsigned)AA_STATIC_SCRATCH_BYTES);
+    DeviceGuard guard(h->cfg.device);
+    if (!guard.ok) return fail(h, AA_ERR_CUDA, "cannot select device %d", h->cfg.device);
+    void* base = nullptr;
+    cudaError_t e = static_scratch_address(h->cfg.device, &base);
+    if (e != cudaSuccess)
+        return fail(h, AA_ERR_CUDA, "cannot resolve the built-in scratch on device %d: %s", h->cfg.device,
+                    cudaGetErrorString(e));
+    h->launches = 0;
+    char* s = static_cast<char*>(base);
+    // do_aggregate clears the arrival counters on the stream before the kernel; the partials are
+    // fully rewritten by every call, so nothing else of the previous call's contents is read.
+    return do_aggregate(h, A, K, V, b1, n_tokens, n_agents, VA_out, reinterpret_cast<float*>(s),
+                        reinterpret_cast<unsigned*>(s + part_bytes), (cudaStream_t)stream);
+}
