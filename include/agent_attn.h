@@ -50,8 +50,10 @@ typedef enum {
 } aa_status;
 
 typedef enum {
-    AA_PATH_AUTO = 0,         /* tensor-core kernels for bf16/f16, fp32 FMA kernels for f32 */
-    AA_PATH_SIMT = 1          /* fp32 FMA kernels for every dtype (slow; for cross-checks) */
+    AA_PATH_AUTO = 0,         /* tensor-core kernels for bf16/f16 (one fused persistent kernel where the
+                                 shape allows it), fp32 FMA kernels for f32 */
+    AA_PATH_SIMT = 1,         /* fp32 FMA kernels for every dtype (slow; for cross-checks) */
+    AA_PATH_UNFUSED = 2       /* like AUTO, but always one kernel per step (pool, aggregate, broadcast) */
 } aa_path;
 
 typedef struct {

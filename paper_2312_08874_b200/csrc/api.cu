@@ -19,6 +19,8 @@ struct agent_attn_handle {
     int elem_bytes;
     int* d_status;          // one device word: bounded waits report here (none of the current kernels wait)
     int launches;
+    int fused_key[3];       // (grid_h, grid_w, n_agents) that fused_plan was made for
+    FusedPlan fused_plan;
     char err[512];
 };
 
@@ -53,7 +55,7 @@ AggPlan plan_for(const agent_attn_handle* h, int n_tokens, int n_agents) {
 struct WsLayout {
     size_t a_off, va_off, part_off, ticket_off, total;
 };
-WsLayout ws_layout(const agent_attn_handle* h, int n_tokens, int n_agents) {
+WsLayout ws_layout(const agent_attn_handle* h, int n_tokens, int n_agents, int grid_h = 0, int grid_w = 0) {
     const size_t slabs = (size_t)h->cfg.batch * h->cfg.heads;
     const AggPlan pl = plan_for(h, n_tokens, n_agents);
     const size_t av = align_up(slabs * n_agents * h->cfg.head_dim * h->elem_bytes, 256);
@@ -61,8 +63,15 @@ WsLayout ws_layout(const agent_attn_handle* h, int n_tokens, int n_agents) {
     w.a_off = 0;
     w.va_off = av;
     w.part_off = 2 * av;
-    w.ticket_off = w.part_off + align_up(slabs * pl.parts * partial_floats(pl.rows_pad, pl.dpad) * sizeof(float), 256);
-    w.total = w.ticket_off + align_up(slabs * sizeof(unsigned), 256);
+    // sized for either launch plan (per-step kernels or the fused kernel)
+    size_t part_floats = slabs * pl.parts * partial_floats(pl.rows_pad, pl.dpad);
+    if (grid_h > 0 && h->cfg.path == AA_PATH_AUTO) {
+        const size_t fused_floats = slabs * (size_t)fused_parts_per_slab(h->cfg.dtype, grid_h, grid_w, h->cfg.head_dim, n_agents) *
+                                    partial_floats(64, h->cfg.head_dim);
+        if (part_floats < fused_floats) part_floats = fused_floats;
+    }
+    w.ticket_off = w.part_off + align_up(part_floats * sizeof(float), 256);
+    w.total = w.ticket_off + align_up(fused_counter_words((int)slabs) * sizeof(unsigned), 256);
     return w;
 }
 
@@ -149,7 +158,7 @@ int agent_attn_create(agent_attn_handle** out, const agent_attn_config* cfg) {
         cfg->max_agents <= 0 || cfg->scale1 < 0.f || cfg->scale2 < 0.f)
         return AA_ERR_INVALID_ARG;
     if (cfg->dtype != AA_F32 && cfg->dtype != AA_BF16 && cfg->dtype != AA_F16) return AA_ERR_UNSUPPORTED;
-    if (cfg->path != AA_PATH_AUTO && cfg->path != AA_PATH_SIMT) return AA_ERR_UNSUPPORTED;
+    if (cfg->path != AA_PATH_AUTO && cfg->path != AA_PATH_SIMT && cfg->path != AA_PATH_UNFUSED) return AA_ERR_UNSUPPORTED;
     const int es = cfg->dtype == AA_F32 ? 4 : 2;
     if (cfg->head_dim > 128 || cfg->head_dim < 8 || (cfg->head_dim * es) % 16 != 0) return AA_ERR_UNSUPPORTED;
     if (cfg->max_agents > 256) return AA_ERR_UNSUPPORTED;
@@ -200,7 +209,7 @@ int agent_attn_last_launch_count(const agent_attn_handle* h) { return h ? h->lau
 size_t agent_attn_workspace_bytes(const agent_attn_handle* h, int grid_h, int grid_w, int n_agents) {
     if (!h || grid_h <= 0 || grid_w <= 0 || n_agents <= 0) return 0;
     if ((long long)grid_h * grid_w > h->cfg.max_tokens || n_agents > h->cfg.max_agents) return 0;
-    return ws_layout(h, grid_h * grid_w, n_agents).total;
+    return ws_layout(h, grid_h * grid_w, n_agents, grid_h, grid_w).total;
 }
 
 int agent_attn_pool(agent_attn_handle* h, const void* Q, int grid_h, int grid_w, int pool_h, int pool_w,
@@ -282,7 +291,7 @@ int agent_attn_forward(agent_attn_handle* h, const void* Q, const void* K, const
         (dwc_weight && misaligned(dwc_weight)))
         return fail(h, AA_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
     if (out == Q || out == K || out == V) return fail(h, AA_ERR_INVALID_ARG, "out must not alias an input");
-    const WsLayout w = ws_layout(h, N, n_agents);
+    const WsLayout w = ws_layout(h, N, n_agents, grid_h, grid_w);
     if (workspace_bytes < w.total)
         return fail(h, AA_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", workspace_bytes, w.total);
     DeviceGuard guard(h->cfg.device);
@@ -290,6 +299,32 @@ int agent_attn_forward(agent_attn_handle* h, const void* Q, const void* K, const
     h->launches = 0;
     cudaStream_t st = (cudaStream_t)stream;
     char* ws = static_cast<char*>(workspace);
+    if (!A && h->cfg.path == AA_PATH_AUTO && h->cfg.dtype != AA_F32) {
+        // one persistent kernel for the whole module where the shape allows it
+        if (h->fused_key[0] != grid_h || h->fused_key[1] != grid_w || h->fused_key[2] != n_agents) {
+            h->fused_plan = plan_fused(h->cfg.dtype, h->cfg.batch * h->cfg.heads, grid_h, grid_w, h->cfg.head_dim,
+                                       n_agents, h->sm_count);
+            h->fused_key[0] = grid_h; h->fused_key[1] = grid_w; h->fused_key[2] = n_agents;
+        }
+        if (h->fused_plan.ok) {
+            const int slabs = h->cfg.batch * h->cfg.heads;
+            unsigned* counters = reinterpret_cast<unsigned*>(ws + w.ticket_off);
+            cudaError_t e = cudaMemsetAsync(counters, 0, fused_counter_words(slabs) * sizeof(unsigned), st);
+            if (e != cudaSuccess) return fail(h, AA_ERR_CUDA, "counter reset failed: %s", cudaGetErrorString(e));
+            FusedArgs fa;
+            memset(&fa, 0, sizeof(fa));
+            fa.q = Q; fa.k = K; fa.v = V; fa.b1 = b1; fa.b2 = b2; fa.dwc_w = dwc_weight; fa.out = out;
+            fa.a_ws = ws + w.a_off; fa.va_ws = ws + w.va_off;
+            fa.partials = reinterpret_cast<float*>(ws + w.part_off);
+            fa.counters = counters; fa.status = h->d_status;
+            fa.slabs = slabs; fa.heads = h->cfg.heads; fa.H = grid_h; fa.W = grid_w; fa.d = h->cfg.head_dim;
+            fa.n = n_agents; fa.p = p; fa.scale1 = h->scale1; fa.scale2 = h->scale2; fa.plan = h->fused_plan;
+            e = launch_fused(h->cfg.dtype, fa, st);
+            if (e != cudaSuccess) return fail(h, AA_ERR_CUDA, "fused launch failed: %s", cudaGetErrorString(e));
+            h->launches = 1;
+            return AA_OK;
+        }
+    }
     const void* agents = A;
     if (!A) {
         if (int rc = do_pool(h, Q, grid_h, grid_w, p, p, ws + w.a_off, st)) return rc;

@@ -60,4 +60,36 @@ cudaError_t launch_broadcast_simt(int dtype, const AttnArgs& p, cudaStream_t st)
 cudaError_t launch_aggregate_mma(int dtype, const AttnArgs& p, const AggPlan& plan, cudaStream_t st);
 cudaError_t launch_broadcast_mma(int dtype, const AttnArgs& p, cudaStream_t st);
 
+// Whole module (Eq. 6) in one persistent kernel for small agent counts (n <= 64, d in {32, 64},
+// block pooling, W <= 64).  Blocks take tasks from a device-side queue: "G" tasks pool their token
+// range of Q, publish those agent rows, wait for the slab's other G tasks, and aggregate their
+// range of K/V; "B" tasks wait for the slab's merged V_A and do the broadcast + DWC for one
+// 128-token tile.  A slab's B tasks follow its G tasks closely, so Q and V are re-read from L2.
+struct FusedPlan {
+    bool ok;            // shape is eligible
+    int g_tasks;        // G tasks per slab
+    int rows_per_g;     // grid rows per G task (a multiple of the pooling window height)
+    int b_tasks;        // B tasks (128-token tiles) per slab
+    int lag;            // slabs between a slab's G tasks and its B tasks in the queue
+    int grid;           // resident blocks
+    int parts;          // partial states per slab
+    size_t smem;        // dynamic shared memory per block
+};
+struct FusedArgs {
+    const void *q, *k, *v, *b1, *b2, *dwc_w;
+    void* out;
+    void* a_ws;           // [slabs][n][d] agents (written by G tasks)
+    void* va_ws;          // [slabs][n][d] agent features (written by the merging G task)
+    float* partials;      // [slabs][parts][partial_floats(64, d)]
+    unsigned* counters;   // zero on entry: a_count[slabs] | tickets[slabs] | va_ready[slabs] | queue[1]
+    int* status;          // device status word: set when a bounded wait gives up
+    int slabs, heads, H, W, d, n, p;
+    float scale1, scale2;
+    FusedPlan plan;
+};
+FusedPlan plan_fused(int dtype, int slabs, int H, int W, int d, int n_agents, int sm_count);
+cudaError_t launch_fused(int dtype, const FusedArgs& a, cudaStream_t st);
+int fused_parts_per_slab(int dtype, int H, int W, int d, int n_agents);   // 0 if the shape is not eligible
+inline size_t fused_counter_words(int slabs) { return 3 * (size_t)slabs + 4; }
+
 }  // namespace aa

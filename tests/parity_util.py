@@ -71,4 +71,5 @@ def gpu_forward(mod: AgentAttention, w: Workload, inp) -> torch.Tensor:
     out = mod.forward(to_dev(inp["q"]), to_dev(inp["k"]), to_dev(inp["v"]), w.grid_h, w.grid_w, w.agents,
                       b1=to_dev(inp["b1"]), b2=to_dev(inp["b2"]), dwc_weight=to_dev(inp["dwc"]))
     torch.cuda.synchronize()
+    assert mod.query_status() == 0, "a device-side bounded wait expired"
     return out

@@ -4,19 +4,22 @@ import pytest
 import torch
 
 from oracle import agent_attention_oracle as orc
-from paper_2312_08874_b200 import AA_PATH_AUTO, AA_PATH_SIMT, WORKLOADS, AgentAttention, Workload, make_inputs
+from paper_2312_08874_b200 import AA_PATH_AUTO, AA_PATH_SIMT, AA_PATH_UNFUSED, WORKLOADS, AgentAttention, Workload, make_inputs
 from tests.parity_util import (assert_close, errors, gpu_forward, make_module, oracle_forward, to_dev, to_np)
 
 pytestmark = pytest.mark.gpu
 
 
 # ------------------------------------------------------------------ the five configurations
+@pytest.mark.parametrize("path", [AA_PATH_AUTO, AA_PATH_UNFUSED], ids=["auto", "unfused"])
 @pytest.mark.parametrize("name", ["cfg1_deit_f32", "cfg2_deit_bf16", "cfg3_pvt_bf16", "cfg4_sd_f16",
                                   "cfg5a_hires_bf16"])
-def test_full_size_configs_match_oracle(name):
+def test_full_size_configs_match_oracle(name, path):
     w = WORKLOADS[name]
+    if path == AA_PATH_UNFUSED and name not in ("cfg2_deit_bf16", "cfg3_pvt_bf16"):
+        pytest.skip("only the small-agent-count configurations have two launch plans")
     inp = make_inputs(w)
-    mod = make_module(w)
+    mod = make_module(w, path=path)
     out = gpu_forward(mod, w, inp)
     ref, a_ref, va_ref = oracle_forward(w, inp, return_intermediates=True)
     assert_close(out, ref, w.dtype, name)
@@ -69,12 +72,16 @@ SWEEP = [
     (1, 2, 36, 36, 96, 10, "bf16", False, True),
     (1, 2, 48, 48, 8, 12, "bf16", True, True),
     (1, 1, 64, 64, 24, 16, "f16", True, False),
+    (5, 2, 28, 56, 64, 7, "bf16", True, True),      # fused path: H != W, ragged last 128-token tile
+    (40, 2, 64, 64, 32, 8, "f16", True, True),      # fused path: widest grid, n = 64, more slabs than lag
+    (3, 1, 56, 56, 64, 7, "bf16", False, False),    # fused path: no bias, no DWC
+    (7, 3, 14, 14, 64, 7, "f16", True, True),       # fused path: one G task per slab, odd-head bias misaligned
     (2, 1, 3, 3, 16, 1, "bf16", True, True),        # one agent, nine tokens
     (1, 1, 1, 1, 64, 1, "bf16", True, True),        # a single token
 ]
 
 
-@pytest.mark.parametrize("path", [AA_PATH_AUTO, AA_PATH_SIMT], ids=["auto", "simt"])
+@pytest.mark.parametrize("path", [AA_PATH_AUTO, AA_PATH_UNFUSED, AA_PATH_SIMT], ids=["auto", "unfused", "simt"])
 @pytest.mark.parametrize("case", SWEEP, ids=[f"B{c[0]}h{c[1]}_{c[2]}x{c[3]}_d{c[4]}_p{c[5]}_{c[6]}" for c in SWEEP])
 def test_shape_sweep(case, path):
     B, heads, H, W, d, pool, dtype, bias, dwc = case
@@ -183,7 +190,7 @@ def test_forward_host_matches_forward():
     out_host = mod.forward_host(pin["q"], pin["k"], pin["v"], w.grid_h, w.grid_w, w.agents, b1=pin["b1"],
                                 b2=pin["b2"], dwc_weight=pin["dwc"])
     assert torch.equal(out_dev, out_host)
-    assert mod.last_launch_count() == 3
+    assert mod.last_launch_count() == 1            # the fused persistent kernel
     assert mod.query_status() == 0
 
 
