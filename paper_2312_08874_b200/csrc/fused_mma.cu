@@ -20,6 +20,7 @@
 #include "kernels.h"
 #include "merge.cuh"
 
+#include <cstdlib>
 #include <cstring>
 
 namespace aa {
@@ -31,6 +32,8 @@ constexpr int NT = 256;           // threads per block (8 warps)
 constexpr int RP = 64;            // agent rows, padded
 constexpr int STAGES = 3;
 constexpr int MAXW = 64;          // widest grid the halo buffer is sized for
+constexpr int MINW = 8;
+constexpr int kHaloTokens = 264;  // max over 8 <= W <= 64 of (R + 2)(W + 2), R = min(16, 128 / W)
 constexpr unsigned kSpinLimit = 1u << 20;
 constexpr int kTimeoutAgents = 1, kTimeoutFeatures = 2;
 
@@ -63,7 +66,8 @@ template <int DK> struct FusedSmem {
     static constexpr int PB = KT + 8;                               // B1 tile row pitch
     static constexpr size_t kA = (size_t)RP * PA * 2;               // resident agents
     static constexpr size_t kVA = kA;                               // resident agent features
-    static constexpr size_t kCommon = kA + kVA;
+    static constexpr size_t kW = (size_t)9 * DK * 4;                // filter taps [9][DK] fp32
+    static constexpr size_t kCommon = kA + kVA + kW;
     // G layout
     static constexpr size_t kTile = (size_t)KT * PA * 2;
     static constexpr size_t kB1 = (size_t)RP * PB * 2;
@@ -72,10 +76,9 @@ template <int DK> struct FusedSmem {
     // B layout
     static constexpr int PO = DK + 8;                               // fp32 patch pitch (floats)
     static constexpr size_t kPatch = (size_t)8 * 16 * PO * 4;       // per-warp [16][PO] fp32 (Q rows alias it)
-    static constexpr size_t kHalo = (size_t)(QT + 2 * MAXW + 2) * DK * 2;
-    static constexpr size_t kB2 = (size_t)QT * RP * 2;
-    static constexpr size_t kW = (size_t)9 * DK * 4;
-    static constexpr size_t kB = kPatch + kHalo + kB2 + kW;
+    static constexpr size_t kHalo = (size_t)kHaloTokens * DK * 2;   // (rows+2) x (W+2) tokens, see plan
+    static constexpr size_t kB2 = (size_t)QT * RP * 2 + 16;         // + one spare vector: pairs are read as two words
+    static constexpr size_t kB = kPatch + kHalo + kB2;
     static constexpr size_t kTotal = kCommon + (kG > kB ? kG : kB);
 };
 
@@ -186,6 +189,11 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
         }
     };
 
+    // column DK of every V tile row holds 1, so the P.V product also yields the row sums of P
+    if (tid < STAGES * KT) {
+        const uint32_t one = pack2<T>(1.f, 0.f);
+        *reinterpret_cast<uint4*>(stage_v(tid / KT) + (tid % KT) * PA + DK) = make_uint4(one, 0u, 0u, 0u);
+    }
     // 1. start the ring
     for (int s = 0; s < STAGES - 1; ++s) {
         if (s < tiles) load_tile(s, s);
@@ -243,15 +251,14 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
 
     const int g = lane >> 2, t4 = lane & 3;
     const int r0 = wm * 16, kw0 = wk * KW;
-    const float scale_log2 = p.scale1 * kLog2e;
     uint32_t af[DK / 16][4];
 #pragma unroll
     for (int ks = 0; ks < DK / 16; ++ks)
         ldmatrix_x4(af[ks][0], af[ks][1], af[ks][2], af[ks][3],
                     sA + (r0 + (lane & 7) + ((lane >> 3) & 1) * 8) * PA + ks * 16 + (lane >> 4) * 8);
 
-    float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
-    float acc[DK / 8][4];
+    float m0 = -INFINITY, m1 = -INFINITY;            // running row maxima, natural units
+    float acc[DK / 8][4], accl[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
     for (int j = 0; j < DK / 8; ++j) { acc[j][0] = acc[j][1] = acc[j][2] = acc[j][3] = 0.f; }
 
@@ -281,21 +288,31 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
                 mma16816<T>(sc[2 * np + 1], af[ks], b2, b3);
             }
         }
+        // logits in natural units: t = scale1 * a.k + b1
         float mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll
         for (int j = 0; j < KW / 8; ++j) {
             const int col = kw0 + 8 * j + 2 * t4;
-            float b00 = 0.f, b01 = 0.f, b10 = 0.f, b11 = 0.f;
+            float2 ba = make_float2(0.f, 0.f), bb = make_float2(0.f, 0.f);
             if (has_bias) {
-                const float2 u0 = unpack2<T>(*reinterpret_cast<const uint32_t*>(sB + (r0 + g) * PB + col));
-                const float2 u1 = unpack2<T>(*reinterpret_cast<const uint32_t*>(sB + (r0 + g + 8) * PB + col));
-                b00 = u0.x * kLog2e; b01 = u0.y * kLog2e; b10 = u1.x * kLog2e; b11 = u1.y * kLog2e;
+                ba = unpack2<T>(*reinterpret_cast<const uint32_t*>(sB + (r0 + g) * PB + col));
+                bb = unpack2<T>(*reinterpret_cast<const uint32_t*>(sB + (r0 + g + 8) * PB + col));
             }
-            const bool ok0 = (c0 + col) < t_end, ok1 = (c0 + col + 1) < t_end;
-            sc[j][0] = ok0 ? fmaf(sc[j][0], scale_log2, b00) : -INFINITY;
-            sc[j][1] = ok1 ? fmaf(sc[j][1], scale_log2, b01) : -INFINITY;
-            sc[j][2] = ok0 ? fmaf(sc[j][2], scale_log2, b10) : -INFINITY;
-            sc[j][3] = ok1 ? fmaf(sc[j][3], scale_log2, b11) : -INFINITY;
+            sc[j][0] = fmaf(sc[j][0], p.scale1, ba.x);
+            sc[j][1] = fmaf(sc[j][1], p.scale1, ba.y);
+            sc[j][2] = fmaf(sc[j][2], p.scale1, bb.x);
+            sc[j][3] = fmaf(sc[j][3], p.scale1, bb.y);
+        }
+        if (c0 + KT > t_end) {          // ragged last tile of the range: keys beyond it do not exist
+#pragma unroll
+            for (int j = 0; j < KW / 8; ++j) {
+                const int key = c0 + kw0 + 8 * j + 2 * t4;
+                if (key >= t_end)     { sc[j][0] = -INFINITY; sc[j][2] = -INFINITY; }
+                if (key + 1 >= t_end) { sc[j][1] = -INFINITY; sc[j][3] = -INFINITY; }
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < KW / 8; ++j) {
             mx0 = fmaxf(mx0, fmaxf(sc[j][0], sc[j][1]));
             mx1 = fmaxf(mx1, fmaxf(sc[j][2], sc[j][3]));
         }
@@ -306,21 +323,20 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
         const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
         const float base0 = (mn0 == -INFINITY) ? 0.f : mn0;
         const float base1 = (mn1 == -INFINITY) ? 0.f : mn1;
-        const float corr0 = fast_exp2(m0 - base0), corr1 = fast_exp2(m1 - base1);
+        const float corr0 = fast_exp2((m0 - base0) * kLog2e), corr1 = fast_exp2((m1 - base1) * kLog2e);
+        const float nb0 = -base0 * kLog2e, nb1 = -base1 * kLog2e;
         m0 = mn0; m1 = mn1;
-        l0 *= corr0; l1 *= corr1;
+        accl[0] *= corr0; accl[1] *= corr0; accl[2] *= corr1; accl[3] *= corr1;
 #pragma unroll
         for (int j = 0; j < DK / 8; ++j) {
             acc[j][0] *= corr0; acc[j][1] *= corr0; acc[j][2] *= corr1; acc[j][3] *= corr1;
         }
+        // probabilities rounded to the operand type; their row sums come out of the same MMA
         uint32_t pk[KW / 8][2];
 #pragma unroll
         for (int j = 0; j < KW / 8; ++j) {
-            pk[j][0] = pack2<T>(fast_exp2(sc[j][0] - base0), fast_exp2(sc[j][1] - base0));
-            pk[j][1] = pack2<T>(fast_exp2(sc[j][2] - base1), fast_exp2(sc[j][3] - base1));
-            const float2 q0 = unpack2<T>(pk[j][0]), q1 = unpack2<T>(pk[j][1]);
-            l0 += q0.x + q0.y;
-            l1 += q1.x + q1.y;
+            pk[j][0] = pack2<T>(fast_exp2(fmaf(sc[j][0], kLog2e, nb0)), fast_exp2(fmaf(sc[j][1], kLog2e, nb0)));
+            pk[j][1] = pack2<T>(fast_exp2(fmaf(sc[j][2], kLog2e, nb1)), fast_exp2(fmaf(sc[j][3], kLog2e, nb1)));
         }
 #pragma unroll
         for (int kk = 0; kk < KW / 16; ++kk) {
@@ -333,14 +349,16 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
                 mma16816<T>(acc[2 * np], pa, b0, b1);
                 mma16816<T>(acc[2 * np + 1], pa, b2, b3);
             }
+            uint32_t o0, o1;
+            ldmatrix_x2_trans(o0, o1, sV + (kw0 + kk * 16 + (lane & 15)) * PA + DK);
+            mma16816<T>(accl, pa, o0, o1);
         }
     }
     cp_async_wait<0>();
 
-    l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
-    l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
-    l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
-    l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+    // row sums sit in column DK of the product: lanes with t4 == 0 hold them
+    const float l0 = __shfl_sync(0xffffffffu, accl[0], lane & ~3);
+    const float l1 = __shfl_sync(0xffffffffu, accl[2], lane & ~3);
 
     // 6. partial state of this warp; the slab's last G task merges and raises the slab's flag
     const int parts = p.plan.parts;
@@ -348,7 +366,7 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
     float* slab_parts = p.partials + (size_t)slab * parts * pf;
     float* part = slab_parts + (size_t)(sub * NWK + wk) * pf;
     if (t4 == 0) {
-        part[r0 + g] = m0;      part[r0 + g + 8] = m1;
+        part[r0 + g] = m0 * kLog2e; part[r0 + g + 8] = m1 * kLog2e;     // the merge works in log2 units
         part[RP + r0 + g] = l0; part[RP + r0 + g + 8] = l1;
     }
     float* pacc = part + 2 * RP;
@@ -367,59 +385,82 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
 }
 
 // ---------------------------------------------------------------------------------- B task
+// One tile = R whole grid rows (R*W <= 128 tokens).  Warps 0..7 own 16 query rows each for the
+// attention part and leave their fp32 result in the patch; then all threads switch to a
+// (row, 4-channel group, x-segment) mapping and slide a 3x3 window along x over the V rows held in
+// shared memory (with explicit zero columns at x = -1 and x = W and zero rows outside the grid),
+// add the depthwise term (Eq. 6), round once and store.
 template <typename T, int DK>
-__device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int tile, unsigned char* smem) {
+__device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int tile, unsigned char* smem,
+                                           int* s_whead) {
     using L = FusedSmem<DK>;
     constexpr int PA = L::PA, PO = L::PO;
     constexpr int cpr = DK / 8;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int head = slab % p.heads;
     const int N = p.H * p.W, n = p.n, W = p.W, H = p.H;
-    const int n_pad = (n + 15) & ~15;
-    const int q0 = tile * QT;
+    const int n8 = (n + 7) >> 3;                      // logit column tiles that hold agents
+    const int n16 = (n + 15) >> 4;
+    const int R = p.plan.rows_per_b;
+    const int y0 = tile * R;
+    const int rows = min(R, H - y0);
+    const int q0 = y0 * W, TQ = rows * W;            // tokens of this tile
     const int i0 = q0 + warp * 16;
+    const bool warp_active = warp * 16 < TQ;
     const bool has_dwc = p.dwc_w != nullptr;
     const bool has_b2 = p.b2 != nullptr;
+    const int HP = W + 2;                             // halo row pitch in tokens
 
     T* sA = reinterpret_cast<T*>(smem);
     T* sVA = reinterpret_cast<T*>(smem + L::kA);
     unsigned char* base = smem + L::kCommon;
-    float* sPatch = reinterpret_cast<float*>(base) + (size_t)warp * 16 * PO;
-    T* sQ = reinterpret_cast<T*>(sPatch);                           // [16][PA], aliases the patch
-    T* sH = reinterpret_cast<T*>(base + L::kPatch);                 // V rows h0..h1, [tokens][DK]
-    T* sB2 = reinterpret_cast<T*>(base + L::kPatch + L::kHalo);     // [rows][n] flat
-    float* sW = reinterpret_cast<float*>(base + L::kPatch + L::kHalo + L::kB2);   // [9][DK]
+    float* sPatchAll = reinterpret_cast<float*>(base);               // [128][PO] fp32
+    float* sPatch = sPatchAll + (size_t)warp * 16 * PO;
+    T* sQ = reinterpret_cast<T*>(sPatch);                            // [16][PA], aliases the warp's patch rows
+    T* sH = reinterpret_cast<T*>(base + L::kPatch);                  // [(rows+2)][W+2][DK] V rows with zero borders
+    T* sB2 = reinterpret_cast<T*>(base + L::kPatch + L::kHalo);      // [TQ][n] flat
+    float* sW = reinterpret_cast<float*>(smem + L::kA + L::kVA);                  // [9][DK], survives G tasks
 
     const T* gQ = static_cast<const T*>(p.q) + (size_t)slab * N * DK;
     const T* gV = static_cast<const T*>(p.v) + (size_t)slab * N * DK;
-    const int h0 = max(0, q0 - W - 1), h1 = min(N, q0 + QT + W + 1);
 
     // 1. loads that do not depend on the aggregation
-    for (int e = lane; e < 16 * cpr; e += 32) {
-        const int r = e / cpr, c = e - r * cpr;
-        const bool ok = (i0 + r) < N;
-        cp_async16(sQ + r * PA + c * 8, gQ + (ok ? ((size_t)(i0 + r) * DK + c * 8) : 0), ok ? 16 : 0);
+    if (warp_active) {
+        for (int e = lane; e < 16 * cpr; e += 32) {
+            const int r = e / cpr, c = e - r * cpr;
+            const bool ok = (warp * 16 + r) < TQ;
+            cp_async16(sQ + r * PA + c * 8, gQ + (ok ? ((size_t)(i0 + r) * DK + c * 8) : 0), ok ? 16 : 0);
+        }
     }
     if (has_dwc) {
-        const int chunks = (h1 - h0) * cpr;
-        const T* src = gV + (size_t)h0 * DK;
-        for (int e = tid; e < chunks; e += NT) cp_async16(sH + e * 8, src + e * 8, 16);
-        const T* w = static_cast<const T*>(p.dwc_w) + (size_t)head * DK * 9;
-        for (int e = tid; e < 9 * DK; e += NT) {
-            const int c = e / 9, tap = e - c * 9;
-            sW[tap * DK + c] = Elem<T>::to_f32(w[e]);
+        for (int hr = 0; hr < rows + 2; ++hr) {
+            const int y = y0 - 1 + hr;
+            const bool ok = (y >= 0) && (y < H);
+            const T* src = gV + (ok ? (size_t)y * W * DK : 0);
+            T* dst = sH + ((size_t)hr * HP + 1) * DK;
+            for (int e = tid; e < W * cpr; e += NT) cp_async16(dst + e * 8, src + e * 8, ok ? 16 : 0);
+            if (tid < 2 * cpr) {       // zero columns x = -1 and x = W
+                const int side = tid / cpr, c = tid - side * cpr;
+                *(reinterpret_cast<uint4*>(sH + ((size_t)hr * HP + (side ? W + 1 : 0)) * DK) + c) = make_uint4(0, 0, 0, 0);
+            }
+        }
+        if (*s_whead != head) {       // filter taps change only with the head
+            const T* w = static_cast<const T*>(p.dwc_w) + (size_t)head * DK * 9;
+            for (int e = tid; e < 9 * DK; e += NT) {
+                const int c = e / 9, tap = e - c * 9;
+                sW[tap * DK + c] = Elem<T>::to_f32(w[e]);
+            }
         }
     }
     if (has_b2) {
-        const int rows = min(QT, N - q0);
         const T* src = static_cast<const T*>(p.b2) + ((size_t)head * N + q0) * n;
-        copy_flat(reinterpret_cast<unsigned char*>(sB2), reinterpret_cast<const unsigned char*>(src),
-                  rows * n * 2, tid);
+        copy_flat(reinterpret_cast<unsigned char*>(sB2), reinterpret_cast<const unsigned char*>(src), TQ * n * 2, tid);
     }
     cp_async_commit();
 
     // 2. wait for the slab's agent features, then fetch A and V_A (L2)
     wait_counter(p.counters + 2 * p.slabs + slab, 1u, p.status, kTimeoutFeatures);
+    if (tid == 0 && has_dwc) *s_whead = head;
     {
         const T* gA = static_cast<const T*>(p.a_ws) + (size_t)slab * n * DK;
         const T* gVA = static_cast<const T*>(p.va_ws) + (size_t)slab * n * DK;
@@ -433,137 +474,178 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
     cp_async_wait<0>();
     __syncthreads();
 
-    // 3. logits of 16 queries per warp against all agents, softmax over agents, times V_A
-    const int g = lane >> 2, t4 = lane & 3;
-    uint32_t qf[DK / 16][4];
+    // 3. attention part: 16 queries per warp against all agents
+    if (warp_active) {
+        const int g = lane >> 2, t4 = lane & 3;
+        uint32_t qf[DK / 16][4];
 #pragma unroll
-    for (int ks = 0; ks < DK / 16; ++ks)
-        ldmatrix_x4(qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3],
-                    sQ + ((lane & 7) + ((lane >> 3) & 1) * 8) * PA + ks * 16 + (lane >> 4) * 8);
-    __syncwarp();
+        for (int ks = 0; ks < DK / 16; ++ks)
+            ldmatrix_x4(qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3],
+                        sQ + ((lane & 7) + ((lane >> 3) & 1) * 8) * PA + ks * 16 + (lane >> 4) * 8);
+        __syncwarp();
 
-    const float scale_log2 = p.scale2 * kLog2e;
-    const int lr_a = warp * 16 + g, lr_b = lr_a + 8;           // rows within the tile
-    float sc[RP / 8][4];
+        const int lr_a = warp * 16 + g, lr_b = lr_a + 8;           // rows within the tile
+        float sc[RP / 8][4];
 #pragma unroll
-    for (int j = 0; j < RP / 8; ++j) { sc[j][0] = sc[j][1] = sc[j][2] = sc[j][3] = 0.f; }
+        for (int j = 0; j < RP / 8; ++j) { sc[j][0] = sc[j][1] = sc[j][2] = sc[j][3] = 0.f; }
 #pragma unroll
-    for (int ks = 0; ks < DK / 16; ++ks) {
+        for (int ks = 0; ks < DK / 16; ++ks) {
 #pragma unroll
-        for (int np = 0; np < RP / 16; ++np) {
-            if (np * 16 < n_pad) {
-                uint32_t b0, b1, b2, b3;
-                ldmatrix_x4(b0, b1, b2, b3,
-                            sA + (np * 16 + (lane & 7) + (lane >> 4) * 8) * PA + ks * 16 + ((lane >> 3) & 1) * 8);
-                mma16816<T>(sc[2 * np], qf[ks], b0, b1);
-                mma16816<T>(sc[2 * np + 1], qf[ks], b2, b3);
-            }
-        }
-    }
-    float mx0 = -INFINITY, mx1 = -INFINITY;
-    const bool row_a_ok = (q0 + lr_a) < N, row_b_ok = (q0 + lr_b) < N;
-#pragma unroll
-    for (int j = 0; j < RP / 8; ++j) {
-        const int col = 8 * j + 2 * t4;
-        const bool ok0 = col < n, ok1 = (col + 1) < n;
-        float b00 = 0.f, b01 = 0.f, b10 = 0.f, b11 = 0.f;
-        if (has_b2) {
-            if (row_a_ok) {
-                if (ok0) b00 = Elem<T>::to_f32(sB2[lr_a * n + col]) * kLog2e;
-                if (ok1) b01 = Elem<T>::to_f32(sB2[lr_a * n + col + 1]) * kLog2e;
-            }
-            if (row_b_ok) {
-                if (ok0) b10 = Elem<T>::to_f32(sB2[lr_b * n + col]) * kLog2e;
-                if (ok1) b11 = Elem<T>::to_f32(sB2[lr_b * n + col + 1]) * kLog2e;
-            }
-        }
-        sc[j][0] = ok0 ? fmaf(sc[j][0], scale_log2, b00) : -INFINITY;
-        sc[j][1] = ok1 ? fmaf(sc[j][1], scale_log2, b01) : -INFINITY;
-        sc[j][2] = ok0 ? fmaf(sc[j][2], scale_log2, b10) : -INFINITY;
-        sc[j][3] = ok1 ? fmaf(sc[j][3], scale_log2, b11) : -INFINITY;
-        mx0 = fmaxf(mx0, fmaxf(sc[j][0], sc[j][1]));
-        mx1 = fmaxf(mx1, fmaxf(sc[j][2], sc[j][3]));
-    }
-    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
-    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
-    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
-    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
-    float l0 = 0.f, l1 = 0.f;
-    uint32_t pk[RP / 8][2];
-#pragma unroll
-    for (int j = 0; j < RP / 8; ++j) {
-        pk[j][0] = pack2<T>(fast_exp2(sc[j][0] - mx0), fast_exp2(sc[j][1] - mx0));
-        pk[j][1] = pack2<T>(fast_exp2(sc[j][2] - mx1), fast_exp2(sc[j][3] - mx1));
-        const float2 u0 = unpack2<T>(pk[j][0]), u1 = unpack2<T>(pk[j][1]);
-        l0 += u0.x + u0.y;
-        l1 += u1.x + u1.y;
-    }
-    l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
-    l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
-    l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
-    l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
-    float acc[DK / 8][4];
-#pragma unroll
-    for (int j = 0; j < DK / 8; ++j) { acc[j][0] = acc[j][1] = acc[j][2] = acc[j][3] = 0.f; }
-#pragma unroll
-    for (int kk = 0; kk < RP / 16; ++kk) {
-        if (kk * 16 < n_pad) {
-            const uint32_t pa[4] = {pk[2 * kk][0], pk[2 * kk][1], pk[2 * kk + 1][0], pk[2 * kk + 1][1]};
-#pragma unroll
-            for (int np = 0; np < DK / 16; ++np) {
-                uint32_t b0, b1, b2, b3;
-                ldmatrix_x4_trans(b0, b1, b2, b3,
-                                  sVA + (kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * PA + np * 16 + (lane >> 4) * 8);
-                mma16816<T>(acc[2 * np], pa, b0, b1);
-                mma16816<T>(acc[2 * np + 1], pa, b2, b3);
-            }
-        }
-    }
-    const float inv0 = 1.f / l0, inv1 = 1.f / l1;
-#pragma unroll
-    for (int j = 0; j < DK / 8; ++j) {
-        const int col = 8 * j + 2 * t4;
-        *reinterpret_cast<float2*>(sPatch + g * PO + col) = make_float2(acc[j][0] * inv0, acc[j][1] * inv0);
-        *reinterpret_cast<float2*>(sPatch + (g + 8) * PO + col) = make_float2(acc[j][2] * inv1, acc[j][3] * inv1);
-    }
-    __syncwarp();
-
-    // 4. (token, 8 channels) items: add the depthwise 3x3 term from the V rows in shared memory, store
-    T* gO = static_cast<T*>(p.out) + (size_t)slab * N * DK;
-    for (int item = lane; item < 16 * cpr; item += 32) {
-        const int r = item / cpr, ch = item - r * cpr;
-        const int tok = i0 + r;
-        if (tok >= N) continue;
-        float o[8];
-        {
-            const float4 x0 = *reinterpret_cast<const float4*>(sPatch + r * PO + ch * 8);
-            const float4 x1 = *reinterpret_cast<const float4*>(sPatch + r * PO + ch * 8 + 4);
-            o[0] = x0.x; o[1] = x0.y; o[2] = x0.z; o[3] = x0.w;
-            o[4] = x1.x; o[5] = x1.y; o[6] = x1.z; o[7] = x1.w;
-        }
-        if (has_dwc) {
-            const int y = tok / W, x = tok - y * W;
-#pragma unroll
-            for (int u = 0; u < 3; ++u) {
-                const int yy = y + u - 1;
-                if (yy < 0 || yy >= H) continue;
-#pragma unroll
-                for (int v = 0; v < 3; ++v) {
-                    const int xx = x + v - 1;
-                    if (xx < 0 || xx >= W) continue;
-                    const uint4 raw = *(reinterpret_cast<const uint4*>(sH + (size_t)(yy * W + xx - h0) * DK) + ch);
-                    float f[8];
-                    unpack16<T>(raw, f);
-                    const float4 w0 = *reinterpret_cast<const float4*>(sW + (u * 3 + v) * DK + ch * 8);
-                    const float4 w1 = *reinterpret_cast<const float4*>(sW + (u * 3 + v) * DK + ch * 8 + 4);
-                    o[0] = fmaf(w0.x, f[0], o[0]); o[1] = fmaf(w0.y, f[1], o[1]);
-                    o[2] = fmaf(w0.z, f[2], o[2]); o[3] = fmaf(w0.w, f[3], o[3]);
-                    o[4] = fmaf(w1.x, f[4], o[4]); o[5] = fmaf(w1.y, f[5], o[5]);
-                    o[6] = fmaf(w1.z, f[6], o[6]); o[7] = fmaf(w1.w, f[7], o[7]);
+            for (int np = 0; np < RP / 16; ++np) {
+                if (np < n16) {
+                    uint32_t b0, b1, b2, b3;
+                    ldmatrix_x4(b0, b1, b2, b3,
+                                sA + (np * 16 + (lane & 7) + (lane >> 4) * 8) * PA + ks * 16 + ((lane >> 3) & 1) * 8);
+                    mma16816<T>(sc[2 * np], qf[ks], b0, b1);
+                    if (2 * np + 1 < n8) mma16816<T>(sc[2 * np + 1], qf[ks], b2, b3);
                 }
             }
         }
-        *(reinterpret_cast<uint4*>(gO + (size_t)tok * DK) + ch) = pack16<T>(o);
+        // logits in natural units: t = scale2 * q.a + b2; p = 2^((t - max) * log2 e)
+        float mx0 = -INFINITY, mx1 = -INFINITY;
+        {
+            // B2 rows are n (possibly odd) elements long, so a pair may straddle two 32-bit words
+            const uint32_t* w32 = reinterpret_cast<const uint32_t*>(sB2);
+            const int ea = lr_a * n + 2 * t4, eb = lr_b * n + 2 * t4;
+            const int sha = (ea & 1) * 16, shb = (eb & 1) * 16;
+#pragma unroll
+            for (int j = 0; j < RP / 8; ++j) {
+                if (j < n8) {
+                    float2 ba = make_float2(0.f, 0.f), bb = make_float2(0.f, 0.f);
+                    if (has_b2) {
+                        const int wa = (ea + 8 * j) >> 1, wb = (eb + 8 * j) >> 1;
+                        ba = unpack2<T>(__funnelshift_r(w32[wa], w32[wa + 1], sha));
+                        bb = unpack2<T>(__funnelshift_r(w32[wb], w32[wb + 1], shb));
+                    }
+                    sc[j][0] = fmaf(sc[j][0], p.scale2, ba.x);
+                    sc[j][1] = fmaf(sc[j][1], p.scale2, ba.y);
+                    sc[j][2] = fmaf(sc[j][2], p.scale2, bb.x);
+                    sc[j][3] = fmaf(sc[j][3], p.scale2, bb.y);
+                    if (8 * j + 8 > n) {     // last column tile: columns >= n are not agents
+                        const int col = 8 * j + 2 * t4;
+                        if (col >= n)     { sc[j][0] = -INFINITY; sc[j][2] = -INFINITY; }
+                        if (col + 1 >= n) { sc[j][1] = -INFINITY; sc[j][3] = -INFINITY; }
+                    }
+                    mx0 = fmaxf(mx0, fmaxf(sc[j][0], sc[j][1]));
+                    mx1 = fmaxf(mx1, fmaxf(sc[j][2], sc[j][3]));
+                }
+            }
+        }
+        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+        const float nm0 = -mx0 * kLog2e, nm1 = -mx1 * kLog2e;
+        uint32_t pk[RP / 8][2];
+#pragma unroll
+        for (int j = 0; j < RP / 8; ++j) {
+            if (j < n8) {
+                pk[j][0] = pack2<T>(fast_exp2(fmaf(sc[j][0], kLog2e, nm0)), fast_exp2(fmaf(sc[j][1], kLog2e, nm0)));
+                pk[j][1] = pack2<T>(fast_exp2(fmaf(sc[j][2], kLog2e, nm1)), fast_exp2(fmaf(sc[j][3], kLog2e, nm1)));
+            } else {
+                pk[j][0] = 0u; pk[j][1] = 0u;
+            }
+        }
+        float acc[DK / 8][4], accl[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int j = 0; j < DK / 8; ++j) { acc[j][0] = acc[j][1] = acc[j][2] = acc[j][3] = 0.f; }
+#pragma unroll
+        for (int kk = 0; kk < RP / 16; ++kk) {
+            if (kk < n16) {
+                const uint32_t pa[4] = {pk[2 * kk][0], pk[2 * kk][1], pk[2 * kk + 1][0], pk[2 * kk + 1][1]};
+#pragma unroll
+                for (int np = 0; np < DK / 16; ++np) {
+                    uint32_t b0, b1, b2, b3;
+                    ldmatrix_x4_trans(b0, b1, b2, b3,
+                                      sVA + (kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * PA + np * 16 + (lane >> 4) * 8);
+                    mma16816<T>(acc[2 * np], pa, b0, b1);
+                    mma16816<T>(acc[2 * np + 1], pa, b2, b3);
+                }
+                uint32_t o0, o1;           // column DK of V_A holds 1: the product's column DK is the row sum
+                ldmatrix_x2_trans(o0, o1, sVA + (kk * 16 + (lane & 15)) * PA + DK);
+                mma16816<T>(accl, pa, o0, o1);
+            }
+        }
+        const float l0 = __shfl_sync(0xffffffffu, accl[0], lane & ~3);
+        const float l1 = __shfl_sync(0xffffffffu, accl[2], lane & ~3);
+        const float inv0 = 1.f / l0, inv1 = 1.f / l1;
+#pragma unroll
+        for (int j = 0; j < DK / 8; ++j) {
+            const int col = 8 * j + 2 * t4;
+            *reinterpret_cast<float2*>(sPatch + g * PO + col) = make_float2(acc[j][0] * inv0, acc[j][1] * inv0);
+            *reinterpret_cast<float2*>(sPatch + (g + 8) * PO + col) = make_float2(acc[j][2] * inv1, acc[j][3] * inv1);
+        }
+    }
+    __syncthreads();
+
+    // 4. depthwise 3x3 term + store: thread = (tile row r, 4-channel group cq, x-segment)
+    {
+        constexpr int NCQ = DK / 4;
+        const int npairs = rows * NCQ;
+        int nseg = NT / npairs;
+        if (nseg < 1) nseg = 1;
+        if (nseg > W) nseg = W;
+        const int seg_len = (W + nseg - 1) / nseg;
+        T* gO = static_cast<T*>(p.out) + ((size_t)slab * N + q0) * DK;
+        for (int item = tid; item < npairs * nseg; item += NT) {
+            const int pair = item % npairs, seg = item / npairs;
+            const int r = pair / NCQ, cq = pair - r * NCQ;
+            const int x0 = seg * seg_len, x1 = min(W, x0 + seg_len);
+            if (x0 >= x1) continue;
+            if (has_dwc) {
+                float2 w[9][2];                 // taps x two channel pairs
+#pragma unroll
+                for (int tap = 0; tap < 9; ++tap) {
+                    const float4 t = *reinterpret_cast<const float4*>(sW + tap * DK + cq * 4);
+                    w[tap][0] = make_float2(t.x, t.y);
+                    w[tap][1] = make_float2(t.z, t.w);
+                }
+                // halo rows r, r+1, r+2 are grid rows y-1, y, y+1; halo column x+1 is grid column x
+                const T* hp = sH + (r * HP) * DK + cq * 4;
+                const float* pp = sPatchAll + (r * W) * PO + cq * 4;
+                T* op = gO + (size_t)(r * W) * DK + cq * 4;
+                float2 ca[3][2], cb[3][2], cc[3][2];
+                auto load_col = [&](int hx, float2 (&c)[3][2]) {
+#pragma unroll
+                    for (int u = 0; u < 3; ++u) {
+                        const uint2 raw = *reinterpret_cast<const uint2*>(hp + (u * HP + hx) * DK);
+                        c[u][0] = unpack2<T>(raw.x);
+                        c[u][1] = unpack2<T>(raw.y);
+                    }
+                };
+                auto emit = [&](int x, const float2 (&l)[3][2], const float2 (&c)[3][2], const float2 (&rr)[3][2]) {
+                    const float4 a4 = *reinterpret_cast<const float4*>(pp + x * PO);
+                    float2 o0 = make_float2(a4.x, a4.y), o1 = make_float2(a4.z, a4.w);
+#pragma unroll
+                    for (int u = 0; u < 3; ++u) {
+                        o0 = ffma2(w[u * 3 + 0][0], l[u][0], o0);  o1 = ffma2(w[u * 3 + 0][1], l[u][1], o1);
+                        o0 = ffma2(w[u * 3 + 1][0], c[u][0], o0);  o1 = ffma2(w[u * 3 + 1][1], c[u][1], o1);
+                        o0 = ffma2(w[u * 3 + 2][0], rr[u][0], o0); o1 = ffma2(w[u * 3 + 2][1], rr[u][1], o1);
+                    }
+                    uint2 outw;
+                    outw.x = pack2<T>(o0.x, o0.y);
+                    outw.y = pack2<T>(o1.x, o1.y);
+                    *reinterpret_cast<uint2*>(op + x * DK) = outw;
+                };
+                load_col(x0, ca);          // grid column x0 - 1
+                load_col(x0 + 1, cb);      // grid column x0
+                int x = x0;
+                while (x < x1) {           // the three window columns rotate roles instead of moving
+                    load_col(x + 2, cc); emit(x, ca, cb, cc); if (++x >= x1) break;
+                    load_col(x + 2, ca); emit(x, cb, cc, ca); if (++x >= x1) break;
+                    load_col(x + 2, cb); emit(x, cc, ca, cb); ++x;
+                }
+            } else {
+                for (int x = x0; x < x1; ++x) {
+                    const int tl = r * W + x;
+                    const float4 a4 = *reinterpret_cast<const float4*>(sPatchAll + (size_t)tl * PO + cq * 4);
+                    uint2 outw;
+                    outw.x = pack2<T>(a4.x, a4.y);
+                    outw.y = pack2<T>(a4.z, a4.w);
+                    *reinterpret_cast<uint2*>(gO + (size_t)tl * DK + cq * 4) = outw;
+                }
+            }
+        }
     }
     __syncthreads();     // shared memory is free for the next task
 }
@@ -572,11 +654,17 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
 template <typename T, int DK>
 __global__ void __launch_bounds__(NT, 2) fused_kernel(const __grid_constant__ FusedArgs p) {
     extern __shared__ __align__(16) unsigned char smem[];
-    __shared__ int s_task, s_flag;
+    __shared__ int s_task, s_flag, s_whead;
     const int tid = threadIdx.x;
     {   // zero once: rows >= n of the resident A / V_A must be finite zeros for the whole kernel
         uint4* z = reinterpret_cast<uint4*>(smem);
         for (int i = tid; i < (int)(FusedSmem<DK>::kTotal / 16); i += NT) z[i] = make_uint4(0, 0, 0, 0);
+    }
+    if (tid == 0) s_whead = -1;
+    __syncthreads();
+    if (tid < RP) {   // column DK of the resident V_A rows holds 1 (row sums of P from the P.V_A product)
+        T* sVA = reinterpret_cast<T*>(smem + FusedSmem<DK>::kA);
+        *reinterpret_cast<uint4*>(sVA + tid * FusedSmem<DK>::PA + DK) = make_uint4(pack2<T>(1.f, 0.f), 0u, 0u, 0u);
     }
     __syncthreads();
     const int G = p.plan.g_tasks, B = p.plan.b_tasks, Lg = p.plan.lag, S = p.slabs;
@@ -606,7 +694,7 @@ __global__ void __launch_bounds__(NT, 2) fused_kernel(const __grid_constant__ Fu
             slab = S - Lg + step; sub = t - step * B; is_g = false;
         }
         if (is_g) run_g_task<T, DK>(p, slab, sub, smem, &s_flag);
-        else      run_b_task<T, DK>(p, slab, sub, smem);
+        else      run_b_task<T, DK>(p, slab, sub, smem, &s_whead);
     }
 }
 
@@ -630,7 +718,7 @@ static bool fused_shape_plan(int dtype, int H, int W, int d, int n_agents, Fused
     memset(pl, 0, sizeof(*pl));
     if (dtype != kBF16 && dtype != kF16) return false;
     if (d != 32 && d != 64) return false;
-    if (n_agents < 1 || n_agents > RP || W > MAXW || H < 1) return false;
+    if (n_agents < 1 || n_agents > RP || W > MAXW || W < MINW || H < 1) return false;
     int p = 1;
     while (p * p < n_agents) ++p;
     if (p * p != n_agents || H % p != 0 || W % p != 0) return false;
@@ -641,7 +729,12 @@ static bool fused_shape_plan(int dtype, int H, int W, int d, int n_agents, Fused
     if (k > p) k = p;
     pl->rows_per_g = k * win_h;
     pl->g_tasks = (p + k - 1) / k;
-    pl->b_tasks = (H * W + QT - 1) / QT;
+    int R = QT / W;
+    if (R > 16) R = 16;
+    if (R > H) R = H;
+    pl->rows_per_b = R;
+    pl->b_tasks = (H + R - 1) / R;
+    if ((R + 2) * (W + 2) > kHaloTokens) return false;
     pl->parts = pl->g_tasks * 2;
     return pl->g_tasks <= 32;
 }
@@ -665,7 +758,9 @@ FusedPlan plan_fused(int dtype, int slabs, int H, int W, int d, int n_agents, in
     pl.grid = (int)grid;
     if (pl.grid < pl.g_tasks || pl.g_tasks > 32) return pl;      // progress needs a resident block per G sibling
     int lag = (3 * pl.grid / 2 + pl.g_tasks + pl.b_tasks - 1) / (pl.g_tasks + pl.b_tasks) + 1;
+    if (const char* e = getenv("AA_FUSED_LAG")) lag = atoi(e);
     if (lag > slabs) lag = slabs;
+    if (lag < 1) lag = 1;
     pl.lag = lag;
     pl.smem = d == 64 ? FusedSmem<64>::kTotal : FusedSmem<32>::kTotal;
     pl.ok = true;

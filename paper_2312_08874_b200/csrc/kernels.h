@@ -69,7 +69,8 @@ struct FusedPlan {
     bool ok;            // shape is eligible
     int g_tasks;        // G tasks per slab
     int rows_per_g;     // grid rows per G task (a multiple of the pooling window height)
-    int b_tasks;        // B tasks (128-token tiles) per slab
+    int rows_per_b;     // grid rows per B task (rows_per_b * W <= 128 tokens)
+    int b_tasks;        // B tasks per slab
     int lag;            // slabs between a slab's G tasks and its B tasks in the queue
     int grid;           // resident blocks
     int parts;          // partial states per slab
