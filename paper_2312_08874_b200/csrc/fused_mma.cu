@@ -61,6 +61,22 @@ __device__ __forceinline__ void publish_add(unsigned* ctr) {
     if (threadIdx.x == 0) { __threadfence(); atomicAdd(ctr, 1u); }
 }
 
+// Optional per-task phase timestamps (debug builds only): define AA_FUSED_TRACE and export a
+// device buffer through aa_fused_trace_buffer; record i of a block goes to slot (blockIdx, i).
+#ifdef AA_FUSED_TRACE
+__device__ unsigned long long* g_trace = nullptr;
+__device__ __forceinline__ void trace_mark(int task_slot, int phase) {
+    if (threadIdx.x == 0 && g_trace && task_slot < 16) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        g_trace[((size_t)blockIdx.x * 16 + task_slot) * 8 + phase] = t;
+    }
+}
+#define TRACE(slot, phase) trace_mark(slot, phase)
+#else
+#define TRACE(slot, phase)
+#endif
+
 template <int DK> struct FusedSmem {
     static constexpr int PA = DK + 8;                               // padded row pitch (elements)
     static constexpr int PB = KT + 8;                               // B1 tile row pitch
@@ -129,7 +145,7 @@ __device__ __forceinline__ void merge_partials_vec(const float* parts_base, int 
 // ---------------------------------------------------------------------------------- G task
 template <typename T, int DK>
 __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub, unsigned char* smem,
-                                           int* s_flag) {
+                                           int* s_flag, int slot) {
     using L = FusedSmem<DK>;
     constexpr int PA = L::PA, PB = L::PB;
     constexpr int NWK = 2, KW = KT / NWK;
@@ -194,6 +210,7 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
         const uint32_t one = pack2<T>(1.f, 0.f);
         *reinterpret_cast<uint4*>(stage_v(tid / KT) + (tid % KT) * PA + DK) = make_uint4(one, 0u, 0u, 0u);
     }
+    TRACE(slot, 0);
     // 1. start the ring
     for (int s = 0; s < STAGES - 1; ++s) {
         if (s < tiles) load_tile(s, s);
@@ -214,15 +231,25 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
             float acc[8];
 #pragma unroll
             for (int k = 0; k < 8; ++k) acc[k] = 0.f;
-#pragma unroll 4
-            for (int i = tsub; i < cnt; i += tpl) {
-                const int wy = i / win_w, wx = i - wy * win_w;
-                const size_t tok = (size_t)(y0 + wy) * W + (x0 + wx);
-                const uint4 raw = __ldg(reinterpret_cast<const uint4*>(gQ + tok * DK) + cg);
-                float f[8];
-                unpack16<T>(raw, f);
+            for (int ib = tsub; ib < cnt; ib += 8 * tpl) {     // eight loads in flight per lane
+                uint4 raw[8];
 #pragma unroll
-                for (int k = 0; k < 8; ++k) acc[k] += f[k];
+                for (int u = 0; u < 8; ++u) {
+                    const int i = ib + u * tpl;
+                    raw[u] = make_uint4(0u, 0u, 0u, 0u);
+                    if (i < cnt) {
+                        const int wy = i / win_w, wx = i - wy * win_w;
+                        const size_t tok = (size_t)(y0 + wy) * W + (x0 + wx);
+                        raw[u] = __ldg(reinterpret_cast<const uint4*>(gQ + tok * DK) + cg);
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    float f[8];
+                    unpack16<T>(raw[u], f);
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) acc[k] += f[k];
+                }
             }
 #pragma unroll
             for (int o = cpr; o < 32; o <<= 1) {
@@ -236,10 +263,12 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
             }
         }
     }
+    TRACE(slot, 1);
     // 3. publish these agent rows, wait for the slab's other G tasks
     publish_add(p.counters + slab);
     wait_counter(p.counters + slab, (unsigned)p.plan.g_tasks, p.status, kTimeoutAgents);
 
+    TRACE(slot, 2);
     // 4. all agents of the slab -> shared memory (L2 reads; rows >= n stay zero)
     for (int e = tid; e < n * cpr; e += NT) {
         const int r = e / cpr, c = e - r * cpr;
@@ -262,6 +291,7 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
 #pragma unroll
     for (int j = 0; j < DK / 8; ++j) { acc[j][0] = acc[j][1] = acc[j][2] = acc[j][3] = 0.f; }
 
+    TRACE(slot, 3);
     // 5. online-softmax aggregation over the range
     for (int it = 0; it < tiles; ++it) {
         cp_async_wait<STAGES - 2>();
@@ -360,28 +390,90 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
     const float l0 = __shfl_sync(0xffffffffu, accl[0], lane & ~3);
     const float l1 = __shfl_sync(0xffffffffu, accl[2], lane & ~3);
 
-    // 6. partial state of this warp; the slab's last G task merges and raises the slab's flag
+    TRACE(slot, 4);
+    // 6. the two key halves of the block combine through shared memory into one partial state;
+    //    the slab's last G task merges all partials and raises the slab's flag
+    __syncthreads();                                   // every warp is done with the ring
+    float* sX = reinterpret_cast<float*>(ring);        // [4 row groups][36 values][32 lanes]
+    float* sWgt = sX + 4 * 36 * 32;                    // merge weights [parts][RP]
+    if (wk == 1) {
+        float* x = sX + wm * 36 * 32 + lane;
+        x[0] = m0; x[32] = m1; x[64] = l0; x[96] = l1;
+#pragma unroll
+        for (int j = 0; j < DK / 8; ++j) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) x[(4 + 4 * j + e) * 32] = acc[j][e];
+        }
+    }
+    __syncthreads();
     const int parts = p.plan.parts;
     const size_t pf = partial_floats(RP, DK);
     float* slab_parts = p.partials + (size_t)slab * parts * pf;
-    float* part = slab_parts + (size_t)(sub * NWK + wk) * pf;
-    if (t4 == 0) {
-        part[r0 + g] = m0 * kLog2e; part[r0 + g + 8] = m1 * kLog2e;     // the merge works in log2 units
-        part[RP + r0 + g] = l0; part[RP + r0 + g + 8] = l1;
-    }
-    float* pacc = part + 2 * RP;
+    if (wk == 0) {
+        const float* x = sX + wm * 36 * 32 + lane;
+        const float om0 = x[0], om1 = x[32];
+        const float mm0 = fmaxf(m0, om0), mm1 = fmaxf(m1, om1);
+        const float bs0 = (mm0 == -INFINITY) ? 0.f : mm0, bs1 = (mm1 == -INFINITY) ? 0.f : mm1;
+        const float wa0 = fast_exp2((m0 - bs0) * kLog2e), wb0 = fast_exp2((om0 - bs0) * kLog2e);
+        const float wa1 = fast_exp2((m1 - bs1) * kLog2e), wb1 = fast_exp2((om1 - bs1) * kLog2e);
+        float* part = slab_parts + (size_t)sub * pf;
+        if (t4 == 0) {
+            part[r0 + g] = mm0 * kLog2e; part[r0 + g + 8] = mm1 * kLog2e;     // the merge works in log2 units
+            part[RP + r0 + g] = l0 * wa0 + x[64] * wb0;
+            part[RP + r0 + g + 8] = l1 * wa1 + x[96] * wb1;
+        }
+        float* pacc = part + 2 * RP;
 #pragma unroll
-    for (int j = 0; j < DK / 8; ++j) {
-        const int col = 8 * j + 2 * t4;
-        *reinterpret_cast<float2*>(pacc + (size_t)(r0 + g) * DK + col) = make_float2(acc[j][0], acc[j][1]);
-        *reinterpret_cast<float2*>(pacc + (size_t)(r0 + g + 8) * DK + col) = make_float2(acc[j][2], acc[j][3]);
+        for (int j = 0; j < DK / 8; ++j) {
+            const int col = 8 * j + 2 * t4;
+            *reinterpret_cast<float2*>(pacc + (size_t)(r0 + g) * DK + col) =
+                make_float2(acc[j][0] * wa0 + x[(4 + 4 * j) * 32] * wb0, acc[j][1] * wa0 + x[(5 + 4 * j) * 32] * wb0);
+            *reinterpret_cast<float2*>(pacc + (size_t)(r0 + g + 8) * DK + col) =
+                make_float2(acc[j][2] * wa1 + x[(6 + 4 * j) * 32] * wb1, acc[j][3] * wa1 + x[(7 + 4 * j) * 32] * wb1);
+        }
     }
     unsigned* ticket = p.counters + p.slabs + slab;
     if (arrive_is_last(ticket, (unsigned)p.plan.g_tasks, s_flag)) {
-        merge_partials_vec<T>(slab_parts, parts, DK, n, DK, static_cast<T*>(p.va_ws) + (size_t)slab * n * DK);
+        // step 1: one thread per agent row turns the parts' (max, sum) into normalised weights
+        if (tid < n) {
+            float mj[32], mmax = -INFINITY, den = 0.f;
+#pragma unroll
+            for (int q = 0; q < 32; ++q) {
+                mj[q] = (q < parts) ? __ldcg(slab_parts + q * pf + tid) : -INFINITY;
+                mmax = fmaxf(mmax, mj[q]);
+            }
+#pragma unroll
+            for (int q = 0; q < 32; ++q) {
+                if (q < parts) {
+                    mj[q] = (mj[q] == -INFINITY) ? 0.f : exp2f(mj[q] - mmax);
+                    den += mj[q] * __ldcg(slab_parts + q * pf + RP + tid);
+                }
+            }
+            const float inv = 1.f / den;
+#pragma unroll
+            for (int q = 0; q < 32; ++q) if (q < parts) sWgt[q * RP + tid] = mj[q] * inv;
+        }
+        __syncthreads();
+        // step 2: V_A[r][c..c+3] = sum over parts of weight * acc, in the fixed order of the parts
+        T* va = static_cast<T*>(p.va_ws) + (size_t)slab * n * DK;
+        for (int e = tid; e < n * (DK / 4); e += NT) {
+            const int r = e / (DK / 4), c = (e - r * (DK / 4)) * 4;
+            float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 8
+            for (int q = 0; q < parts; ++q) {
+                const float wq = sWgt[q * RP + r];
+                const float4 a = __ldcg(reinterpret_cast<const float4*>(slab_parts + q * pf + 2 * RP + (size_t)r * DK + c));
+                num.x += wq * a.x; num.y += wq * a.y; num.z += wq * a.z; num.w += wq * a.w;
+            }
+            uint2 o;
+            o.x = pack2<T>(num.x, num.y);
+            o.y = pack2<T>(num.z, num.w);
+            *reinterpret_cast<uint2*>(va + (size_t)r * DK + c) = o;
+        }
         publish_add(p.counters + 2 * p.slabs + slab);
     }
     __syncthreads();     // the ring is free for the next task
+    TRACE(slot, 5);
 }
 
 // ---------------------------------------------------------------------------------- B task
@@ -392,7 +484,7 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
 // add the depthwise term (Eq. 6), round once and store.
 template <typename T, int DK>
 __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int tile, unsigned char* smem,
-                                           int* s_whead) {
+                                           int* s_whead, int slot) {
     using L = FusedSmem<DK>;
     constexpr int PA = L::PA, PO = L::PO;
     constexpr int cpr = DK / 8;
@@ -424,7 +516,20 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
     const T* gQ = static_cast<const T*>(p.q) + (size_t)slab * N * DK;
     const T* gV = static_cast<const T*>(p.v) + (size_t)slab * N * DK;
 
+    TRACE(slot, 0);
+    const unsigned* va_flag = p.counters + 2 * p.slabs + slab;
+    const bool early = ld_acquire(va_flag) >= 1u;      // usual case: the slab's aggregation is long done
+    auto load_agents = [&]() {
+        const T* gA = static_cast<const T*>(p.a_ws) + (size_t)slab * n * DK;
+        const T* gVA = static_cast<const T*>(p.va_ws) + (size_t)slab * n * DK;
+        for (int e = tid; e < n * cpr; e += NT) {
+            const int r = e / cpr, c = e - r * cpr;
+            cp_async16(sA + r * PA + c * 8, gA + (size_t)r * DK + c * 8, 16);
+            cp_async16(sVA + r * PA + c * 8, gVA + (size_t)r * DK + c * 8, 16);
+        }
+    };
     // 1. loads that do not depend on the aggregation
+    if (early) load_agents();
     if (warp_active) {
         for (int e = lane; e < 16 * cpr; e += 32) {
             const int r = e / cpr, c = e - r * cpr;
@@ -458,22 +563,17 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
     }
     cp_async_commit();
 
+    TRACE(slot, 1);
     // 2. wait for the slab's agent features, then fetch A and V_A (L2)
-    wait_counter(p.counters + 2 * p.slabs + slab, 1u, p.status, kTimeoutFeatures);
+    wait_counter(va_flag, 1u, p.status, kTimeoutFeatures);
+    TRACE(slot, 2);
     if (tid == 0 && has_dwc) *s_whead = head;
-    {
-        const T* gA = static_cast<const T*>(p.a_ws) + (size_t)slab * n * DK;
-        const T* gVA = static_cast<const T*>(p.va_ws) + (size_t)slab * n * DK;
-        for (int e = tid; e < n * cpr; e += NT) {
-            const int r = e / cpr, c = e - r * cpr;
-            cp_async16(sA + r * PA + c * 8, gA + (size_t)r * DK + c * 8, 16);
-            cp_async16(sVA + r * PA + c * 8, gVA + (size_t)r * DK + c * 8, 16);
-        }
-    }
+    if (!early) load_agents();
     cp_async_commit();
     cp_async_wait<0>();
     __syncthreads();
 
+    TRACE(slot, 3);
     // 3. attention part: 16 queries per warp against all agents
     if (warp_active) {
         const int g = lane >> 2, t4 = lane & 3;
@@ -578,6 +678,7 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
     }
     __syncthreads();
 
+    TRACE(slot, 4);
     // 4. depthwise 3x3 term + store: thread = (tile row r, 4-channel group cq, x-segment)
     {
         constexpr int NCQ = DK / 4;
@@ -648,6 +749,7 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
         }
     }
     __syncthreads();     // shared memory is free for the next task
+    TRACE(slot, 5);
 }
 
 // ---------------------------------------------------------------------------------- kernel
@@ -671,6 +773,7 @@ __global__ void __launch_bounds__(NT, 2) fused_kernel(const __grid_constant__ Fu
     const int count0 = Lg * G, count1 = (S - Lg) * (G + B);
     const int total = S * (G + B);
     unsigned* queue = p.counters + 3 * (size_t)S;
+    int slot = 0;
     for (;;) {
         if (tid == 0) s_task = (int)atomicAdd(queue, 1u);
         __syncthreads();
@@ -693,8 +796,15 @@ __global__ void __launch_bounds__(NT, 2) fused_kernel(const __grid_constant__ Fu
             const int step = t / B;
             slab = S - Lg + step; sub = t - step * B; is_g = false;
         }
-        if (is_g) run_g_task<T, DK>(p, slab, sub, smem, &s_flag);
-        else      run_b_task<T, DK>(p, slab, sub, smem, &s_whead);
+        if (is_g) run_g_task<T, DK>(p, slab, sub, smem, &s_flag, slot);
+        else      run_b_task<T, DK>(p, slab, sub, smem, &s_whead, slot);
+#ifdef AA_FUSED_TRACE
+        if (tid == 0 && g_trace && slot < 16) {
+            g_trace[((size_t)blockIdx.x * 16 + slot) * 8 + 6] = is_g ? 1 : 2;
+            g_trace[((size_t)blockIdx.x * 16 + slot) * 8 + 7] = (unsigned long long)task;
+        }
+#endif
+        ++slot;
     }
 }
 
@@ -735,7 +845,7 @@ static bool fused_shape_plan(int dtype, int H, int W, int d, int n_agents, Fused
     pl->rows_per_b = R;
     pl->b_tasks = (H + R - 1) / R;
     if ((R + 2) * (W + 2) > kHaloTokens) return false;
-    pl->parts = pl->g_tasks * 2;
+    pl->parts = pl->g_tasks;
     return pl->g_tasks <= 32;
 }
 
@@ -757,7 +867,7 @@ FusedPlan plan_fused(int dtype, int slabs, int H, int W, int d, int n_agents, in
     if (grid > total) grid = total;
     pl.grid = (int)grid;
     if (pl.grid < pl.g_tasks || pl.g_tasks > 32) return pl;      // progress needs a resident block per G sibling
-    int lag = (3 * pl.grid / 2 + pl.g_tasks + pl.b_tasks - 1) / (pl.g_tasks + pl.b_tasks) + 1;
+    int lag = (5 * pl.grid / 2 + pl.g_tasks + pl.b_tasks - 1) / (pl.g_tasks + pl.b_tasks) + 2;
     if (const char* e = getenv("AA_FUSED_LAG")) lag = atoi(e);
     if (lag > slabs) lag = slabs;
     if (lag < 1) lag = 1;
@@ -780,3 +890,9 @@ cudaError_t launch_fused(int dtype, const FusedArgs& a, cudaStream_t st) {
 }
 
 }  // namespace aa
+
+#ifdef AA_FUSED_TRACE
+extern "C" int aa_fused_trace_buffer(void* device_buffer) {
+    return (int)cudaMemcpyToSymbol(aa::g_trace, &device_buffer, sizeof(void*));
+}
+#endif
