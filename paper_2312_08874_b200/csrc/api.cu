@@ -319,6 +319,7 @@ int agent_attn_forward(agent_attn_handle* h, const void* Q, const void* K, const
             fa.counters = counters; fa.status = h->d_status;
             fa.slabs = slabs; fa.heads = h->cfg.heads; fa.H = grid_h; fa.W = grid_w; fa.d = h->cfg.head_dim;
             fa.n = n_agents; fa.p = p; fa.scale1 = h->scale1; fa.scale2 = h->scale2; fa.plan = h->fused_plan;
+            if (!fused_make_maps(&fa)) return fail(h, AA_ERR_CUDA, "tensor map encoding failed");
             e = launch_fused(h->cfg.dtype, fa, st);
             if (e != cudaSuccess) return fail(h, AA_ERR_CUDA, "fused launch failed: %s", cudaGetErrorString(e));
             h->launches = 1;

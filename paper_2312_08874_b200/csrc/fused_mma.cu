@@ -1,24 +1,28 @@
-// The whole module of Eq. 6 in one persistent kernel, for small agent counts (n <= 64).
+// The whole module of Eq. 6 in one persistent kernel, for small agent counts (n <= 64, d = 64).
 //
 // Why one kernel: the path reads Q twice (pooling, broadcast) and V twice (aggregation, DWC).
 // Run phase by phase over a large batch, the second reads come from HBM.  Here resident blocks
 // pull tasks from a queue ordered slab by slab, so a slab's second reads follow its first ones
 // within microseconds and are served by L2; HBM sees every input once.
 //
-//   G task (slab, range of grid rows): start the K/V/B1 tile ring, pool Q over the range (whole
-//     pooling windows: these are complete agent rows), publish them, wait until the slab's other G
-//     tasks have published theirs, then run the split aggregation over the range (Eq. 3, Eq. 5).
-//     The last G task of a slab merges the partial states into V_A and raises the slab's flag.
-//   B task (slab, 128-token tile): start loading Q, the V rows with their 3x3 halo and the B2 tile,
-//     wait for the slab's flag, load A and V_A, then broadcast + DWC (Eq. 3, Eq. 5, Eq. 6).
+//   G task (slab, range of grid rows): start the K/V/B1 tile ring (TMA, 128-byte swizzle), pool Q
+//     over the range (whole pooling windows: complete agent rows), publish them, wait until the
+//     slab's other G tasks have published theirs, then run the split aggregation over the range
+//     (Eq. 3, Eq. 5).  The last G task of a slab merges the partial states into V_A and raises the
+//     slab's flag.
+//   B task (slab, tile of whole grid rows, <= 128 tokens): start the bulk copies of the V rows
+//     (with their 3x3 halo) and of the B2 tile, load Q fragments straight into registers, wait for
+//     the slab's flag, fetch A and V_A (TMA), then broadcast + DWC (Eq. 3, Eq. 5, Eq. 6).
 //
-// Every wait is bounded: after kSpinLimit polls the block records a timeout in the status word
-// and carries on (the result is then wrong, but nothing hangs).  Queue order guarantees progress:
-// a task only waits for tasks that precede it or for its own slab's G siblings, which are adjacent
-// in the queue, and the grid holds at least as many resident blocks as a slab has G tasks.
+// Every wait is bounded: flag polls and mbarrier waits give up after a fixed number of tries,
+// record a code in the status word and carry on (the result is then wrong, but nothing hangs).
+// Queue order guarantees progress: a task only waits for tasks that precede it or for its own
+// slab's G siblings, which are adjacent in the queue, and the grid holds at least as many
+// resident blocks as a slab has G tasks.  No TMA multicast is used.
 #include "common.cuh"
 #include "kernels.h"
 #include "merge.cuh"
+#include "tma.cuh"
 
 #include <cstdlib>
 #include <cstring>
@@ -26,16 +30,42 @@
 namespace aa {
 
 namespace {
+constexpr int DK = 64;            // head dim handled by this kernel
 constexpr int KT = 64;            // tokens per aggregation tile
-constexpr int QT = 128;           // tokens per broadcast tile
+constexpr int QT = 128;           // most tokens per broadcast tile
 constexpr int NT = 256;           // threads per block (8 warps)
 constexpr int RP = 64;            // agent rows, padded
 constexpr int STAGES = 3;
-constexpr int MAXW = 64;          // widest grid the halo buffer is sized for
+constexpr int MAXW = 64;          // widest grid the V-row buffer is sized for
 constexpr int MINW = 8;
 constexpr int kHaloTokens = 264;  // max over 8 <= W <= 64 of (R + 2)(W + 2), R = min(16, 128 / W)
-constexpr unsigned kSpinLimit = 1u << 20;
-constexpr int kTimeoutAgents = 1, kTimeoutFeatures = 2;
+constexpr unsigned kSpinLimit = 1u << 20;      // flag polls
+constexpr unsigned kBarLimit = 1u << 22;       // mbarrier try_wait attempts
+constexpr int kTimeoutAgents = 1, kTimeoutFeatures = 2, kTimeoutTile = 3, kTimeoutLoads = 4;
+
+// shared-memory map (bytes from a 1024-byte aligned base)
+constexpr int kTileBytes = KT * 128;                    // one swizzled 64 x 64 tile of 16-bit elements
+constexpr int OFF_A = 0;                                // resident agents A            [64][128 B] swizzled
+constexpr int OFF_VA = OFF_A + kTileBytes;              // resident agent features V_A  [64][128 B] swizzled
+constexpr int OFF_W = OFF_VA + kTileBytes;              // filter taps [9][64] fp32
+constexpr int OFF_UNION = 19456;                        // 19 KiB: start of the per-task area
+// G tasks: ring of STAGES x (K tile | V tile | B1 tile)
+constexpr int kStageBytes = 3 * kTileBytes;
+constexpr int kGBytes = STAGES * kStageBytes;
+// B tasks: fp32 patch | V rows with zero borders | B2 tile
+constexpr int PO = DK + 8;                              // patch pitch (floats)
+constexpr int OFF_PATCH = OFF_UNION;
+constexpr int kPatchBytes = QT * PO * 4;
+constexpr int OFF_HALO = OFF_PATCH + kPatchBytes;
+constexpr int kHaloBytes = kHaloTokens * DK * 2;
+constexpr int OFF_B2 = OFF_HALO + kHaloBytes;
+constexpr int kB2Bytes = QT * RP * 2 + 16;              // + one spare vector: pairs are read as two words
+constexpr int kBBytes = kPatchBytes + kHaloBytes + kB2Bytes;
+constexpr int OFF_BAR = OFF_UNION + (kGBytes > kBBytes ? kGBytes : kBBytes);   // mbarriers (8 bytes each)
+constexpr int kNumBars = STAGES + 2;                    // ring stages, agents, broadcast inputs
+constexpr int kSmemBytes = OFF_BAR + 8 * kNumBars + 1024;   // + slack to align the base to 1024
+static_assert(OFF_W + 9 * DK * 4 <= OFF_UNION, "common area overflows");
+static_assert(OFF_UNION % 1024 == 0 && kStageBytes % 1024 == 0 && OFF_BAR % 8 == 0, "alignment");
 
 __device__ __forceinline__ unsigned ld_acquire(const unsigned* p) {
     unsigned v;
@@ -60,9 +90,18 @@ __device__ __forceinline__ void publish_add(unsigned* ctr) {
     __syncthreads();
     if (threadIdx.x == 0) { __threadfence(); atomicAdd(ctr, 1u); }
 }
+// All threads wait for a phase of an mbarrier; on expiry the block records `code` and goes on.
+__device__ __forceinline__ void wait_bar(uint32_t bar, uint32_t parity, int* status, int code) {
+    if (!mbar_wait_bounded(bar, parity, kBarLimit)) atomicExch(status, code);
+}
+// Byte offset of element (row, col) in a swizzled [rows][64] tile of 16-bit elements: the 16-byte
+// chunk index is XORed with the row index modulo 8 (the TMA 128-byte swizzle).
+__device__ __forceinline__ int swz(int row, int col) {
+    return row * 128 + ((((col >> 3) ^ row) & 7) << 4) + (col & 7) * 2;
+}
 
-// Optional per-task phase timestamps (debug builds only): define AA_FUSED_TRACE and export a
-// device buffer through aa_fused_trace_buffer; record i of a block goes to slot (blockIdx, i).
+// Optional per-task phase timestamps (debug builds only): define AA_FUSED_TRACE and hand a device
+// buffer to aa_fused_trace_buffer; record i of a block goes to slot (blockIdx, i).
 #ifdef AA_FUSED_TRACE
 __device__ unsigned long long* g_trace = nullptr;
 __device__ __forceinline__ void trace_mark(int task_slot, int phase) {
@@ -77,78 +116,30 @@ __device__ __forceinline__ void trace_mark(int task_slot, int phase) {
 #define TRACE(slot, phase)
 #endif
 
-template <int DK> struct FusedSmem {
-    static constexpr int PA = DK + 8;                               // padded row pitch (elements)
-    static constexpr int PB = KT + 8;                               // B1 tile row pitch
-    static constexpr size_t kA = (size_t)RP * PA * 2;               // resident agents
-    static constexpr size_t kVA = kA;                               // resident agent features
-    static constexpr size_t kW = (size_t)9 * DK * 4;                // filter taps [9][DK] fp32
-    static constexpr size_t kCommon = kA + kVA + kW;
-    // G layout
-    static constexpr size_t kTile = (size_t)KT * PA * 2;
-    static constexpr size_t kB1 = (size_t)RP * PB * 2;
-    static constexpr size_t kStage = 2 * kTile + kB1;
-    static constexpr size_t kG = STAGES * kStage;
-    // B layout
-    static constexpr int PO = DK + 8;                               // fp32 patch pitch (floats)
-    static constexpr size_t kPatch = (size_t)8 * 16 * PO * 4;       // per-warp [16][PO] fp32 (Q rows alias it)
-    static constexpr size_t kHalo = (size_t)kHaloTokens * DK * 2;   // (rows+2) x (W+2) tokens, see plan
-    static constexpr size_t kB2 = (size_t)QT * RP * 2 + 16;         // + one spare vector: pairs are read as two words
-    static constexpr size_t kB = kPatch + kHalo + kB2;
-    static constexpr size_t kTotal = kCommon + (kG > kB ? kG : kB);
-};
-
-// Flat global -> shared copy of `bytes` (a multiple of 2) with the widest cp.async the source
-// alignment allows; the tail and 2-byte-aligned sources go through plain loads.
+// Flat global -> shared copy of `bytes` (a multiple of 2) by plain loads: the fallback when a
+// bulk copy's alignment rules do not hold.
 __device__ __forceinline__ void copy_flat(unsigned char* dst, const unsigned char* src, int bytes, int tid) {
-    const uintptr_t a = reinterpret_cast<uintptr_t>(src);
-    if ((a & 15) == 0) {
-        const int n16 = bytes >> 4;
-        for (int i = tid; i < n16; i += NT) cp_async16(dst + 16 * i, src + 16 * i, 16);
-        for (int i = (n16 << 4) + 2 * tid; i < bytes; i += 2 * NT)
-            *reinterpret_cast<unsigned short*>(dst + i) = *reinterpret_cast<const unsigned short*>(src + i);
-    } else {
-        for (int i = 2 * tid; i < bytes; i += 2 * NT)
-            *reinterpret_cast<unsigned short*>(dst + i) = *reinterpret_cast<const unsigned short*>(src + i);
-    }
+    for (int i = 2 * tid; i < bytes; i += 2 * NT)
+        *reinterpret_cast<unsigned short*>(dst + i) = *reinterpret_cast<const unsigned short*>(src + i);
 }
+
+// Block-level state that persists across tasks: mbarrier phase parities.
+struct BlockState {
+    uint32_t bar_base;          // shared address of the first mbarrier
+    uint32_t ph;                // parity to wait for next: bit s = ring stage s, then agents, broadcast inputs
+};
+constexpr int kBitAgents = STAGES, kBitBin = STAGES + 1;
+__device__ __forceinline__ uint32_t bar_full(const BlockState& st, int s) { return st.bar_base + 8 * s; }
+__device__ __forceinline__ uint32_t bar_agents(const BlockState& st) { return st.bar_base + 8 * STAGES; }
+__device__ __forceinline__ uint32_t bar_bin(const BlockState& st) { return st.bar_base + 8 * (STAGES + 1); }
 }  // namespace
 
-// Faster merge for the fused kernel: one thread per (agent row, 4 channels), float4 loads.
-template <typename T>
-__device__ __forceinline__ void merge_partials_vec(const float* parts_base, int parts, int dpad, int rows,
-                                                   int d, T* out) {
-    const size_t pf = partial_floats(RP, dpad);
-    const int cq = d / 4;
-    for (int e = threadIdx.x; e < rows * cq; e += NT) {
-        const int r = e / cq, c = (e - r * cq) * 4;
-        float m = -INFINITY;
-        for (int j = 0; j < parts; ++j) m = fmaxf(m, __ldcg(parts_base + j * pf + r));
-        float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
-        float den = 0.f;
-#pragma unroll 4
-        for (int j = 0; j < parts; ++j) {
-            const float* pj = parts_base + j * pf;
-            const float mj = __ldcg(pj + r);
-            const float w = (mj == -INFINITY) ? 0.f : exp2f(mj - m);
-            den += w * __ldcg(pj + RP + r);
-            const float4 a = __ldcg(reinterpret_cast<const float4*>(pj + 2 * RP + (size_t)r * dpad + c));
-            num.x += w * a.x; num.y += w * a.y; num.z += w * a.z; num.w += w * a.w;
-        }
-        const float inv = 1.f / den;
-        T* o = out + (size_t)r * d + c;
-        o[0] = Elem<T>::from_f32(num.x * inv); o[1] = Elem<T>::from_f32(num.y * inv);
-        o[2] = Elem<T>::from_f32(num.z * inv); o[3] = Elem<T>::from_f32(num.w * inv);
-    }
-}
-
 // ---------------------------------------------------------------------------------- G task
-template <typename T, int DK>
+template <typename T>
 __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub, unsigned char* smem,
-                                           int* s_flag, int slot) {
-    using L = FusedSmem<DK>;
-    constexpr int PA = L::PA, PB = L::PB;
+                                           BlockState& st, int* s_flag, int slot) {
     constexpr int NWK = 2, KW = KT / NWK;
+    constexpr int cpr = DK / 8;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int wm = warp & 3, wk = warp >> 2;
     const int head = slab % p.heads;
@@ -158,64 +149,40 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
     const int t_begin = gr0 * W, t_end = gr1 * W;
     const int tiles = (t_end - t_begin + KT - 1) / KT;
     const bool has_bias = p.b1 != nullptr;
-    const bool bias_vec = has_bias && (N % 8 == 0) && (t_begin % 8 == 0);
+    const bool bias_tma = has_bias && p.b1_tma;
 
-    T* sA = reinterpret_cast<T*>(smem);
-    unsigned char* ring = smem + L::kCommon;
-    auto stage_k = [&](int s) { return reinterpret_cast<T*>(ring + s * L::kStage); };
-    auto stage_v = [&](int s) { return reinterpret_cast<T*>(ring + s * L::kStage + L::kTile); };
-    auto stage_b = [&](int s) { return reinterpret_cast<T*>(ring + s * L::kStage + 2 * L::kTile); };
-
+    unsigned char* sA = smem + OFF_A;
+    unsigned char* ring = smem + OFF_UNION;
+    const uint32_t ring_u32 = smem_u32(ring);
     const T* gQ = static_cast<const T*>(p.q) + (size_t)slab * N * DK;
-    const T* gK = static_cast<const T*>(p.k) + (size_t)slab * N * DK;
-    const T* gV = static_cast<const T*>(p.v) + (size_t)slab * N * DK;
     const T* gB = has_bias ? static_cast<const T*>(p.b1) + (size_t)head * n * N : nullptr;
     T* gA = static_cast<T*>(p.a_ws) + (size_t)slab * n * DK;
-    constexpr int cpr = DK / 8;
+    const uint32_t tile_tx = 2 * kTileBytes + (bias_tma ? kTileBytes : 0);
 
-    auto load_tile = [&](int t, int s) {
+    // tile t of this range -> ring stage s: K and V rows, and the B1 columns of the same tokens
+    auto issue_tile = [&](int t, int s) {
         const int c0 = t_begin + t * KT;
-        T* sK = stage_k(s);
-        T* sV = stage_v(s);
-        for (int e = tid; e < KT * cpr; e += NT) {
-            const int j = e / cpr, c = e - j * cpr;
-            const int key = c0 + j;
-            const bool ok = key < t_end;
-            const size_t off = ok ? ((size_t)key * DK + c * 8) : 0;
-            cp_async16(sK + j * PA + c * 8, gK + off, ok ? 16 : 0);
-            cp_async16(sV + j * PA + c * 8, gV + off, ok ? 16 : 0);
+        if (tid == 0) {
+            const uint32_t bar = bar_full(st, s), dst = ring_u32 + s * kStageBytes;
+            mbar_arrive_expect_tx(bar, tile_tx);
+            tma_load_2d(dst, &p.tm_k, 0, slab * N + c0, bar);
+            tma_load_2d(dst + kTileBytes, &p.tm_v, 0, slab * N + c0, bar);
+            if (bias_tma) tma_load_2d(dst + 2 * kTileBytes, &p.tm_b1, c0, head * n, bar);
         }
-        if (has_bias) {
-            T* sB = stage_b(s);
-            if (bias_vec) {
-                for (int e = tid; e < n * (KT / 8); e += NT) {
-                    const int r = e / (KT / 8), c = e - r * (KT / 8);
-                    const int key = c0 + c * 8;
-                    int bytes = (t_end - key) * 2;
-                    bytes = bytes < 0 ? 0 : (bytes > 16 ? 16 : bytes);
-                    cp_async16(sB + r * PB + c * 8, gB + (bytes ? ((size_t)r * N + key) : 0), bytes);
-                }
-            } else {
-                for (int e = tid; e < n * KT; e += NT) {
-                    const int r = e / KT, j = e - r * KT;
-                    const int key = c0 + j;
-                    sB[r * PB + j] = key < t_end ? gB[(size_t)r * N + key] : Elem<T>::from_f32(0.f);
-                }
+        if (has_bias && !bias_tma) {       // B1 rows not 16-byte aligned: plain loads into the same layout
+            unsigned char* sB = ring + s * kStageBytes + 2 * kTileBytes;
+            for (int e = tid; e < n * KT; e += NT) {
+                const int r = e / KT, j = e - r * KT;
+                const int key = c0 + j;
+                *reinterpret_cast<T*>(sB + swz(r, j)) = key < t_end ? gB[(size_t)r * N + key] : Elem<T>::from_f32(0.f);
             }
         }
     };
 
-    // column DK of every V tile row holds 1, so the P.V product also yields the row sums of P
-    if (tid < STAGES * KT) {
-        const uint32_t one = pack2<T>(1.f, 0.f);
-        *reinterpret_cast<uint4*>(stage_v(tid / KT) + (tid % KT) * PA + DK) = make_uint4(one, 0u, 0u, 0u);
-    }
     TRACE(slot, 0);
     // 1. start the ring
-    for (int s = 0; s < STAGES - 1; ++s) {
-        if (s < tiles) load_tile(s, s);
-        cp_async_commit();
-    }
+    for (int s = 0; s < STAGES - 1; ++s)
+        if (s < tiles) issue_tile(s, s);
 
     // 2. pool this range of Q: whole windows, i.e. complete rows of A (text under Eq. 6)
     {
@@ -269,22 +236,24 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
     wait_counter(p.counters + slab, (unsigned)p.plan.g_tasks, p.status, kTimeoutAgents);
 
     TRACE(slot, 2);
-    // 4. all agents of the slab -> shared memory (L2 reads; rows >= n stay zero)
-    for (int e = tid; e < n * cpr; e += NT) {
-        const int r = e / cpr, c = e - r * cpr;
-        cp_async16(sA + r * PA + c * 8, gA + (size_t)r * DK + c * 8, 16);
+    // 4. all agents of the slab -> shared memory (rows >= n receive foreign rows; they only feed
+    //    padded agent rows, which are never merged)
+    if (tid == 0) {
+        mbar_arrive_expect_tx(bar_agents(st), kTileBytes);
+        tma_load_2d(smem_u32(sA), &p.tm_a, 0, slab * n, bar_agents(st));
     }
-    cp_async_commit();
-    cp_async_wait<0>();
-    __syncthreads();
+    wait_bar(bar_agents(st), (st.ph >> kBitAgents) & 1u, p.status, kTimeoutLoads);
+    st.ph ^= 1u << kBitAgents;
 
-    const int g = lane >> 2, t4 = lane & 3;
+    const int g = lane >> 2, t4 = lane & 3, xr = lane & 7;
     const int r0 = wm * 16, kw0 = wk * KW;
     uint32_t af[DK / 16][4];
 #pragma unroll
     for (int ks = 0; ks < DK / 16; ++ks)
         ldmatrix_x4(af[ks][0], af[ks][1], af[ks][2], af[ks][3],
-                    sA + (r0 + (lane & 7) + ((lane >> 3) & 1) * 8) * PA + ks * 16 + (lane >> 4) * 8);
+                    sA + (r0 + xr + ((lane >> 3) & 1) * 8) * 128 + (((ks * 2 + (lane >> 4)) ^ xr) << 4));
+    // B fragment that is 1 in column 0: one more MMA per key block yields the row sums of P
+    const uint32_t ones = (g == 0) ? pack2<T>(1.f, 1.f) : 0u;
 
     float m0 = -INFINITY, m1 = -INFINITY;            // running row maxima, natural units
     float acc[DK / 8][4], accl[4] = {0.f, 0.f, 0.f, 0.f};
@@ -294,14 +263,13 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
     TRACE(slot, 3);
     // 5. online-softmax aggregation over the range
     for (int it = 0; it < tiles; ++it) {
-        cp_async_wait<STAGES - 2>();
-        __syncthreads();
-        if (it + STAGES - 1 < tiles) load_tile(it + STAGES - 1, (it + STAGES - 1) % STAGES);
-        cp_async_commit();
         const int s = it % STAGES;
-        const T* sK = stage_k(s);
-        const T* sV = stage_v(s);
-        const T* sB = stage_b(s);
+        if (it + STAGES - 1 < tiles) issue_tile(it + STAGES - 1, (it + STAGES - 1) % STAGES);
+        wait_bar(bar_full(st, s), (st.ph >> s) & 1u, p.status, kTimeoutTile);
+        st.ph ^= 1u << s;
+        const unsigned char* sK = ring + s * kStageBytes;
+        const unsigned char* sV = sK + kTileBytes;
+        const unsigned char* sB = sV + kTileBytes;
         const int c0 = t_begin + it * KT;
 
         float sc[KW / 8][4];
@@ -313,27 +281,26 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
             for (int np = 0; np < KW / 16; ++np) {
                 uint32_t b0, b1, b2, b3;
                 ldmatrix_x4(b0, b1, b2, b3,
-                            sK + (kw0 + np * 16 + (lane & 7) + (lane >> 4) * 8) * PA + ks * 16 + ((lane >> 3) & 1) * 8);
+                            sK + (kw0 + np * 16 + xr + (lane >> 4) * 8) * 128 + (((ks * 2 + ((lane >> 3) & 1)) ^ xr) << 4));
                 mma16816<T>(sc[2 * np], af[ks], b0, b1);
                 mma16816<T>(sc[2 * np + 1], af[ks], b2, b3);
             }
         }
         // logits in natural units: t = scale1 * a.k + b1
-        float mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll
         for (int j = 0; j < KW / 8; ++j) {
-            const int col = kw0 + 8 * j + 2 * t4;
             float2 ba = make_float2(0.f, 0.f), bb = make_float2(0.f, 0.f);
             if (has_bias) {
-                ba = unpack2<T>(*reinterpret_cast<const uint32_t*>(sB + (r0 + g) * PB + col));
-                bb = unpack2<T>(*reinterpret_cast<const uint32_t*>(sB + (r0 + g + 8) * PB + col));
+                const int cb = (((kw0 >> 3) + j) ^ g) << 4;      // rows r0+g and r0+g+8 share row % 8 = g
+                ba = unpack2<T>(*reinterpret_cast<const uint32_t*>(sB + (r0 + g) * 128 + cb + t4 * 4));
+                bb = unpack2<T>(*reinterpret_cast<const uint32_t*>(sB + (r0 + g + 8) * 128 + cb + t4 * 4));
             }
             sc[j][0] = fmaf(sc[j][0], p.scale1, ba.x);
             sc[j][1] = fmaf(sc[j][1], p.scale1, ba.y);
             sc[j][2] = fmaf(sc[j][2], p.scale1, bb.x);
             sc[j][3] = fmaf(sc[j][3], p.scale1, bb.y);
         }
-        if (c0 + KT > t_end) {          // ragged last tile of the range: keys beyond it do not exist
+        if (c0 + KT > t_end) {          // ragged last tile of the range: keys beyond it do not belong to it
 #pragma unroll
             for (int j = 0; j < KW / 8; ++j) {
                 const int key = c0 + kw0 + 8 * j + 2 * t4;
@@ -341,6 +308,7 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
                 if (key + 1 >= t_end) { sc[j][1] = -INFINITY; sc[j][3] = -INFINITY; }
             }
         }
+        float mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll
         for (int j = 0; j < KW / 8; ++j) {
             mx0 = fmaxf(mx0, fmaxf(sc[j][0], sc[j][1]));
@@ -353,15 +321,18 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
         const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
         const float base0 = (mn0 == -INFINITY) ? 0.f : mn0;
         const float base1 = (mn1 == -INFINITY) ? 0.f : mn1;
-        const float corr0 = fast_exp2((m0 - base0) * kLog2e), corr1 = fast_exp2((m1 - base1) * kLog2e);
         const float nb0 = -base0 * kLog2e, nb1 = -base1 * kLog2e;
-        m0 = mn0; m1 = mn1;
-        accl[0] *= corr0; accl[1] *= corr0; accl[2] *= corr1; accl[3] *= corr1;
+        // rescale the running state only when some row of the warp saw a new maximum
+        if (__any_sync(0xffffffffu, (mn0 != m0) || (mn1 != m1))) {
+            const float corr0 = fast_exp2(fmaf(m0, kLog2e, nb0)), corr1 = fast_exp2(fmaf(m1, kLog2e, nb1));
+            accl[0] *= corr0; accl[2] *= corr1;
 #pragma unroll
-        for (int j = 0; j < DK / 8; ++j) {
-            acc[j][0] *= corr0; acc[j][1] *= corr0; acc[j][2] *= corr1; acc[j][3] *= corr1;
+            for (int j = 0; j < DK / 8; ++j) {
+                acc[j][0] *= corr0; acc[j][1] *= corr0; acc[j][2] *= corr1; acc[j][3] *= corr1;
+            }
         }
-        // probabilities rounded to the operand type; their row sums come out of the same MMA
+        m0 = mn0; m1 = mn1;
+        // probabilities rounded to the operand type; their row sums come out of one more MMA
         uint32_t pk[KW / 8][2];
 #pragma unroll
         for (int j = 0; j < KW / 8; ++j) {
@@ -375,25 +346,22 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
             for (int np = 0; np < DK / 16; ++np) {
                 uint32_t b0, b1, b2, b3;
                 ldmatrix_x4_trans(b0, b1, b2, b3,
-                                  sV + (kw0 + kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * PA + np * 16 + (lane >> 4) * 8);
+                                  sV + (kw0 + kk * 16 + xr + ((lane >> 3) & 1) * 8) * 128 + (((np * 2 + (lane >> 4)) ^ xr) << 4));
                 mma16816<T>(acc[2 * np], pa, b0, b1);
                 mma16816<T>(acc[2 * np + 1], pa, b2, b3);
             }
-            uint32_t o0, o1;
-            ldmatrix_x2_trans(o0, o1, sV + (kw0 + kk * 16 + (lane & 15)) * PA + DK);
-            mma16816<T>(accl, pa, o0, o1);
+            mma16816<T>(accl, pa, ones, ones);
         }
+        __syncthreads();               // every warp is done with stage s before it is refilled
     }
-    cp_async_wait<0>();
 
-    // row sums sit in column DK of the product: lanes with t4 == 0 hold them
+    // row sums sit in column 0 of the extra product: lanes with t4 == 0 hold them
     const float l0 = __shfl_sync(0xffffffffu, accl[0], lane & ~3);
     const float l1 = __shfl_sync(0xffffffffu, accl[2], lane & ~3);
 
     TRACE(slot, 4);
     // 6. the two key halves of the block combine through shared memory into one partial state;
     //    the slab's last G task merges all partials and raises the slab's flag
-    __syncthreads();                                   // every warp is done with the ring
     float* sX = reinterpret_cast<float*>(ring);        // [4 row groups][36 values][32 lanes]
     float* sWgt = sX + 4 * 36 * 32;                    // merge weights [parts][RP]
     if (wk == 1) {
@@ -472,22 +440,20 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
         }
         publish_add(p.counters + 2 * p.slabs + slab);
     }
-    __syncthreads();     // the ring is free for the next task
+    fence_proxy_async();   // this task's plain shared-memory writes precede the next task's TMA writes
+    __syncthreads();       // the ring is free for the next task
     TRACE(slot, 5);
 }
 
 // ---------------------------------------------------------------------------------- B task
-// One tile = R whole grid rows (R*W <= 128 tokens).  Warps 0..7 own 16 query rows each for the
-// attention part and leave their fp32 result in the patch; then all threads switch to a
-// (row, 4-channel group, x-segment) mapping and slide a 3x3 window along x over the V rows held in
-// shared memory (with explicit zero columns at x = -1 and x = W and zero rows outside the grid),
-// add the depthwise term (Eq. 6), round once and store.
-template <typename T, int DK>
+// One tile = R whole grid rows (R*W <= 128 tokens).  Warps own 16 query rows each for the attention
+// part and leave their fp32 result in the patch; then all threads switch to a (row, 4-channel
+// group, x-segment) mapping and slide a 3x3 window along x over the V rows held in shared memory
+// (with explicit zero columns at x = -1 and x = W and zero rows outside the grid), add the
+// depthwise term (Eq. 6), round once and store.
+template <typename T>
 __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int tile, unsigned char* smem,
-                                           int* s_whead, int slot) {
-    using L = FusedSmem<DK>;
-    constexpr int PA = L::PA, PO = L::PO;
-    constexpr int cpr = DK / 8;
+                                           BlockState& st, int* s_whead, int slot) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int head = slab % p.heads;
     const int N = p.H * p.W, n = p.n, W = p.W, H = p.H;
@@ -497,58 +463,79 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
     const int y0 = tile * R;
     const int rows = min(R, H - y0);
     const int q0 = y0 * W, TQ = rows * W;            // tokens of this tile
-    const int i0 = q0 + warp * 16;
     const bool warp_active = warp * 16 < TQ;
     const bool has_dwc = p.dwc_w != nullptr;
     const bool has_b2 = p.b2 != nullptr;
-    const int HP = W + 2;                             // halo row pitch in tokens
+    const int HP = W + 2;                             // V-row pitch in tokens (zero columns at both ends)
+    const int g = lane >> 2, t4 = lane & 3, xr = lane & 7;
 
-    T* sA = reinterpret_cast<T*>(smem);
-    T* sVA = reinterpret_cast<T*>(smem + L::kA);
-    unsigned char* base = smem + L::kCommon;
-    float* sPatchAll = reinterpret_cast<float*>(base);               // [128][PO] fp32
-    float* sPatch = sPatchAll + (size_t)warp * 16 * PO;
-    T* sQ = reinterpret_cast<T*>(sPatch);                            // [16][PA], aliases the warp's patch rows
-    T* sH = reinterpret_cast<T*>(base + L::kPatch);                  // [(rows+2)][W+2][DK] V rows with zero borders
-    T* sB2 = reinterpret_cast<T*>(base + L::kPatch + L::kHalo);      // [TQ][n] flat
-    float* sW = reinterpret_cast<float*>(smem + L::kA + L::kVA);                  // [9][DK], survives G tasks
+    unsigned char* sA = smem + OFF_A;
+    unsigned char* sVA = smem + OFF_VA;
+    float* sW = reinterpret_cast<float*>(smem + OFF_W);
+    float* sPatchAll = reinterpret_cast<float*>(smem + OFF_PATCH);   // [128][PO] fp32
+    float* sPatch = sPatchAll + warp * 16 * PO;
+    T* sH = reinterpret_cast<T*>(smem + OFF_HALO);                   // [(rows+2)][W+2][DK]
+    T* sB2 = reinterpret_cast<T*>(smem + OFF_B2);                    // [TQ][n] flat
 
-    const T* gQ = static_cast<const T*>(p.q) + (size_t)slab * N * DK;
+    const T* gQ = static_cast<const T*>(p.q) + ((size_t)slab * N + q0) * DK;
     const T* gV = static_cast<const T*>(p.v) + (size_t)slab * N * DK;
+    const unsigned* va_flag = p.counters + 2 * p.slabs + slab;
 
     TRACE(slot, 0);
-    const unsigned* va_flag = p.counters + 2 * p.slabs + slab;
     const bool early = ld_acquire(va_flag) >= 1u;      // usual case: the slab's aggregation is long done
-    auto load_agents = [&]() {
-        const T* gA = static_cast<const T*>(p.a_ws) + (size_t)slab * n * DK;
-        const T* gVA = static_cast<const T*>(p.va_ws) + (size_t)slab * n * DK;
-        for (int e = tid; e < n * cpr; e += NT) {
-            const int r = e / cpr, c = e - r * cpr;
-            cp_async16(sA + r * PA + c * 8, gA + (size_t)r * DK + c * 8, 16);
-            cp_async16(sVA + r * PA + c * 8, gVA + (size_t)r * DK + c * 8, 16);
+    auto issue_agents = [&]() {
+        if (tid == 0) {
+            mbar_arrive_expect_tx(bar_agents(st), 2 * kTileBytes);
+            tma_load_2d(smem_u32(sA), &p.tm_a, 0, slab * n, bar_agents(st));
+            tma_load_2d(smem_u32(sVA), &p.tm_va, 0, slab * n, bar_agents(st));
         }
     };
-    // 1. loads that do not depend on the aggregation
-    if (early) load_agents();
-    if (warp_active) {
-        for (int e = lane; e < 16 * cpr; e += 32) {
-            const int r = e / cpr, c = e - r * cpr;
-            const bool ok = (warp * 16 + r) < TQ;
-            cp_async16(sQ + r * PA + c * 8, gQ + (ok ? ((size_t)(i0 + r) * DK + c * 8) : 0), ok ? 16 : 0);
+    // 1. bulk copies that do not depend on the aggregation: V rows y0-1 .. y0+rows, the B2 tile
+    const T* b2src = has_b2 ? static_cast<const T*>(p.b2) + ((size_t)head * N + q0) * n : nullptr;
+    const int b2bytes = TQ * n * 2;
+    const bool b2_bulk = has_b2 && ((reinterpret_cast<uintptr_t>(b2src) & 15u) == 0) && ((b2bytes & 15) == 0);
+    int vrows = 0;
+    if (has_dwc) vrows = min(H, y0 + rows + 1) - max(0, y0 - 1);
+    const uint32_t bin_bytes = (uint32_t)vrows * W * DK * 2 + (b2_bulk ? b2bytes : 0);
+    if (tid == 0 && bin_bytes) {
+        const uint32_t bar = bar_bin(st);
+        mbar_arrive_expect_tx(bar, bin_bytes);
+        if (has_dwc) {
+            for (int hr = 0; hr < rows + 2; ++hr) {
+                const int y = y0 - 1 + hr;
+                if (y >= 0 && y < H)
+                    bulk_load_1d(smem_u32(sH + ((size_t)hr * HP + 1) * DK), gV + (size_t)y * W * DK, W * DK * 2, bar);
+            }
+        }
+        if (b2_bulk) bulk_load_1d(smem_u32(sB2), b2src, b2bytes, bar);
+    }
+    if (early) issue_agents();
+    // Q fragments of this warp's 16 rows straight into registers
+    uint32_t qf[DK / 16][4];
+    {
+        const bool oka = (warp * 16 + g) < TQ, okb = (warp * 16 + g + 8) < TQ;
+        const uint32_t* ra = reinterpret_cast<const uint32_t*>(gQ + (size_t)(warp * 16 + g) * DK) + t4;
+        const uint32_t* rb = reinterpret_cast<const uint32_t*>(gQ + (size_t)(warp * 16 + g + 8) * DK) + t4;
+#pragma unroll
+        for (int ks = 0; ks < DK / 16; ++ks) {
+            qf[ks][0] = oka ? __ldg(ra + ks * 8) : 0u;
+            qf[ks][1] = okb ? __ldg(rb + ks * 8) : 0u;
+            qf[ks][2] = oka ? __ldg(ra + ks * 8 + 4) : 0u;
+            qf[ks][3] = okb ? __ldg(rb + ks * 8 + 4) : 0u;
         }
     }
     if (has_dwc) {
-        for (int hr = 0; hr < rows + 2; ++hr) {
-            const int y = y0 - 1 + hr;
-            const bool ok = (y >= 0) && (y < H);
-            const T* src = gV + (ok ? (size_t)y * W * DK : 0);
-            T* dst = sH + ((size_t)hr * HP + 1) * DK;
-            for (int e = tid; e < W * cpr; e += NT) cp_async16(dst + e * 8, src + e * 8, ok ? 16 : 0);
-            if (tid < 2 * cpr) {       // zero columns x = -1 and x = W
-                const int side = tid / cpr, c = tid - side * cpr;
-                *(reinterpret_cast<uint4*>(sH + ((size_t)hr * HP + (side ? W + 1 : 0)) * DK) + c) = make_uint4(0, 0, 0, 0);
-            }
+        // zero borders: columns x = -1 and x = W of every row, and rows that fall outside the grid
+        for (int e = tid; e < (rows + 2) * 2 * (DK / 8); e += NT) {
+            const int hr = e / (2 * (DK / 8)), rest = e - hr * 2 * (DK / 8);
+            const int side = rest / (DK / 8), c = rest - side * (DK / 8);
+            *(reinterpret_cast<uint4*>(sH + ((size_t)hr * HP + (side ? W + 1 : 0)) * DK) + c) = make_uint4(0, 0, 0, 0);
         }
+        if (y0 == 0)
+            for (int e = tid; e < W * (DK / 8); e += NT) *(reinterpret_cast<uint4*>(sH + DK) + e) = make_uint4(0, 0, 0, 0);
+        if (y0 + rows >= H)
+            for (int e = tid; e < W * (DK / 8); e += NT)
+                *(reinterpret_cast<uint4*>(sH + ((size_t)(rows + 1) * HP + 1) * DK) + e) = make_uint4(0, 0, 0, 0);
         if (*s_whead != head) {       // filter taps change only with the head
             const T* w = static_cast<const T*>(p.dwc_w) + (size_t)head * DK * 9;
             for (int e = tid; e < 9 * DK; e += NT) {
@@ -557,33 +544,29 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
             }
         }
     }
-    if (has_b2) {
-        const T* src = static_cast<const T*>(p.b2) + ((size_t)head * N + q0) * n;
-        copy_flat(reinterpret_cast<unsigned char*>(sB2), reinterpret_cast<const unsigned char*>(src), TQ * n * 2, tid);
-    }
-    cp_async_commit();
+    if (has_b2 && !b2_bulk)
+        copy_flat(reinterpret_cast<unsigned char*>(sB2), reinterpret_cast<const unsigned char*>(b2src), b2bytes, tid);
 
     TRACE(slot, 1);
     // 2. wait for the slab's agent features, then fetch A and V_A (L2)
     wait_counter(va_flag, 1u, p.status, kTimeoutFeatures);
     TRACE(slot, 2);
     if (tid == 0 && has_dwc) *s_whead = head;
-    if (!early) load_agents();
-    cp_async_commit();
-    cp_async_wait<0>();
+    if (!early) issue_agents();
+    wait_bar(bar_agents(st), (st.ph >> kBitAgents) & 1u, p.status, kTimeoutLoads);
+    st.ph ^= 1u << kBitAgents;
+    if (bin_bytes) {
+        wait_bar(bar_bin(st), (st.ph >> kBitBin) & 1u, p.status, kTimeoutLoads);
+        st.ph ^= 1u << kBitBin;
+    }
+    // rows >= n of the V_A tile hold foreign rows: they must be zero, since 0 * NaN is not 0
+    for (int e = tid; e < (RP - n) * 8; e += NT)
+        *(reinterpret_cast<uint4*>(sVA + (n + e / 8) * 128) + (e & 7)) = make_uint4(0, 0, 0, 0);
     __syncthreads();
 
     TRACE(slot, 3);
     // 3. attention part: 16 queries per warp against all agents
     if (warp_active) {
-        const int g = lane >> 2, t4 = lane & 3;
-        uint32_t qf[DK / 16][4];
-#pragma unroll
-        for (int ks = 0; ks < DK / 16; ++ks)
-            ldmatrix_x4(qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3],
-                        sQ + ((lane & 7) + ((lane >> 3) & 1) * 8) * PA + ks * 16 + (lane >> 4) * 8);
-        __syncwarp();
-
         const int lr_a = warp * 16 + g, lr_b = lr_a + 8;           // rows within the tile
         float sc[RP / 8][4];
 #pragma unroll
@@ -595,7 +578,7 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
                 if (np < n16) {
                     uint32_t b0, b1, b2, b3;
                     ldmatrix_x4(b0, b1, b2, b3,
-                                sA + (np * 16 + (lane & 7) + (lane >> 4) * 8) * PA + ks * 16 + ((lane >> 3) & 1) * 8);
+                                sA + (np * 16 + xr + (lane >> 4) * 8) * 128 + (((ks * 2 + ((lane >> 3) & 1)) ^ xr) << 4));
                     mma16816<T>(sc[2 * np], qf[ks], b0, b1);
                     if (2 * np + 1 < n8) mma16816<T>(sc[2 * np + 1], qf[ks], b2, b3);
                 }
@@ -646,6 +629,7 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
                 pk[j][0] = 0u; pk[j][1] = 0u;
             }
         }
+        const uint32_t ones = (g == 0) ? pack2<T>(1.f, 1.f) : 0u;      // column 0 of the extra product = row sums
         float acc[DK / 8][4], accl[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int j = 0; j < DK / 8; ++j) { acc[j][0] = acc[j][1] = acc[j][2] = acc[j][3] = 0.f; }
@@ -657,13 +641,11 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
                 for (int np = 0; np < DK / 16; ++np) {
                     uint32_t b0, b1, b2, b3;
                     ldmatrix_x4_trans(b0, b1, b2, b3,
-                                      sVA + (kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * PA + np * 16 + (lane >> 4) * 8);
+                                      sVA + (kk * 16 + xr + ((lane >> 3) & 1) * 8) * 128 + (((np * 2 + (lane >> 4)) ^ xr) << 4));
                     mma16816<T>(acc[2 * np], pa, b0, b1);
                     mma16816<T>(acc[2 * np + 1], pa, b2, b3);
                 }
-                uint32_t o0, o1;           // column DK of V_A holds 1: the product's column DK is the row sum
-                ldmatrix_x2_trans(o0, o1, sVA + (kk * 16 + (lane & 15)) * PA + DK);
-                mma16816<T>(accl, pa, o0, o1);
+                mma16816<T>(accl, pa, ones, ones);
             }
         }
         const float l0 = __shfl_sync(0xffffffffu, accl[0], lane & ~3);
@@ -677,8 +659,8 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
         }
     }
     __syncthreads();
-
     TRACE(slot, 4);
+
     // 4. depthwise 3x3 term + store: thread = (tile row r, 4-channel group cq, x-segment)
     {
         constexpr int NCQ = DK / 4;
@@ -693,6 +675,8 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
             const int r = pair / NCQ, cq = pair - r * NCQ;
             const int x0 = seg * seg_len, x1 = min(W, x0 + seg_len);
             if (x0 >= x1) continue;
+            const float* pp = sPatchAll + (r * W) * PO + cq * 4;
+            T* op = gO + (size_t)(r * W) * DK + cq * 4;
             if (has_dwc) {
                 float2 w[9][2];                 // taps x two channel pairs
 #pragma unroll
@@ -701,10 +685,8 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
                     w[tap][0] = make_float2(t.x, t.y);
                     w[tap][1] = make_float2(t.z, t.w);
                 }
-                // halo rows r, r+1, r+2 are grid rows y-1, y, y+1; halo column x+1 is grid column x
+                // buffer rows r, r+1, r+2 are grid rows y-1, y, y+1; buffer column x+1 is grid column x
                 const T* hp = sH + (r * HP) * DK + cq * 4;
-                const float* pp = sPatchAll + (r * W) * PO + cq * 4;
-                T* op = gO + (size_t)(r * W) * DK + cq * 4;
                 float2 ca[3][2], cb[3][2], cc[3][2];
                 auto load_col = [&](int hx, float2 (&c)[3][2]) {
 #pragma unroll
@@ -738,35 +720,35 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
                 }
             } else {
                 for (int x = x0; x < x1; ++x) {
-                    const int tl = r * W + x;
-                    const float4 a4 = *reinterpret_cast<const float4*>(sPatchAll + (size_t)tl * PO + cq * 4);
+                    const float4 a4 = *reinterpret_cast<const float4*>(pp + x * PO);
                     uint2 outw;
                     outw.x = pack2<T>(a4.x, a4.y);
                     outw.y = pack2<T>(a4.z, a4.w);
-                    *reinterpret_cast<uint2*>(gO + (size_t)tl * DK + cq * 4) = outw;
+                    *reinterpret_cast<uint2*>(op + x * DK) = outw;
                 }
             }
         }
     }
-    __syncthreads();     // shared memory is free for the next task
+    fence_proxy_async();   // this task's plain shared-memory writes precede the next task's TMA writes
+    __syncthreads();       // shared memory is free for the next task
     TRACE(slot, 5);
 }
 
 // ---------------------------------------------------------------------------------- kernel
-template <typename T, int DK>
+template <typename T>
 __global__ void __launch_bounds__(NT, 2) fused_kernel(const __grid_constant__ FusedArgs p) {
-    extern __shared__ __align__(16) unsigned char smem[];
+    extern __shared__ unsigned char smem_raw[];
     __shared__ int s_task, s_flag, s_whead;
+    // TMA tiles with the 128-byte swizzle want a 1024-byte aligned base
+    unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     const int tid = threadIdx.x;
-    {   // zero once: rows >= n of the resident A / V_A must be finite zeros for the whole kernel
-        uint4* z = reinterpret_cast<uint4*>(smem);
-        for (int i = tid; i < (int)(FusedSmem<DK>::kTotal / 16); i += NT) z[i] = make_uint4(0, 0, 0, 0);
-    }
-    if (tid == 0) s_whead = -1;
-    __syncthreads();
-    if (tid < RP) {   // column DK of the resident V_A rows holds 1 (row sums of P from the P.V_A product)
-        T* sVA = reinterpret_cast<T*>(smem + FusedSmem<DK>::kA);
-        *reinterpret_cast<uint4*>(sVA + tid * FusedSmem<DK>::PA + DK) = make_uint4(pack2<T>(1.f, 0.f), 0u, 0u, 0u);
+    BlockState st;
+    st.bar_base = smem_u32(smem + OFF_BAR);
+    st.ph = 0u;
+    if (tid == 0) {
+        s_whead = -1;
+        for (int i = 0; i < kNumBars; ++i) mbar_init(st.bar_base + 8 * i, 1);
+        mbar_fence_init();
     }
     __syncthreads();
     const int G = p.plan.g_tasks, B = p.plan.b_tasks, Lg = p.plan.lag, S = p.slabs;
@@ -796,8 +778,8 @@ __global__ void __launch_bounds__(NT, 2) fused_kernel(const __grid_constant__ Fu
             const int step = t / B;
             slab = S - Lg + step; sub = t - step * B; is_g = false;
         }
-        if (is_g) run_g_task<T, DK>(p, slab, sub, smem, &s_flag, slot);
-        else      run_b_task<T, DK>(p, slab, sub, smem, &s_whead, slot);
+        if (is_g) run_g_task<T>(p, slab, sub, smem, st, &s_flag, slot);
+        else      run_b_task<T>(p, slab, sub, smem, st, &s_whead, slot);
 #ifdef AA_FUSED_TRACE
         if (tid == 0 && g_trace && slot < 16) {
             g_trace[((size_t)blockIdx.x * 16 + slot) * 8 + 6] = is_g ? 1 : 2;
@@ -808,15 +790,15 @@ __global__ void __launch_bounds__(NT, 2) fused_kernel(const __grid_constant__ Fu
     }
 }
 
-template <typename T, int DK>
+template <typename T>
 static int fused_occupancy() {
     int occ = 0;
-    auto kern = fused_kernel<T, DK>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FusedSmem<DK>::kTotal) != cudaSuccess) {
+    auto kern = fused_kernel<T>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess) {
         cudaGetLastError();
         return 0;
     }
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, NT, FusedSmem<DK>::kTotal) != cudaSuccess) {
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, NT, kSmemBytes) != cudaSuccess) {
         cudaGetLastError();
         return 0;
     }
@@ -827,7 +809,7 @@ static int fused_occupancy() {
 static bool fused_shape_plan(int dtype, int H, int W, int d, int n_agents, FusedPlan* pl) {
     memset(pl, 0, sizeof(*pl));
     if (dtype != kBF16 && dtype != kF16) return false;
-    if (d != 32 && d != 64) return false;
+    if (d != DK) return false;
     if (n_agents < 1 || n_agents > RP || W > MAXW || W < MINW || H < 1) return false;
     int p = 1;
     while (p * p < n_agents) ++p;
@@ -857,36 +839,43 @@ int fused_parts_per_slab(int dtype, int H, int W, int d, int n_agents) {
 FusedPlan plan_fused(int dtype, int slabs, int H, int W, int d, int n_agents, int sm_count) {
     FusedPlan pl;
     if (!fused_shape_plan(dtype, H, W, d, n_agents, &pl)) { pl.ok = false; return pl; }
-    int occ;
-    if (dtype == kBF16) occ = d == 64 ? fused_occupancy<__nv_bfloat16, 64>() : fused_occupancy<__nv_bfloat16, 32>();
-    else                occ = d == 64 ? fused_occupancy<__half, 64>() : fused_occupancy<__half, 32>();
+    if (!encode_tiled_fn()) return pl;            // no tensor-map encoder: use the per-step kernels
+    int occ = dtype == kBF16 ? fused_occupancy<__nv_bfloat16>() : fused_occupancy<__half>();
     if (occ < 1) return pl;
     if (occ > 2) occ = 2;
     const long long total = (long long)slabs * (pl.g_tasks + pl.b_tasks);
     long long grid = (long long)occ * sm_count;
     if (grid > total) grid = total;
     pl.grid = (int)grid;
-    if (pl.grid < pl.g_tasks || pl.g_tasks > 32) return pl;      // progress needs a resident block per G sibling
+    if (pl.grid < pl.g_tasks) return pl;          // progress needs a resident block per G sibling
     int lag = (5 * pl.grid / 2 + pl.g_tasks + pl.b_tasks - 1) / (pl.g_tasks + pl.b_tasks) + 2;
     if (const char* e = getenv("AA_FUSED_LAG")) lag = atoi(e);
     if (lag > slabs) lag = slabs;
     if (lag < 1) lag = 1;
     pl.lag = lag;
-    pl.smem = d == 64 ? FusedSmem<64>::kTotal : FusedSmem<32>::kTotal;
+    pl.smem = kSmemBytes;
     pl.ok = true;
     return pl;
 }
 
-template <typename T, int DK>
-static cudaError_t launch_fused_t(const FusedArgs& a, cudaStream_t st) {
-    fused_kernel<T, DK><<<a.plan.grid, NT, FusedSmem<DK>::kTotal, st>>>(a);
-    return cudaGetLastError();
+// Fills the tensor maps of `a` from its pointers and shape; false if one cannot be encoded.
+bool fused_make_maps(FusedArgs* a) {
+    const uint64_t N = (uint64_t)a->H * a->W, S = a->slabs;
+    if (!make_map_2d_u16(&a->tm_k, a->k, S * N, DK, KT, DK)) return false;
+    if (!make_map_2d_u16(&a->tm_v, a->v, S * N, DK, KT, DK)) return false;
+    if (!make_map_2d_u16(&a->tm_a, a->a_ws, S * a->n, DK, RP, DK)) return false;
+    if (!make_map_2d_u16(&a->tm_va, a->va_ws, S * a->n, DK, RP, DK)) return false;
+    a->b1_tma = 0;
+    if (a->b1 && N % 8 == 0 && ((uint64_t)a->plan.rows_per_g * a->W) % 8 == 0 && N >= KT)
+        a->b1_tma = make_map_2d_u16(&a->tm_b1, a->b1, (uint64_t)a->heads * a->n, N, RP, KT) ? 1 : 0;
+    return true;
 }
 
 cudaError_t launch_fused(int dtype, const FusedArgs& a, cudaStream_t st) {
-    if (dtype == kBF16) return a.d == 64 ? launch_fused_t<__nv_bfloat16, 64>(a, st) : launch_fused_t<__nv_bfloat16, 32>(a, st);
-    if (dtype == kF16)  return a.d == 64 ? launch_fused_t<__half, 64>(a, st) : launch_fused_t<__half, 32>(a, st);
-    return cudaErrorInvalidValue;
+    if (dtype == kBF16) fused_kernel<__nv_bfloat16><<<a.plan.grid, NT, kSmemBytes, st>>>(a);
+    else if (dtype == kF16) fused_kernel<__half><<<a.plan.grid, NT, kSmemBytes, st>>>(a);
+    else return cudaErrorInvalidValue;
+    return cudaGetLastError();
 }
 
 }  // namespace aa

@@ -1,6 +1,7 @@
 // Host-side launch interface between the C ABI (api.cu) and the kernel files.
 #pragma once
 
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stddef.h>
 #include <stdint.h>
@@ -60,7 +61,7 @@ cudaError_t launch_broadcast_simt(int dtype, const AttnArgs& p, cudaStream_t st)
 cudaError_t launch_aggregate_mma(int dtype, const AttnArgs& p, const AggPlan& plan, cudaStream_t st);
 cudaError_t launch_broadcast_mma(int dtype, const AttnArgs& p, cudaStream_t st);
 
-// Whole module (Eq. 6) in one persistent kernel for small agent counts (n <= 64, d in {32, 64},
+// Whole module (Eq. 6) in one persistent kernel for small agent counts (n <= 64, d = 64,
 // block pooling, W <= 64).  Blocks take tasks from a device-side queue: "G" tasks pool their token
 // range of Q, publish those agent rows, wait for the slab's other G tasks, and aggregate their
 // range of K/V; "B" tasks wait for the slab's merged V_A and do the broadcast + DWC for one
@@ -87,8 +88,13 @@ struct FusedArgs {
     int slabs, heads, H, W, d, n, p;
     float scale1, scale2;
     FusedPlan plan;
+    // TMA descriptors (128-byte swizzle, 64-column boxes): K and V as [slabs*N][d] with 64-row boxes,
+    // B1 as [heads*n][N] with 64x64 boxes, A and V_A workspaces as [slabs*n][d] with 64-row boxes
+    int b1_tma;           // B1 tiles come through TMA (needs N % 8 == 0 and 8-aligned task ranges)
+    alignas(64) CUtensorMap tm_k, tm_v, tm_b1, tm_a, tm_va;
 };
 FusedPlan plan_fused(int dtype, int slabs, int H, int W, int d, int n_agents, int sm_count);
+bool fused_make_maps(FusedArgs* a);     // encode the tensor maps from a's pointers and shape
 cudaError_t launch_fused(int dtype, const FusedArgs& a, cudaStream_t st);
 int fused_parts_per_slab(int dtype, int H, int W, int d, int n_agents);   // 0 if the shape is not eligible
 inline size_t fused_counter_words(int slabs) { return 3 * (size_t)slabs + 4; }
