@@ -198,10 +198,10 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
             float acc[8];
 #pragma unroll
             for (int k = 0; k < 8; ++k) acc[k] = 0.f;
-            for (int ib = tsub; ib < cnt; ib += 8 * tpl) {     // eight loads in flight per lane
-                uint4 raw[8];
+            for (int ib = tsub; ib < cnt; ib += 16 * tpl) {    // sixteen loads in flight per lane
+                uint4 raw[16];
 #pragma unroll
-                for (int u = 0; u < 8; ++u) {
+                for (int u = 0; u < 16; ++u) {
                     const int i = ib + u * tpl;
                     raw[u] = make_uint4(0u, 0u, 0u, 0u);
                     if (i < cnt) {
@@ -211,7 +211,7 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
                     }
                 }
 #pragma unroll
-                for (int u = 0; u < 8; ++u) {
+                for (int u = 0; u < 16; ++u) {
                     float f[8];
                     unpack16<T>(raw[u], f);
 #pragma unroll
@@ -848,7 +848,13 @@ FusedPlan plan_fused(int dtype, int slabs, int H, int W, int d, int n_agents, in
     if (grid > total) grid = total;
     pl.grid = (int)grid;
     if (pl.grid < pl.g_tasks) return pl;          // progress needs a resident block per G sibling
+    // The aggregation runs ahead of the broadcast by `lag` slabs: far enough that B tasks rarely wait
+    // for their slab's flag, close enough that the Q and V of the slabs in between stay in L2
+    // (budget: half of a 126 MB L2 for those re-reads).
+    const long long slab_qv_bytes = 2LL * H * W * d * 2;
+    long long lag_l2 = (64LL << 20) / slab_qv_bytes;
     int lag = (5 * pl.grid / 2 + pl.g_tasks + pl.b_tasks - 1) / (pl.g_tasks + pl.b_tasks) + 2;
+    if (lag_l2 > lag) lag = (int)(lag_l2 > 1000000 ? 1000000 : lag_l2);
     if (const char* e = getenv("AA_FUSED_LAG")) lag = atoi(e);
     if (lag > slabs) lag = slabs;
     if (lag < 1) lag = 1;
