@@ -31,6 +31,9 @@ METRIC = "agent-attention fwd tokens/s and % of HBM roofline at N=3136,n=49,d=64
 UNIT = "tokens/s"
 DEFAULT_WORKLOAD = "cfg3_pvt_bf16"
 L2_BYTES = 126 * 1024 * 1024
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu captures
+# summarised under profiles/ (None where the kernel has changed since its counters were taken)
+NCU_TRAFFIC = {("cfg3_pvt_bf16", "fused_kernel"): 103.56e6}
 
 
 def measured_peaks():
@@ -221,38 +224,45 @@ def main():
     tokens_per_step = world * w.batch * w.tokens
     value = tokens_per_step / (ms_step * 1e-3)
 
-    # per-kernel durations: the same steps issued through the step-level entry points with an
-    # event between kernels (on the launching stream)
-    kb_steps = min(args.steps, 200)
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(kb_steps)]
-    a_buf = torch.empty((w.batch, w.heads, w.agents, w.head_dim), dtype=dt, device=dev)
-    va_buf = torch.empty_like(a_buf)
-    torch.cuda.synchronize()
-    for i in range(kb_steps):
-        d = sets[i % n_sets]
-        evs[i][0].record(stream)
-        mod.pool(d["q"], w.grid_h, w.grid_w, w.pool, w.pool, out=a_buf, stream=stream)
-        evs[i][1].record(stream)
-        mod.aggregate(a_buf, d["k"], d["v"], b1=d["b1"], out=va_buf, workspace=ws, stream=stream)
-        evs[i][2].record(stream)
-        mod.broadcast(d["q"], a_buf, va_buf, d["v"], w.grid_h, w.grid_w, b2=d["b2"], dwc_weight=d["dwc"],
-                      out=d["out"], stream=stream)
-        evs[i][3].record(stream)
-    torch.cuda.synchronize()
-    kern_ms = {nm: statistics.mean(evs[i][j].elapsed_time(evs[i][j + 1]) for i in range(kb_steps))
-               for j, nm in enumerate(("pool", "aggregate", "broadcast_dwc"))}
     s = w.elem_bytes
     unit = w.slabs * w.tokens * w.head_dim * s                       # one [B,h,N,d] tensor
     bias_b = w.heads * w.agents * w.tokens * s if w.bias else 0
-    kern_bytes = {"pool": unit, "aggregate": 2 * unit + bias_b,
-                  "broadcast_dwc": unit + bias_b + (9 * w.heads * w.head_dim * s if w.dwc else 0)}
-    dominant = max(kern_ms, key=kern_ms.get)
     peak, peak_src = measured_peaks()
+    if launches_per_step == 1:
+        # the whole path is one persistent kernel: its launch duration is the step time (the only other
+        # node on the stream is a few-hundred-byte memset), its algorithmic bytes are the path's
+        dominant = "fused_kernel"
+        kern_ms = {dominant: ms_step}
+        kern_bytes = {dominant: set_bytes}
+    else:
+        # one kernel per step of the path: time each between events on the launching stream, through the
+        # step-level entry points
+        kb_steps = min(args.steps, 200)
+        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(kb_steps)]
+        a_buf = torch.empty((w.batch, w.heads, w.agents, w.head_dim), dtype=dt, device=dev)
+        va_buf = torch.empty_like(a_buf)
+        torch.cuda.synchronize()
+        for i in range(kb_steps):
+            d = sets[i % n_sets]
+            evs[i][0].record(stream)
+            mod.pool(d["q"], w.grid_h, w.grid_w, w.pool, w.pool, out=a_buf, stream=stream)
+            evs[i][1].record(stream)
+            mod.aggregate(a_buf, d["k"], d["v"], b1=d["b1"], out=va_buf, workspace=ws, stream=stream)
+            evs[i][2].record(stream)
+            mod.broadcast(d["q"], a_buf, va_buf, d["v"], w.grid_h, w.grid_w, b2=d["b2"], dwc_weight=d["dwc"],
+                          out=d["out"], stream=stream)
+            evs[i][3].record(stream)
+        torch.cuda.synchronize()
+        kern_ms = {nm: statistics.mean(evs[i][j].elapsed_time(evs[i][j + 1]) for i in range(kb_steps))
+                   for j, nm in enumerate(("pool", "aggregate", "broadcast_dwc"))}
+        kern_bytes = {"pool": unit, "aggregate": 2 * unit + bias_b,
+                      "broadcast_dwc": unit + bias_b + (9 * w.heads * w.head_dim * s if w.dwc else 0)}
+        dominant = max(kern_ms, key=kern_ms.get)
     dom_gbs = kern_bytes[dominant] / (kern_ms[dominant] * 1e-3) / 1e9
     path_gbs = set_bytes / (ms_step * 1e-3) / 1e9
     roofline = {
         "bound": "hbm", "kernel": dominant, "achieved": dom_gbs, "peak": peak, "unit": "GB/s",
-        "frac": dom_gbs / peak, "traffic": None, "peak_source": peak_src,
+        "frac": dom_gbs / peak, "traffic": NCU_TRAFFIC.get((w.name, dominant)), "peak_source": peak_src,
         "kernel_ms": kern_ms, "kernel_algorithmic_bytes": kern_bytes,
         "path_achieved": path_gbs, "path_frac": path_gbs / peak, "path_frac_nominal_8TBs": path_gbs / 8000.0,
         "path_algorithmic_bytes": set_bytes, "path_tflops": flops_of(w) / (ms_step * 1e-3) / 1e12,
