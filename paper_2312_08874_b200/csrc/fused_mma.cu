@@ -8,8 +8,8 @@
 //   G task (slab, range of grid rows): start the K/V/B1 tile ring (TMA, 128-byte swizzle), pool Q
 //     over the range (whole pooling windows: complete agent rows), publish them, wait until the
 //     slab's other G tasks have published theirs, then run the split aggregation over the range
-//     (Eq. 3, Eq. 5).  The last G task of a slab merges the partial states into V_A and raises the
-//     slab's flag.
+//     (Eq. 3, Eq. 5).  When all G tasks of the slab have written their partial states, each merges
+//     its share of the agent rows into V_A and counts itself done on the slab's flag.
 //   B task (slab, tile of whole grid rows, <= 128 tokens): start the bulk copies of the V rows
 //     (with their 3x3 halo) and of the B2 tile, load Q fragments straight into registers, wait for
 //     the slab's flag, fetch A and V_A (TMA), then broadcast + DWC (Eq. 3, Eq. 5, Eq. 6).
@@ -90,9 +90,17 @@ __device__ __forceinline__ void publish_add(unsigned* ctr) {
     __syncthreads();
     if (threadIdx.x == 0) { __threadfence(); atomicAdd(ctr, 1u); }
 }
-// All threads wait for a phase of an mbarrier; on expiry the block records `code` and goes on.
+// Thread 0 waits (bounded, with back-off so that it does not eat issue slots) for a phase of an
+// mbarrier; the caller follows with __syncthreads(), which passes the completed copies on to the
+// rest of the block.  On expiry the block records `code` and goes on.
 __device__ __forceinline__ void wait_bar(uint32_t bar, uint32_t parity, int* status, int code) {
-    if (!mbar_wait_bounded(bar, parity, kBarLimit)) atomicExch(status, code);
+    if (threadIdx.x == 0) {
+        unsigned tries = 0;
+        while (!mbar_try_wait(bar, parity)) {
+            if (++tries > kBarLimit) { atomicExch(status, code); break; }
+            __nanosleep(32);
+        }
+    }
 }
 // Byte offset of element (row, col) in a swizzled [rows][64] tile of 16-bit elements: the 16-byte
 // chunk index is XORed with the row index modulo 8 (the TMA 128-byte swizzle).
@@ -244,6 +252,7 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
     }
     wait_bar(bar_agents(st), (st.ph >> kBitAgents) & 1u, p.status, kTimeoutLoads);
     st.ph ^= 1u << kBitAgents;
+    __syncthreads();
 
     const int g = lane >> 2, t4 = lane & 3, xr = lane & 7;
     const int r0 = wm * 16, kw0 = wk * KW;
@@ -264,9 +273,10 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
     // 5. online-softmax aggregation over the range
     for (int it = 0; it < tiles; ++it) {
         const int s = it % STAGES;
-        if (it + STAGES - 1 < tiles) issue_tile(it + STAGES - 1, (it + STAGES - 1) % STAGES);
         wait_bar(bar_full(st, s), (st.ph >> s) & 1u, p.status, kTimeoutTile);
         st.ph ^= 1u << s;
+        __syncthreads();               // tile `it` has landed, and every warp is done with tile it-1
+        if (it + STAGES - 1 < tiles) issue_tile(it + STAGES - 1, (it + STAGES - 1) % STAGES);
         const unsigned char* sK = ring + s * kStageBytes;
         const unsigned char* sV = sK + kTileBytes;
         const unsigned char* sB = sV + kTileBytes;
@@ -352,8 +362,8 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
             }
             mma16816<T>(accl, pa, ones, ones);
         }
-        __syncthreads();               // every warp is done with stage s before it is refilled
     }
+    __syncthreads();                   // every warp is done with the ring
 
     // row sums sit in column 0 of the extra product: lanes with t4 == 0 hold them
     const float l0 = __shfl_sync(0xffffffffu, accl[0], lane & ~3);
@@ -361,9 +371,7 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
 
     TRACE(slot, 4);
     // 6. the two key halves of the block combine through shared memory into one partial state;
-    //    the slab's last G task merges all partials and raises the slab's flag
     float* sX = reinterpret_cast<float*>(ring);        // [4 row groups][36 values][32 lanes]
-    float* sWgt = sX + 4 * 36 * 32;                    // merge weights [parts][RP]
     if (wk == 1) {
         float* x = sX + wm * 36 * 32 + lane;
         x[0] = m0; x[32] = m1; x[64] = l0; x[96] = l1;
@@ -400,46 +408,41 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
                 make_float2(acc[j][2] * wa1 + x[(6 + 4 * j) * 32] * wb1, acc[j][3] * wa1 + x[(7 + 4 * j) * 32] * wb1);
         }
     }
-    unsigned* ticket = p.counters + p.slabs + slab;
-    if (arrive_is_last(ticket, (unsigned)p.plan.g_tasks, s_flag)) {
-        // step 1: one thread per agent row turns the parts' (max, sum) into normalised weights
-        if (tid < n) {
-            float mj[32], mmax = -INFINITY, den = 0.f;
-#pragma unroll
-            for (int q = 0; q < 32; ++q) {
-                mj[q] = (q < parts) ? __ldcg(slab_parts + q * pf + tid) : -INFINITY;
-                mmax = fmaxf(mmax, mj[q]);
-            }
-#pragma unroll
-            for (int q = 0; q < 32; ++q) {
-                if (q < parts) {
-                    mj[q] = (mj[q] == -INFINITY) ? 0.f : exp2f(mj[q] - mmax);
-                    den += mj[q] * __ldcg(slab_parts + q * pf + RP + tid);
-                }
-            }
-            const float inv = 1.f / den;
-#pragma unroll
-            for (int q = 0; q < 32; ++q) if (q < parts) sWgt[q * RP + tid] = mj[q] * inv;
-        }
-        __syncthreads();
-        // step 2: V_A[r][c..c+3] = sum over parts of weight * acc, in the fixed order of the parts
+    // 7. when all of the slab's partial states are written, every G task merges its share of the
+    //    agent rows (fixed order of the parts: bit-reproducible) and counts itself done
+    unsigned* arrived = p.counters + p.slabs + slab;
+    publish_add(arrived);
+    wait_counter(arrived, (unsigned)p.plan.g_tasks, p.status, kTimeoutAgents);
+    {
+        const int rows_per = (n + p.plan.g_tasks - 1) / p.plan.g_tasks;
+        const int rb = sub * rows_per, re = min(n, rb + rows_per);
         T* va = static_cast<T*>(p.va_ws) + (size_t)slab * n * DK;
-        for (int e = tid; e < n * (DK / 4); e += NT) {
-            const int r = e / (DK / 4), c = (e - r * (DK / 4)) * 4;
+        for (int e = tid; e < (re - rb) * (DK / 4); e += NT) {
+            const int r = rb + e / (DK / 4), c = (e % (DK / 4)) * 4;
+            float mx = -INFINITY, den = 0.f;
             float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll 8
             for (int q = 0; q < parts; ++q) {
-                const float wq = sWgt[q * RP + r];
-                const float4 a = __ldcg(reinterpret_cast<const float4*>(slab_parts + q * pf + 2 * RP + (size_t)r * DK + c));
-                num.x += wq * a.x; num.y += wq * a.y; num.z += wq * a.z; num.w += wq * a.w;
+                const float* pq = slab_parts + q * pf;
+                const float mq = __ldcg(pq + r);
+                const float lq = __ldcg(pq + RP + r);
+                const float4 a = __ldcg(reinterpret_cast<const float4*>(pq + 2 * RP + (size_t)r * DK + c));
+                const float mn = fmaxf(mx, mq);
+                const float bs = (mn == -INFINITY) ? 0.f : mn;
+                const float c0 = exp2f(mx - bs), c1 = exp2f(mq - bs);
+                den = den * c0 + lq * c1;
+                num.x = num.x * c0 + a.x * c1; num.y = num.y * c0 + a.y * c1;
+                num.z = num.z * c0 + a.z * c1; num.w = num.w * c0 + a.w * c1;
+                mx = mn;
             }
+            const float inv = 1.f / den;
             uint2 o;
-            o.x = pack2<T>(num.x, num.y);
-            o.y = pack2<T>(num.z, num.w);
+            o.x = pack2<T>(num.x * inv, num.y * inv);
+            o.y = pack2<T>(num.z * inv, num.w * inv);
             *reinterpret_cast<uint2*>(va + (size_t)r * DK + c) = o;
         }
-        publish_add(p.counters + 2 * p.slabs + slab);
     }
+    publish_add(p.counters + 2 * p.slabs + slab);
     fence_proxy_async();   // this task's plain shared-memory writes precede the next task's TMA writes
     __syncthreads();       // the ring is free for the next task
     TRACE(slot, 5);
@@ -482,7 +485,8 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
     const unsigned* va_flag = p.counters + 2 * p.slabs + slab;
 
     TRACE(slot, 0);
-    const bool early = ld_acquire(va_flag) >= 1u;      // usual case: the slab's aggregation is long done
+    const unsigned va_target = (unsigned)p.plan.g_tasks;   // every G task of the slab merged its rows
+    const bool early = ld_acquire(va_flag) >= va_target;      // usual case: the slab's aggregation is long done
     auto issue_agents = [&]() {
         if (tid == 0) {
             mbar_arrive_expect_tx(bar_agents(st), 2 * kTileBytes);
@@ -549,7 +553,7 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
 
     TRACE(slot, 1);
     // 2. wait for the slab's agent features, then fetch A and V_A (L2)
-    wait_counter(va_flag, 1u, p.status, kTimeoutFeatures);
+    wait_counter(va_flag, va_target, p.status, kTimeoutFeatures);
     TRACE(slot, 2);
     if (tid == 0 && has_dwc) *s_whead = head;
     if (!early) issue_agents();
@@ -559,6 +563,7 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
         wait_bar(bar_bin(st), (st.ph >> kBitBin) & 1u, p.status, kTimeoutLoads);
         st.ph ^= 1u << kBitBin;
     }
+    __syncthreads();
     // rows >= n of the V_A tile hold foreign rows: they must be zero, since 0 * NaN is not 0
     for (int e = tid; e < (RP - n) * 8; e += NT)
         *(reinterpret_cast<uint4*>(sVA + (n + e / 8) * 128) + (e & 7)) = make_uint4(0, 0, 0, 0);
