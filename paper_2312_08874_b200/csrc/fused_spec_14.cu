@@ -1,0 +1,10 @@
+// Fused persistent kernel specialised at compile time for the 14x14 token grid with 7x7 agents,
+// both biases and the depthwise term present (a layer shape of the paper's App. G).
+#include "fused_kernel.cuh"
+
+namespace aa {
+int fused_occupancy_s14(int dtype) { return fused_occupancy_dt<FusedShape<14, 14, 7>>(dtype); }
+cudaError_t launch_fused_s14(int dtype, const FusedArgs& a, cudaStream_t st) {
+    return fused_launch_dt<FusedShape<14, 14, 7>>(dtype, a, st);
+}
+}  // namespace aa

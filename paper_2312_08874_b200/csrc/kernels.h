@@ -75,6 +75,7 @@ struct FusedPlan {
     int lag;            // slabs between a slab's G tasks and its B tasks in the queue
     int grid;           // resident blocks
     int parts;          // partial states per slab
+    int spec;           // 0 = generic kernel, else index of a kernel specialised for this shape
     size_t smem;        // dynamic shared memory per block
 };
 struct FusedArgs {
