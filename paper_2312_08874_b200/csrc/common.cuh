@@ -13,17 +13,20 @@ constexpr float kLog2e = 1.4426950408889634f;
 // ----------------------------------------------------------------------------- element types
 template <typename T> struct Elem;
 template <> struct Elem<float> {
-    static constexpr int kVec = 4;                       // elements per 16-byte vector
+    static constexpr int kVec = 4;
+    static constexpr bool kIsBf16 = false;                       // elements per 16-byte vector
     __device__ static float to_f32(float x) { return x; }
     __device__ static float from_f32(float x) { return x; }
 };
 template <> struct Elem<__nv_bfloat16> {
     static constexpr int kVec = 8;
+    static constexpr bool kIsBf16 = true;
     __device__ static float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
     __device__ static __nv_bfloat16 from_f32(float x) { return __float2bfloat16_rn(x); }
 };
 template <> struct Elem<__half> {
     static constexpr int kVec = 8;
+    static constexpr bool kIsBf16 = false;
     __device__ static float to_f32(__half x) { return __half2float(x); }
     __device__ static __half from_f32(float x) { return __float2half_rn(x); }
 };

@@ -24,6 +24,7 @@
 #include "kernels.h"
 #include "merge.cuh"
 #include "tma.cuh"
+#include "umma.cuh"
 
 namespace aa {
 
@@ -51,7 +52,7 @@ constexpr int OFF_UNION = 19456;                        // 19 KiB: start of the 
 constexpr int kStageBytes = 3 * kTileBytes;
 constexpr int kGBytes = STAGES * kStageBytes;
 // B tasks: fp32 patch | V rows with zero borders | B2 tile
-constexpr int PO = DK + 8;                              // patch pitch (floats)
+constexpr int PO = DK + 4;                              // patch pitch (floats): row-per-thread 16-byte stores spread over all banks
 constexpr int OFF_PATCH = OFF_UNION;
 constexpr int kPatchBytes = QT * PO * 4;
 constexpr int OFF_HALO = OFF_PATCH + kPatchBytes;
@@ -60,7 +61,9 @@ constexpr int OFF_B2 = OFF_HALO + kHaloBytes;
 constexpr int kB2Bytes = QT * RP * 2 + 16;              // + one spare vector: pairs are read as two words
 constexpr int kBBytes = kPatchBytes + kHaloBytes + kB2Bytes;
 constexpr int OFF_BAR = OFF_UNION + (kGBytes > kBBytes ? kGBytes : kBBytes);   // mbarriers (8 bytes each)
-constexpr int kNumBars = STAGES + 2;                    // ring stages, agents, broadcast inputs
+constexpr int kNumBars = STAGES + 3;                    // ring stages, agents, broadcast inputs, MMA completion
+constexpr int kTmemCols = 128;                          // per block: 64 columns of logits + 64 of output
+static_assert(kPatchBytes >= 2 * QT * 128, "the Q and P operand tiles alias the patch");
 constexpr int kSmemBytes = OFF_BAR + 8 * kNumBars + 1024;   // + slack to align the base to 1024
 static_assert(OFF_W + 9 * DK * 4 <= OFF_UNION, "common area overflows");
 static_assert(OFF_UNION % 1024 == 0 && kStageBytes % 1024 == 0 && OFF_BAR % 8 == 0, "alignment");
@@ -132,12 +135,16 @@ __device__ __forceinline__ void copy_flat(unsigned char* dst, const unsigned cha
 // Block-level state that persists across tasks: mbarrier phase parities.
 struct BlockState {
     uint32_t bar_base;          // shared address of the first mbarrier
-    uint32_t ph;                // parity to wait for next: bit s = ring stage s, then agents, broadcast inputs
+    uint32_t ph;                // parity to wait for next: bit s = ring stage s, then agents, broadcast inputs, MMA
+    uint32_t tmem;              // base address of this block's tensor-memory columns
 };
-constexpr int kBitAgents = STAGES, kBitBin = STAGES + 1;
+constexpr int kBitAgents = STAGES, kBitBin = STAGES + 1, kBitMma = STAGES + 2;
 __device__ __forceinline__ uint32_t bar_full(const BlockState& st, int s) { return st.bar_base + 8 * s; }
 __device__ __forceinline__ uint32_t bar_agents(const BlockState& st) { return st.bar_base + 8 * STAGES; }
 __device__ __forceinline__ uint32_t bar_bin(const BlockState& st) { return st.bar_base + 8 * (STAGES + 1); }
+__device__ __forceinline__ uint32_t bar_mma(const BlockState& st) { return st.bar_base + 8 * (STAGES + 2); }
+// barrier among the 128 threads of warps 0-3 (the threads that own TMEM lanes in the broadcast)
+__device__ __forceinline__ void sync_rows() { asm volatile("bar.sync 1, 128;\n" ::: "memory"); }
 }  // namespace
 
 // Compile-time shape: a kernel instantiated for one token grid and agent grid (with biases and the
@@ -475,7 +482,6 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
     const int y0 = tile * R;
     const int rows = min(R, H - y0);
     const int q0 = y0 * W, TQ = rows * W;            // tokens of this tile
-    const bool warp_active = warp * 16 < TQ;
     const bool has_dwc = SH::kFixed ? true : (p.dwc_w != nullptr);
     const bool has_b2 = SH::kFixed ? true : (p.b2 != nullptr);
     const int HP = W + 2;                             // V-row pitch in tokens (zero columns at both ends)
@@ -485,7 +491,6 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
     unsigned char* sVA = smem + OFF_VA;
     float* sW = reinterpret_cast<float*>(smem + OFF_W);
     float* sPatchAll = reinterpret_cast<float*>(smem + OFF_PATCH);   // [128][PO] fp32
-    float* sPatch = sPatchAll + warp * 16 * PO;
     T* sH = reinterpret_cast<T*>(smem + OFF_HALO);                   // [(rows+2)][W+2][DK]
     T* sB2 = reinterpret_cast<T*>(smem + OFF_B2);                    // [TQ][n] flat
 
@@ -509,10 +514,12 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
     const bool b2_bulk = has_b2 && ((reinterpret_cast<uintptr_t>(b2src) & 15u) == 0) && ((b2bytes & 15) == 0);
     int vrows = 0;
     if (has_dwc) vrows = min(H, y0 + rows + 1) - max(0, y0 - 1);
-    const uint32_t bin_bytes = (uint32_t)vrows * W * DK * 2 + (b2_bulk ? b2bytes : 0);
-    if (tid == 0 && bin_bytes) {
+    const uint32_t bin_bytes = (uint32_t)QT * DK * 2 + (uint32_t)vrows * W * DK * 2 + (b2_bulk ? b2bytes : 0);
+    if (tid == 0) {
         const uint32_t bar = bar_bin(st);
         mbar_arrive_expect_tx(bar, bin_bytes);
+        // Q tile: 128 rows from the tile's first token (rows past the tile feed rows that are never stored)
+        tma_load_2d(smem_u32(smem + OFF_PATCH), &p.tm_q, 0, slab * N + q0, bar);
         if (has_dwc) {
             for (int hr = 0; hr < rows + 2; ++hr) {
                 const int y = y0 - 1 + hr;
@@ -523,20 +530,6 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
         if (b2_bulk) bulk_load_1d(smem_u32(sB2), b2src, b2bytes, bar);
     }
     if (early) issue_agents();
-    // Q fragments of this warp's 16 rows straight into registers
-    uint32_t qf[DK / 16][4];
-    {
-        const bool oka = (warp * 16 + g) < TQ, okb = (warp * 16 + g + 8) < TQ;
-        const uint32_t* ra = reinterpret_cast<const uint32_t*>(gQ + (size_t)(warp * 16 + g) * DK) + t4;
-        const uint32_t* rb = reinterpret_cast<const uint32_t*>(gQ + (size_t)(warp * 16 + g + 8) * DK) + t4;
-#pragma unroll
-        for (int ks = 0; ks < DK / 16; ++ks) {
-            qf[ks][0] = oka ? __ldg(ra + ks * 8) : 0u;
-            qf[ks][1] = okb ? __ldg(rb + ks * 8) : 0u;
-            qf[ks][2] = oka ? __ldg(ra + ks * 8 + 4) : 0u;
-            qf[ks][3] = okb ? __ldg(rb + ks * 8 + 4) : 0u;
-        }
-    }
     if (has_dwc) {
         // zero borders: columns x = -1 and x = W of every row, and rows that fall outside the grid
         for (int e = tid; e < (rows + 2) * 2 * (DK / 8); e += NT) {
@@ -576,101 +569,105 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
     // rows >= n of the V_A tile hold foreign rows: they must be zero, since 0 * NaN is not 0
     for (int e = tid; e < (RP - n) * 8; e += NT)
         *(reinterpret_cast<uint4*>(sVA + (n + e / 8) * 128) + (e & 7)) = make_uint4(0, 0, 0, 0);
+    fence_proxy_async();          // the tensor core reads V_A through the async proxy
     __syncthreads();
 
     TRACE(slot, 3);
-    // 3. attention part: 16 queries per warp against all agents
-    if (warp_active) {
-        const int lr_a = warp * 16 + g, lr_b = lr_a + 8;           // rows within the tile
-        float sc[RP / 8][4];
+    // 3. attention part on the 5th-generation tensor cores: logits S = Q A^T accumulate in tensor
+    //    memory, one thread per query row does the softmax on its row, the probabilities go back
+    //    through shared memory as the A operand of O = P V_A, and the normalised rows land in the patch
+    if (tid < 128) {
+        unsigned char* sQt = smem + OFF_PATCH;                 // [128][128 B] swizzled Q tile (TMA)
+        unsigned char* sPt = smem + OFF_PATCH + QT * 128;      // [128][128 B] swizzled P tile
+        constexpr int fmt = sizeof(T) == 2 && Elem<T>::kIsBf16 ? 1 : 0;
+        const uint32_t tS = st.tmem, tO = st.tmem + 64;
+        if (tid == 0) {
+            tc_fence_after_sync();
+            const uint32_t idesc = umma_idesc(fmt, 128, 64, 0);
 #pragma unroll
-        for (int j = 0; j < RP / 8; ++j) { sc[j][0] = sc[j][1] = sc[j][2] = sc[j][3] = 0.f; }
-#pragma unroll
-        for (int ks = 0; ks < DK / 16; ++ks) {
-#pragma unroll
-            for (int np = 0; np < RP / 16; ++np) {
-                if (np < n16) {
-                    uint32_t b0, b1, b2, b3;
-                    ldmatrix_x4(b0, b1, b2, b3,
-                                sA + (np * 16 + xr + (lane >> 4) * 8) * 128 + (((ks * 2 + ((lane >> 3) & 1)) ^ xr) << 4));
-                    mma16816<T>(sc[2 * np], qf[ks], b0, b1);
-                    if (2 * np + 1 < n8) mma16816<T>(sc[2 * np + 1], qf[ks], b2, b3);
-                }
-            }
+            for (int kk = 0; kk < DK / 16; ++kk)
+                umma_f16(tS, umma_desc_sw128(smem_u32(sQt) + kk * 32), umma_desc_sw128(smem_u32(sA) + kk * 32), idesc, kk > 0);
+            umma_commit(bar_mma(st));
         }
-        // logits in natural units: t = scale2 * q.a + b2; p = 2^((t - max) * log2 e)
-        float mx0 = -INFINITY, mx1 = -INFINITY;
+        wait_bar(bar_mma(st), (st.ph >> kBitMma) & 1u, p.status, kTimeoutLoads);
+        st.ph ^= 1u << kBitMma;
+        sync_rows();
+        tc_fence_after_sync();
+        const uint32_t lane_base = ((uint32_t)(32 * warp)) << 16;      // this warp's 32 rows
+        float s[64];
         {
-            // B2 rows are n (possibly odd) elements long, so a pair may straddle two 32-bit words
-            const uint32_t* w32 = reinterpret_cast<const uint32_t*>(sB2);
-            const int ea = lr_a * n + 2 * t4, eb = lr_b * n + 2 * t4;
-            const int sha = (ea & 1) * 16, shb = (eb & 1) * 16;
+            uint32_t r[32];
+            tmem_ld32(tS + lane_base, r);
+            tmem_ld_wait();
 #pragma unroll
-            for (int j = 0; j < RP / 8; ++j) {
-                if (j < n8) {
-                    float2 ba = make_float2(0.f, 0.f), bb = make_float2(0.f, 0.f);
-                    if (has_b2) {
-                        const int wa = (ea + 8 * j) >> 1, wb = (eb + 8 * j) >> 1;
-                        ba = unpack2<T>(__funnelshift_r(w32[wa], w32[wa + 1], sha));
-                        bb = unpack2<T>(__funnelshift_r(w32[wb], w32[wb + 1], shb));
-                    }
-                    sc[j][0] = fmaf(sc[j][0], p.scale2, ba.x);
-                    sc[j][1] = fmaf(sc[j][1], p.scale2, ba.y);
-                    sc[j][2] = fmaf(sc[j][2], p.scale2, bb.x);
-                    sc[j][3] = fmaf(sc[j][3], p.scale2, bb.y);
-                    if (8 * j + 8 > n) {     // last column tile: columns >= n are not agents
-                        const int col = 8 * j + 2 * t4;
-                        if (col >= n)     { sc[j][0] = -INFINITY; sc[j][2] = -INFINITY; }
-                        if (col + 1 >= n) { sc[j][1] = -INFINITY; sc[j][3] = -INFINITY; }
-                    }
-                    mx0 = fmaxf(mx0, fmaxf(sc[j][0], sc[j][1]));
-                    mx1 = fmaxf(mx1, fmaxf(sc[j][2], sc[j][3]));
-                }
+            for (int i = 0; i < 32; ++i) s[i] = __uint_as_float(r[i]);
+            tmem_ld32(tS + lane_base + 32, r);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) s[32 + i] = __uint_as_float(r[i]);
+        }
+        // logits in natural units: t = scale2 * q.a + b2; columns >= n are not agents
+        const int row = tid;
+        const uint32_t* w32 = reinterpret_cast<const uint32_t*>(sB2) + ((row * n) >> 1);
+        const int sh = ((row * n) & 1) * 16;     // rows are n (possibly odd) elements long
+        float mx = -INFINITY;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+            if (2 * j < n) {
+                float2 b = make_float2(0.f, 0.f);
+                if (has_b2) b = unpack2<T>(__funnelshift_r(w32[j], w32[j + 1], sh));
+                s[2 * j] = fmaf(s[2 * j], p.scale2, b.x);
+                s[2 * j + 1] = (2 * j + 1 < n) ? fmaf(s[2 * j + 1], p.scale2, b.y) : -INFINITY;
+                mx = fmaxf(mx, fmaxf(s[2 * j], s[2 * j + 1]));
             }
         }
-        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
-        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
-        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
-        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
-        const float nm0 = -mx0 * kLog2e, nm1 = -mx1 * kLog2e;
-        uint32_t pk[RP / 8][2];
+        const float nm = -mx * kLog2e;
+        float l = 0.f;
+        uint32_t pk[32];
 #pragma unroll
-        for (int j = 0; j < RP / 8; ++j) {
-            if (j < n8) {
-                pk[j][0] = pack2<T>(fast_exp2(fmaf(sc[j][0], kLog2e, nm0)), fast_exp2(fmaf(sc[j][1], kLog2e, nm0)));
-                pk[j][1] = pack2<T>(fast_exp2(fmaf(sc[j][2], kLog2e, nm1)), fast_exp2(fmaf(sc[j][3], kLog2e, nm1)));
+        for (int j = 0; j < 32; ++j) {
+            if (2 * j < n) {
+                const float p0 = fast_exp2(fmaf(s[2 * j], kLog2e, nm));
+                const float p1 = fast_exp2(fmaf(s[2 * j + 1], kLog2e, nm));      // exp2(-inf) = 0 past the last agent
+                pk[j] = pack2<T>(p0, p1);
+                const float2 q = unpack2<T>(pk[j]);    // the normaliser sums the rounded weights
+                l += q.x + q.y;
             } else {
-                pk[j][0] = 0u; pk[j][1] = 0u;
+                pk[j] = 0u;
             }
         }
-        const uint32_t ones = (g == 0) ? pack2<T>(1.f, 1.f) : 0u;      // column 0 of the extra product = row sums
-        float acc[DK / 8][4], accl[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-        for (int j = 0; j < DK / 8; ++j) { acc[j][0] = acc[j][1] = acc[j][2] = acc[j][3] = 0.f; }
-#pragma unroll
-        for (int kk = 0; kk < RP / 16; ++kk) {
-            if (kk < n16) {
-                const uint32_t pa[4] = {pk[2 * kk][0], pk[2 * kk][1], pk[2 * kk + 1][0], pk[2 * kk + 1][1]};
-#pragma unroll
-                for (int np = 0; np < DK / 16; ++np) {
-                    uint32_t b0, b1, b2, b3;
-                    ldmatrix_x4_trans(b0, b1, b2, b3,
-                                      sVA + (kk * 16 + xr + ((lane >> 3) & 1) * 8) * 128 + (((np * 2 + (lane >> 4)) ^ xr) << 4));
-                    mma16816<T>(acc[2 * np], pa, b0, b1);
-                    mma16816<T>(acc[2 * np + 1], pa, b2, b3);
-                }
-                mma16816<T>(accl, pa, ones, ones);
-            }
+        for (int c = 0; c < 8; ++c)
+            *reinterpret_cast<uint4*>(sPt + row * 128 + ((c ^ (row & 7)) << 4)) =
+                make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+        fence_proxy_async();              // the tensor core reads P through the async proxy
+        tc_fence_before_sync();
+        sync_rows();
+        if (tid == 0) {
+            tc_fence_after_sync();
+            const uint32_t idesc = umma_idesc(fmt, 128, 64, 1);       // V_A is [agents][d]: MN-major B operand
+            for (int kk = 0; kk < n16; ++kk)
+                umma_f16(tO, umma_desc_sw128(smem_u32(sPt) + kk * 32), umma_desc_sw128(smem_u32(sVA) + kk * 2048), idesc, kk > 0);
+            umma_commit(bar_mma(st));
         }
-        const float l0 = __shfl_sync(0xffffffffu, accl[0], lane & ~3);
-        const float l1 = __shfl_sync(0xffffffffu, accl[2], lane & ~3);
-        const float inv0 = 1.f / l0, inv1 = 1.f / l1;
+        wait_bar(bar_mma(st), (st.ph >> kBitMma) & 1u, p.status, kTimeoutLoads);
+        st.ph ^= 1u << kBitMma;
+        sync_rows();
+        tc_fence_after_sync();
+        const float inv = 1.f / l;
+        float* prow = sPatchAll + row * PO;
 #pragma unroll
-        for (int j = 0; j < DK / 8; ++j) {
-            const int col = 8 * j + 2 * t4;
-            *reinterpret_cast<float2*>(sPatch + g * PO + col) = make_float2(acc[j][0] * inv0, acc[j][1] * inv0);
-            *reinterpret_cast<float2*>(sPatch + (g + 8) * PO + col) = make_float2(acc[j][2] * inv1, acc[j][3] * inv1);
+        for (int h = 0; h < 2; ++h) {
+            uint32_t r[32];
+            tmem_ld32(tO + lane_base + 32 * h, r);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                *reinterpret_cast<float4*>(prow + 32 * h + 4 * i) =
+                    make_float4(__uint_as_float(r[4 * i]) * inv, __uint_as_float(r[4 * i + 1]) * inv,
+                                __uint_as_float(r[4 * i + 2]) * inv, __uint_as_float(r[4 * i + 3]) * inv);
         }
+        tc_fence_before_sync();
     }
     __syncthreads();
     TRACE(slot, 4);
@@ -753,6 +750,7 @@ template <typename T, typename SH>
 __global__ void __launch_bounds__(NT, 2) fused_kernel(const __grid_constant__ FusedArgs p) {
     extern __shared__ unsigned char smem_raw[];
     __shared__ int s_task, s_flag, s_whead;
+    __shared__ uint32_t s_tmem;
     // TMA tiles with the 128-byte swizzle want a 1024-byte aligned base
     unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     const int tid = threadIdx.x;
@@ -764,7 +762,12 @@ __global__ void __launch_bounds__(NT, 2) fused_kernel(const __grid_constant__ Fu
         for (int i = 0; i < kNumBars; ++i) mbar_init(st.bar_base + 8 * i, 1);
         mbar_fence_init();
     }
+    // tensor memory for the broadcast MMAs: warp 0 allocates (and frees at the end)
+    if (tid < 32) tmem_alloc(smem_u32(&s_tmem), kTmemCols);
+    tc_fence_before_sync();
     __syncthreads();
+    tc_fence_after_sync();
+    st.tmem = s_tmem;
     const int G = p.plan.g_tasks, B = p.plan.b_tasks, Lg = p.plan.lag, S = p.slabs;
     const int count0 = Lg * G, count1 = (S - Lg) * (G + B);
     const int total = S * (G + B);
@@ -802,6 +805,9 @@ __global__ void __launch_bounds__(NT, 2) fused_kernel(const __grid_constant__ Fu
 #endif
         ++slot;
     }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (tid < 32) tmem_dealloc(st.tmem, kTmemCols);
 }
 
 

@@ -86,6 +86,7 @@ bool fused_make_maps(FusedArgs* a) {
     const uint64_t N = (uint64_t)a->H * a->W, S = a->slabs;
     if (!make_map_2d_u16(&a->tm_k, a->k, S * N, DK, KT, DK)) return false;
     if (!make_map_2d_u16(&a->tm_v, a->v, S * N, DK, KT, DK)) return false;
+    if (!make_map_2d_u16(&a->tm_q, a->q, S * N, DK, QT, DK)) return false;
     if (!make_map_2d_u16(&a->tm_a, a->a_ws, S * a->n, DK, RP, DK)) return false;
     if (!make_map_2d_u16(&a->tm_va, a->va_ws, S * a->n, DK, RP, DK)) return false;
     a->b1_tma = 0;

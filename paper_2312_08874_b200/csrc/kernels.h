@@ -93,6 +93,7 @@ struct FusedArgs {
     // B1 as [heads*n][N] with 64x64 boxes, A and V_A workspaces as [slabs*n][d] with 64-row boxes
     int b1_tma;           // B1 tiles come through TMA (needs N % 8 == 0 and 8-aligned task ranges)
     alignas(64) CUtensorMap tm_k, tm_v, tm_b1, tm_a, tm_va;
+    alignas(64) CUtensorMap tm_q;     // Q as [slabs*N][d] with 128-row boxes (A operand of the broadcast MMA)
 };
 FusedPlan plan_fused(int dtype, int slabs, int H, int W, int d, int n_agents, int sm_count);
 bool fused_make_maps(FusedArgs* a);     // encode the tensor maps from a's pointers and shape
