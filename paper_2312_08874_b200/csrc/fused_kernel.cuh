@@ -471,7 +471,7 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
 // depthwise term (Eq. 6), round once and store.
 template <typename T, typename SH>
 __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int tile, unsigned char* smem,
-                                           BlockState& st, int* s_whead, int slot) {
+                                           BlockState& st, int* s_whead, float (*s_red)[128], int slot) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int head = slab % p.heads;
     const int H = SH::kFixed ? SH::kH : p.H, W = SH::kFixed ? SH::kW : p.W;
@@ -574,13 +574,16 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
 
     TRACE(slot, 3);
     // 3. attention part on the 5th-generation tensor cores: logits S = Q A^T accumulate in tensor
-    //    memory, one thread per query row does the softmax on its row, the probabilities go back
-    //    through shared memory as the A operand of O = P V_A, and the normalised rows land in the patch
-    if (tid < 128) {
+    //    memory; two threads share each query row (32 logit columns each: warps w and w+4 own the same
+    //    tensor-memory lanes), exchange their partial maxima and sums through shared memory, write the
+    //    probabilities back as the A operand of O = P V_A, and put the normalised row into the patch
+    {
         unsigned char* sQt = smem + OFF_PATCH;                 // [128][128 B] swizzled Q tile (TMA)
         unsigned char* sPt = smem + OFF_PATCH + QT * 128;      // [128][128 B] swizzled P tile
-        constexpr int fmt = sizeof(T) == 2 && Elem<T>::kIsBf16 ? 1 : 0;
+        constexpr int fmt = Elem<T>::kIsBf16 ? 1 : 0;
         const uint32_t tS = st.tmem, tO = st.tmem + 64;
+        const int half = warp >> 2, row = tid & 127, c0 = 32 * half;
+        const uint32_t lane_base = ((uint32_t)(32 * (warp & 3))) << 16;     // this warp's 32 rows
         if (tid == 0) {
             tc_fence_after_sync();
             const uint32_t idesc = umma_idesc(fmt, 128, 64, 0);
@@ -591,42 +594,39 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
         }
         wait_bar(bar_mma(st), (st.ph >> kBitMma) & 1u, p.status, kTimeoutLoads);
         st.ph ^= 1u << kBitMma;
-        sync_rows();
+        __syncthreads();
         tc_fence_after_sync();
-        const uint32_t lane_base = ((uint32_t)(32 * warp)) << 16;      // this warp's 32 rows
-        float s[64];
+        float s[32];
         {
             uint32_t r[32];
-            tmem_ld32(tS + lane_base, r);
+            tmem_ld32(tS + lane_base + c0, r);
             tmem_ld_wait();
 #pragma unroll
             for (int i = 0; i < 32; ++i) s[i] = __uint_as_float(r[i]);
-            tmem_ld32(tS + lane_base + 32, r);
-            tmem_ld_wait();
-#pragma unroll
-            for (int i = 0; i < 32; ++i) s[32 + i] = __uint_as_float(r[i]);
         }
         // logits in natural units: t = scale2 * q.a + b2; columns >= n are not agents
-        const int row = tid;
-        const uint32_t* w32 = reinterpret_cast<const uint32_t*>(sB2) + ((row * n) >> 1);
+        const uint32_t* w32 = reinterpret_cast<const uint32_t*>(sB2) + ((row * n) >> 1) + 16 * half;
         const int sh = ((row * n) & 1) * 16;     // rows are n (possibly odd) elements long
         float mx = -INFINITY;
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-            if (2 * j < n) {
+        for (int j = 0; j < 16; ++j) {
+            if (c0 + 2 * j < n) {
                 float2 b = make_float2(0.f, 0.f);
                 if (has_b2) b = unpack2<T>(__funnelshift_r(w32[j], w32[j + 1], sh));
                 s[2 * j] = fmaf(s[2 * j], p.scale2, b.x);
-                s[2 * j + 1] = (2 * j + 1 < n) ? fmaf(s[2 * j + 1], p.scale2, b.y) : -INFINITY;
+                s[2 * j + 1] = (c0 + 2 * j + 1 < n) ? fmaf(s[2 * j + 1], p.scale2, b.y) : -INFINITY;
                 mx = fmaxf(mx, fmaxf(s[2 * j], s[2 * j + 1]));
             }
         }
+        s_red[half][row] = mx;
+        __syncthreads();
+        mx = fmaxf(mx, s_red[half ^ 1][row]);
         const float nm = -mx * kLog2e;
         float l = 0.f;
-        uint32_t pk[32];
+        uint32_t pk[16];
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-            if (2 * j < n) {
+        for (int j = 0; j < 16; ++j) {
+            if (c0 + 2 * j < n) {
                 const float p0 = fast_exp2(fmaf(s[2 * j], kLog2e, nm));
                 const float p1 = fast_exp2(fmaf(s[2 * j + 1], kLog2e, nm));      // exp2(-inf) = 0 past the last agent
                 pk[j] = pack2<T>(p0, p1);
@@ -636,13 +636,14 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
                 pk[j] = 0u;
             }
         }
+        s_red[2 + half][row] = l;
 #pragma unroll
-        for (int c = 0; c < 8; ++c)
-            *reinterpret_cast<uint4*>(sPt + row * 128 + ((c ^ (row & 7)) << 4)) =
+        for (int c = 0; c < 4; ++c)
+            *reinterpret_cast<uint4*>(sPt + row * 128 + (((4 * half + c) ^ (row & 7)) << 4)) =
                 make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
         fence_proxy_async();              // the tensor core reads P through the async proxy
         tc_fence_before_sync();
-        sync_rows();
+        __syncthreads();
         if (tid == 0) {
             tc_fence_after_sync();
             const uint32_t idesc = umma_idesc(fmt, 128, 64, 1);       // V_A is [agents][d]: MN-major B operand
@@ -652,18 +653,17 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
         }
         wait_bar(bar_mma(st), (st.ph >> kBitMma) & 1u, p.status, kTimeoutLoads);
         st.ph ^= 1u << kBitMma;
-        sync_rows();
+        __syncthreads();
         tc_fence_after_sync();
-        const float inv = 1.f / l;
-        float* prow = sPatchAll + row * PO;
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
+        const float inv = 1.f / (s_red[2][row] + s_red[3][row]);
+        float* prow = sPatchAll + row * PO + c0;
+        {
             uint32_t r[32];
-            tmem_ld32(tO + lane_base + 32 * h, r);
+            tmem_ld32(tO + lane_base + c0, r);
             tmem_ld_wait();
 #pragma unroll
             for (int i = 0; i < 8; ++i)
-                *reinterpret_cast<float4*>(prow + 32 * h + 4 * i) =
+                *reinterpret_cast<float4*>(prow + 4 * i) =
                     make_float4(__uint_as_float(r[4 * i]) * inv, __uint_as_float(r[4 * i + 1]) * inv,
                                 __uint_as_float(r[4 * i + 2]) * inv, __uint_as_float(r[4 * i + 3]) * inv);
         }
@@ -751,6 +751,7 @@ __global__ void __launch_bounds__(NT, 2) fused_kernel(const __grid_constant__ Fu
     extern __shared__ unsigned char smem_raw[];
     __shared__ int s_task, s_flag, s_whead;
     __shared__ uint32_t s_tmem;
+    __shared__ float s_red[4][128];     // per query row: partial maxima and partial sums of the two column halves
     // TMA tiles with the 128-byte swizzle want a 1024-byte aligned base
     unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     const int tid = threadIdx.x;
@@ -763,7 +764,7 @@ __global__ void __launch_bounds__(NT, 2) fused_kernel(const __grid_constant__ Fu
         mbar_fence_init();
     }
     // tensor memory for the broadcast MMAs: warp 0 allocates (and frees at the end)
-    if (tid < 32) tmem_alloc(smem_u32(&s_tmem), kTmemCols);
+    if (tid < 32) tmem_alloc<kTmemCols>(smem_u32(&s_tmem));
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
@@ -796,7 +797,7 @@ __global__ void __launch_bounds__(NT, 2) fused_kernel(const __grid_constant__ Fu
             slab = S - Lg + step; sub = t - step * B; is_g = false;
         }
         if (is_g) run_g_task<T, SH>(p, slab, sub, smem, st, &s_flag, slot);
-        else      run_b_task<T, SH>(p, slab, sub, smem, st, &s_whead, slot);
+        else      run_b_task<T, SH>(p, slab, sub, smem, st, &s_whead, s_red, slot);
 #ifdef AA_FUSED_TRACE
         if (tid == 0 && g_trace && slot < 16) {
             g_trace[((size_t)blockIdx.x * 16 + slot) * 8 + 6] = is_g ? 1 : 2;
@@ -807,7 +808,7 @@ __global__ void __launch_bounds__(NT, 2) fused_kernel(const __grid_constant__ Fu
     }
     tc_fence_before_sync();
     __syncthreads();
-    if (tid < 32) tmem_dealloc(st.tmem, kTmemCols);
+    if (tid < 32) tmem_dealloc<kTmemCols>(st.tmem);
 }
 
 

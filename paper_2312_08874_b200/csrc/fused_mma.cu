@@ -3,6 +3,8 @@
 // shapes (App. G: 56x56 grid with 7x7 agents, 14x14 grid with 7x7 agents).
 #include "fused_kernel.cuh"
 
+#include <algorithm>
+#include <cstdio>
 #include <cstdlib>
 #include <cstring>
 
@@ -15,6 +17,9 @@ cudaError_t launch_fused_s56(int dtype, const FusedArgs& a, cudaStream_t st);
 cudaError_t launch_fused_s14(int dtype, const FusedArgs& a, cudaStream_t st);
 
 static int fused_spec_of(int H, int W, int n_agents) {
+#ifdef AA_FUSED_TRACE
+    return 0;                      // debug builds trace the generic kernel
+#endif
     if (H == 56 && W == 56 && n_agents == 49) return 1;
     if (H == 14 && W == 14 && n_agents == 49) return 2;
     return 0;
@@ -57,8 +62,32 @@ FusedPlan plan_fused(int dtype, int slabs, int H, int W, int d, int n_agents, in
     if (!fused_shape_plan(dtype, H, W, d, n_agents, &pl)) { pl.ok = false; return pl; }
     if (!encode_tiled_fn()) return pl;            // no tensor-map encoder: use the per-step kernels
     pl.spec = fused_spec_of(H, W, n_agents);
-    int occ = pl.spec == 1 ? fused_occupancy_s56(dtype) : pl.spec == 2 ? fused_occupancy_s14(dtype) : fused_occupancy_dt<ShapeAny>(dtype);
+    // (each query also raises that kernel's dynamic shared-memory limit; the generic kernel serves a
+    // specialised shape whenever a bias or the depthwise filter is absent)
+    int occ = fused_occupancy_dt<ShapeAny>(dtype);
+    if (pl.spec == 1) occ = std::min(occ, fused_occupancy_s56(dtype));
+    if (pl.spec == 2) occ = std::min(occ, fused_occupancy_s14(dtype));
     if (occ < 1) return pl;
+    // The occupancy query counts a block that allocates tensor memory as taking all of it.  Two blocks
+    // of 128 columns each fit the 512 columns of an SM, so where registers and shared memory allow a
+    // second block the grid is sized for two (the queue only needs g_tasks resident blocks to progress).
+    {
+        cudaFuncAttributes fa;
+        cudaDeviceProp prop;
+        int dev = 0;
+        const void* fn = dtype == kBF16 ? (const void*)fused_kernel<__nv_bfloat16, ShapeAny> : (const void*)fused_kernel<__half, ShapeAny>;
+        if (cudaGetDevice(&dev) == cudaSuccess && cudaGetDeviceProperties(&prop, dev) == cudaSuccess &&
+            cudaFuncGetAttributes(&fa, fn) == cudaSuccess) {
+            const size_t smem_block = (size_t)kSmemBytes + fa.sharedSizeBytes + 1024;
+            if (2 * smem_block <= prop.sharedMemPerMultiprocessor && 2 * fa.numRegs * NT <= prop.regsPerMultiprocessor &&
+                2 * kTmemCols <= 512)
+                occ = 2;
+        } else {
+            cudaGetLastError();
+        }
+    }
+    if (getenv("AGENT_ATTN_LOG"))
+        fprintf(stderr, "agent_attn: fused kernel spec=%d, %d blocks/SM, %d bytes of shared memory\n", pl.spec, occ, kSmemBytes);
     if (occ > 2) occ = 2;
     const long long total = (long long)slabs * (pl.g_tasks + pl.b_tasks);
     long long grid = (long long)occ * sm_count;
@@ -72,7 +101,6 @@ FusedPlan plan_fused(int dtype, int slabs, int H, int W, int d, int n_agents, in
     long long lag_l2 = (64LL << 20) / slab_qv_bytes;
     int lag = (5 * pl.grid / 2 + pl.g_tasks + pl.b_tasks - 1) / (pl.g_tasks + pl.b_tasks) + 2;
     if (lag_l2 > lag) lag = (int)(lag_l2 > 1000000 ? 1000000 : lag_l2);
-    if (const char* e = getenv("AA_FUSED_LAG")) lag = atoi(e);
     if (lag > slabs) lag = slabs;
     if (lag < 1) lag = 1;
     pl.lag = lag;
