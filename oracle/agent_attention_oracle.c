@@ -203,6 +203,49 @@ void aa_oracle_explicit(const double* Q, const double* A, const double* K, const
 }
 
 /* ---------------------------------------------------------------------------------
+ * Composition of an agent bias from its three components (App. B):
+ *   B = (B'_c + B'_r + B'_b).reshape(n, N),  N = h*w,
+ * with the column bias col [n][w] repeated over the h rows, the row bias row [n][h] repeated over
+ * the w columns, and the block bias blk [n][h0][w0] resized to h x w.  The paper says "repeating
+ * or interpolating"; the reading taken here resizes the block bias by bilinear interpolation with
+ * half-pixel centres and edge clamping (source coordinate max(0, (y + 0.5) * h0 / h - 0.5), and
+ * likewise in x), which is the identity when h0 = h and w0 = w.  Any component may be NULL (zero).
+ * transpose == 0 writes [n][N] (the layout of B1); transpose != 0 writes [N][n] (that of B2).
+ * ------------------------------------------------------------------------------- */
+void aa_oracle_compose_bias(const double* col, const double* row, const double* blk,
+                            int n, int h, int w, int h0, int w0, int transpose, double* out)
+{
+    const int N = h * w;
+    for (int a = 0; a < n; ++a)
+        for (int y = 0; y < h; ++y)
+            for (int x = 0; x < w; ++x) {
+                double v = 0.0;
+                if (col) v += col[(size_t)a * w + x];
+                if (row) v += row[(size_t)a * h + y];
+                if (blk) {
+                    double sy = ((double)y + 0.5) * (double)h0 / (double)h - 0.5;
+                    double sx = ((double)x + 0.5) * (double)w0 / (double)w - 0.5;
+                    if (sy < 0.0) sy = 0.0;
+                    if (sx < 0.0) sx = 0.0;
+                    int y0 = (int)floor(sy), x0 = (int)floor(sx);
+                    if (y0 > h0 - 1) y0 = h0 - 1;
+                    if (x0 > w0 - 1) x0 = w0 - 1;
+                    int y1 = y0 < h0 - 1 ? y0 + 1 : y0;
+                    int x1 = x0 < w0 - 1 ? x0 + 1 : x0;
+                    double ly = sy - (double)y0, lx = sx - (double)x0;
+                    if (ly > 1.0) ly = 1.0;
+                    if (lx > 1.0) lx = 1.0;
+                    const double* b = blk + (size_t)a * h0 * w0;
+                    v += (1.0 - ly) * ((1.0 - lx) * b[y0 * w0 + x0] + lx * b[y0 * w0 + x1])
+                       +        ly  * ((1.0 - lx) * b[y1 * w0 + x0] + lx * b[y1 * w0 + x1]);
+                }
+                const int t = y * w + x;
+                if (transpose) out[(size_t)t * n + a] = v;
+                else           out[(size_t)a * N + t] = v;
+            }
+}
+
+/* ---------------------------------------------------------------------------------
  * Module complexity, Eq. 7, in multiply-accumulates for N tokens, C channels (all heads),
  * n agents, DWC kernel size k:
  *   parts = { 4NC^2 (projections), NC (agents), 2nNC (aggregation: logits and weighted

@@ -51,6 +51,8 @@ def _load() -> ctypes.CDLL:
         lib.aa_oracle_explicit.restype = None
         lib.aa_oracle_macs.argtypes = [ctypes.c_longlong] * 4 + [ctypes.POINTER(ctypes.c_longlong)]
         lib.aa_oracle_macs.restype = ctypes.c_longlong
+        lib.aa_oracle_compose_bias.argtypes = [_DP] * 3 + [ctypes.c_int] * 6 + [_DP]
+        lib.aa_oracle_compose_bias.restype = None
         lib.aa_oracle_max_threads.argtypes = []
         lib.aa_oracle_max_threads.restype = ctypes.c_int
         _lib = lib
@@ -173,3 +175,20 @@ def macs(N: int, C: int, n: int, k: int = 3):
     parts = (ctypes.c_longlong * 5)()
     total = _load().aa_oracle_macs(N, C, n, k, parts)
     return int(total), [int(x) for x in parts]
+
+
+def compose_bias(col, row, blk, grid_h: int, grid_w: int, transpose: bool = False):
+    """App. B for one head: col [n, w], row [n, h], blk [n, h0, w0] (any may be None) -> [n, N] or [N, n]."""
+    parts = [x for x in (col, row, blk) if x is not None]
+    assert parts, "at least one component is needed"
+    n = parts[0].shape[0]
+    col = None if col is None else _c(col)
+    row = None if row is None else _c(row)
+    blk = None if blk is None else _c(blk)
+    assert col is None or col.shape == (n, grid_w)
+    assert row is None or row.shape == (n, grid_h)
+    h0, w0 = (blk.shape[1], blk.shape[2]) if blk is not None else (1, 1)
+    N = grid_h * grid_w
+    out = np.empty((N, n) if transpose else (n, N), dtype=np.float64)
+    _load().aa_oracle_compose_bias(_p(col), _p(row), _p(blk), n, grid_h, grid_w, h0, w0, int(bool(transpose)), _p(out))
+    return out

@@ -32,6 +32,9 @@ MUTANTS = [
     ("b2_head_offset_dropped", "b2 ? b2 + (size_t)head * N * n : NULL", "b2 ? b2 : NULL"),
     ("dwc_head_offset_dropped", "wd + (size_t)head * d * 9", "wd"),
     ("broadcast_uses_v_not_va", "aa_oracle_softmax_attention(q, a, va,", "aa_oracle_softmax_attention(q, a, v,"),
+    ("bias_block_align_corners", "double sy = ((double)y + 0.5) * (double)h0 / (double)h - 0.5;", "double sy = (double)y * (double)(h0 - 1) / (double)(h > 1 ? h - 1 : 1);"),
+    ("bias_row_col_swapped", "if (row) v += row[(size_t)a * h + y];", "if (row) v += row[(size_t)a * h + (x < h ? x : h - 1)];"),
+    ("bias_transpose_ignored", "if (transpose) out[(size_t)t * n + a] = v;", "if (0) out[(size_t)t * n + a] = v;"),
     ("eq7_aggregation_halved", "p[2] = 2 * n * N * C;", "p[2] = n * N * C;"),
 ]
 

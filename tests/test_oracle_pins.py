@@ -320,3 +320,38 @@ def test_threads_do_not_change_the_result():
     o1 = orc.forward(q, k, v, H, W, pool_hw=(p, p), threads=1)
     o4 = orc.forward(q, k, v, H, W, pool_hw=(p, p), threads=4)
     assert np.array_equal(o1, o4)
+
+
+# ----------------------------------------------------------------- App. B: bias composition
+@pytest.mark.parametrize("h,w,h0,w0", [(14, 14, 7, 7), (8, 12, 3, 5), (9, 7, 9, 7), (16, 16, 1, 1), (5, 6, 2, 9)])
+def test_bias_composition_equals_broadcast_plus_library_bilinear_resize(h, w, h0, w0):
+    n = 5
+    r = _rng(30 + h + w0)
+    col, row, blk = r.standard_normal((n, w)), r.standard_normal((n, h)), r.standard_normal((n, h0, w0))
+    got = orc.compose_bias(col, row, blk, h, w)
+    resized = F.interpolate(torch.from_numpy(blk)[None], size=(h, w), mode="bilinear", align_corners=False)[0].numpy()
+    ref = (col[:, None, :] + row[:, :, None] + resized).reshape(n, h * w)
+    np.testing.assert_allclose(got, ref, atol=1e-12)
+    np.testing.assert_allclose(orc.compose_bias(col, row, blk, h, w, transpose=True), ref.T, atol=1e-12)
+
+
+def test_bias_composition_closed_forms():
+    n, h, w = 3, 6, 4
+    r = _rng(31)
+    col, row = r.standard_normal((n, w)), r.standard_normal((n, h))
+    full = r.standard_normal((n, h, w))
+    np.testing.assert_allclose(orc.compose_bias(None, None, full, h, w), full.reshape(n, h * w), atol=1e-14)   # h0 = h: identity
+    const = np.tile(np.array([1.5, -2.0, 0.25])[:, None, None], (1, 2, 3))
+    np.testing.assert_allclose(orc.compose_bias(None, None, const, h, w), np.repeat(const[:, 0, 0], h * w).reshape(n, -1), atol=1e-14)
+    only_col = orc.compose_bias(col, None, None, h, w).reshape(n, h, w)
+    for y in range(h):
+        np.testing.assert_allclose(only_col[:, y, :], col, atol=0)
+    only_row = orc.compose_bias(None, row, None, h, w).reshape(n, h, w)
+    for x in range(w):
+        np.testing.assert_allclose(only_row[:, :, x], row, atol=0)
+    # the module with a composed bias equals the module with the dense bias (the operator takes dense biases)
+    q, k, v = _slab(32, h, w, 4)
+    blk = r.standard_normal((4, 2, 2))
+    b1 = orc.compose_bias(r.standard_normal((4, w)), r.standard_normal((4, h)), blk, h, w)
+    o = orc.forward(q[None, None], k[None, None], v[None, None], h, w, pool_hw=(2, 2), b1=b1[None])
+    assert np.all(np.isfinite(o))
