@@ -137,6 +137,18 @@ int agent_attn_broadcast(agent_attn_handle* h, const void* Q, const void* A, con
                          const void* V, const void* b2, const void* dwc_weight,
                          int grid_h, int grid_w, int n_agents, void* out, void* stream);
 
+/* Dense agent bias from its three components (App. B): out = (B'_c + B'_r + B'_b).reshape(n, N).
+ *   col   device [heads][n][grid_w]            column bias, repeated over the grid rows, or NULL
+ *   row   device [heads][n][grid_h]            row bias, repeated over the grid columns, or NULL
+ *   blk   device [heads][n][block_h][block_w]  block bias, resized to grid_h x grid_w by bilinear
+ *         interpolation with half-pixel centres and edge clamping (the paper says "repeating or
+ *         interpolating"; this is the reading taken), or NULL
+ *   transpose == 0: out device [heads][n][N] (the layout of b1);  != 0: [heads][N][n] (that of b2)
+ * At least one component must be given.  The result is what agent_attn_forward takes as a bias. */
+int agent_attn_compose_bias(agent_attn_handle* h, const void* col, const void* row, const void* blk,
+                            int block_h, int block_w, int grid_h, int grid_w, int n_agents,
+                            int transpose, void* out, void* stream);
+
 /* Bytes of device staging memory that agent_attn_forward_host needs (room for Q, K, V, A, B1,
  * B2, Wd, out and the workspace, each 256-byte aligned).  0 on invalid arguments. */
 size_t agent_attn_staging_bytes(const agent_attn_handle* h, int grid_h, int grid_w, int n_agents);

@@ -25,6 +25,7 @@ EXPORTS = [
     "agent_attn_forward", "agent_attn_pool", "agent_attn_aggregate", "agent_attn_broadcast",
     "agent_attn_staging_bytes", "agent_attn_forward_host", "agent_attn_query_status",
     "agent_attn_last_launch_count", "agent_attn_aggregate_static", "agent_attn_static_scratch_bytes",
+    "agent_attn_compose_bias",
 ]
 
 
@@ -91,6 +92,8 @@ def load_library(build_if_missing: bool = True) -> ctypes.CDLL:
     lib.agent_attn_last_launch_count.restype = ci
     lib.agent_attn_aggregate_static.argtypes = [vp, vp, vp, vp, vp, ci, ci, vp, vp]
     lib.agent_attn_aggregate_static.restype = ci
+    lib.agent_attn_compose_bias.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, vp, vp]
+    lib.agent_attn_compose_bias.restype = ci
     lib.agent_attn_static_scratch_bytes.argtypes = []
     lib.agent_attn_static_scratch_bytes.restype = sz
     _lib = lib
@@ -244,6 +247,23 @@ class AgentAttention:
         self._check(self.lib.agent_attn_broadcast(self._h, _ptr(q), _ptr(agents), _ptr(va), _ptr(v), _ptr(b2),
                                                   _ptr(dwc_weight), grid_h, grid_w, n, _ptr(out),
                                                   _stream_ptr(stream)))
+        return out
+
+    def compose_bias(self, col, row, blk, grid_h: int, grid_w: int, n_agents: int, transpose: bool = False,
+                     out=None, stream=None):
+        """`agent_attn_compose_bias`: dense B1 ([heads, n, N]) or B2 ([heads, N, n], transpose=True)
+        from column [heads, n, w], row [heads, n, h] and block [heads, n, h0, w0] components (App. B)."""
+        h, N = self.heads, grid_h * grid_w
+        self._chk_tensor(col, (h, n_agents, grid_w), "col")
+        self._chk_tensor(row, (h, n_agents, grid_h), "row")
+        h0, w0 = (blk.shape[2], blk.shape[3]) if blk is not None else (1, 1)
+        self._chk_tensor(blk, (h, n_agents, h0, w0), "blk")
+        shape = (h, N, n_agents) if transpose else (h, n_agents, N)
+        if out is None:
+            out = torch.empty(shape, dtype=self.dtype, device=self.device)
+        self._chk_tensor(out, shape, "out")
+        self._check(self.lib.agent_attn_compose_bias(self._h, _ptr(col), _ptr(row), _ptr(blk), h0, w0, grid_h, grid_w,
+                                                     n_agents, int(transpose), _ptr(out), _stream_ptr(stream)))
         return out
 
     def forward_host(self, q, k, v, grid_h: int, grid_w: int, n_agents: int, agents=None, b1=None, b2=None,

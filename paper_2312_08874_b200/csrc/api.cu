@@ -338,6 +338,29 @@ int agent_attn_forward(agent_attn_handle* h, const void* Q, const void* K, const
     return do_broadcast(h, Q, agents, va, V, b2, dwc_weight, grid_h, grid_w, n_agents, out, st);
 }
 
+int agent_attn_compose_bias(agent_attn_handle* h, const void* col, const void* row, const void* blk, int block_h,
+                            int block_w, int grid_h, int grid_w, int n_agents, int transpose, void* out,
+                            void* stream) {
+    if (!h) return AA_ERR_INVALID_ARG;
+    h->err[0] = 0;
+    if (!out || (!col && !row && !blk)) return fail(h, AA_ERR_INVALID_ARG, "null pointer");
+    if (grid_h <= 0 || grid_w <= 0) return fail(h, AA_ERR_INVALID_ARG, "grid must be positive");
+    if (blk && (block_h <= 0 || block_w <= 0)) return fail(h, AA_ERR_INVALID_ARG, "block bias needs a positive size");
+    if (int rc = check_shape(h, grid_h * grid_w, n_agents)) return rc;
+    if (misaligned(out) || (col && misaligned(col)) || (row && misaligned(row)) || (blk && misaligned(blk)))
+        return fail(h, AA_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
+    DeviceGuard guard(h->cfg.device);
+    if (!guard.ok) return fail(h, AA_ERR_CUDA, "cannot select device %d", h->cfg.device);
+    ComposeArgs a;
+    a.col = col; a.row = row; a.blk = blk; a.out = out;
+    a.heads = h->cfg.heads; a.n = n_agents; a.h = grid_h; a.w = grid_w;
+    a.h0 = blk ? block_h : 1; a.w0 = blk ? block_w : 1; a.transpose = transpose ? 1 : 0;
+    cudaError_t e = launch_compose_bias(h->cfg.dtype, a, (cudaStream_t)stream);
+    if (e != cudaSuccess) return fail(h, AA_ERR_CUDA, "bias composition launch failed: %s", cudaGetErrorString(e));
+    h->launches = 1;
+    return AA_OK;
+}
+
 size_t agent_attn_staging_bytes(const agent_attn_handle* h, int grid_h, int grid_w, int n_agents) {
     const size_t ws = agent_attn_workspace_bytes(h, grid_h, grid_w, n_agents);
     if (!ws) return 0;

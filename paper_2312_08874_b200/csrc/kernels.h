@@ -25,6 +25,15 @@ struct PoolArgs {
 };
 cudaError_t launch_pool(int dtype, const PoolArgs& p, cudaStream_t st);
 
+// Dense agent bias from column [heads][n][w], row [heads][n][h] and block [heads][n][h0][w0]
+// components (any may be null); out is [heads][n][N] or, transposed, [heads][N][n].
+struct ComposeArgs {
+    const void *col, *row, *blk;
+    void* out;
+    int heads, n, h, w, h0, w0, transpose;
+};
+cudaError_t launch_compose_bias(int dtype, const ComposeArgs& p, cudaStream_t st);
+
 // One softmax attention with an additive bias, out = softmax(scale * Qm Km^T + bias) Vm.
 // Aggregation: rows = agents, cols = tokens (split over blocks, merged by the last block).
 // Broadcast:   rows = tokens, cols = agents, plus the depthwise 3x3 term on `dwc_v`.

@@ -194,6 +194,28 @@ def test_forward_host_matches_forward():
     assert mod.query_status() == 0
 
 
+# ------------------------------------------------------------------ App. B: bias composition
+@pytest.mark.parametrize("dtype", ["f32", "bf16", "f16"])
+@pytest.mark.parametrize("transpose", [False, True])
+def test_bias_composition_matches_oracle(dtype, transpose):
+    from paper_2312_08874_b200.workloads import TORCH_DTYPE
+    heads, n, H, W, h0, w0 = 3, 49, 14, 20, 5, 7
+    g = torch.Generator().manual_seed(40)
+    dt = TORCH_DTYPE[dtype]
+    col = torch.randn((heads, n, W), generator=g).to(dt)
+    row = torch.randn((heads, n, H), generator=g).to(dt)
+    blk = torch.randn((heads, n, h0, w0), generator=g).to(dt)
+    mod = AgentAttention(1, heads, 64, H * W, n, dt)
+    got = mod.compose_bias(col.cuda(), row.cuda(), blk.cuda(), H, W, n, transpose=transpose)
+    torch.cuda.synchronize()
+    ref = np.stack([orc.compose_bias(to_np(col[h]), to_np(row[h]), to_np(blk[h]), H, W, transpose=transpose)
+                    for h in range(heads)])
+    assert_close(got, ref, dtype, "composed bias", scale=1.0 if dtype != "f32" else 1.0)
+    only_blk = mod.compose_bias(None, None, blk.cuda(), H, W, n, transpose=transpose)
+    ref_blk = np.stack([orc.compose_bias(None, None, to_np(blk[h]), H, W, transpose=transpose) for h in range(heads)])
+    assert_close(only_blk, ref_blk, dtype, "block bias alone")
+
+
 # --------------------------------------------------------------------------------- error paths
 def test_invalid_arguments_are_rejected_without_launching():
     from paper_2312_08874_b200 import AgentAttnError
