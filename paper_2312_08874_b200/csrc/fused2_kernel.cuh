@@ -1,30 +1,33 @@
 // The whole module of Eq. 6 in one persistent, role-specialised kernel for small agent counts
-// (n <= 64, d = 64, 16-bit elements): one block per SM, nine warps.
+// (n <= 64, d = 64, 16-bit elements): one block of sixteen warps per SM.
 //
-//   warps 0-3  "row group":   own the 128 lanes of tensor memory.  Aggregation: one thread per agent
-//                             row does the online softmax on logits that tcgen05.mma left in tensor
-//                             memory.  Broadcast: one thread per query row does the softmax over the
-//                             agents and hands the normalised row to the stencil group.
-//   warps 4-7  "stencil group": depthwise 3x3 term (Eq. 6) and the store of O, one tile behind the
-//                             row group; pooling (together with the row group).
-//   warp 8     "producer":    one lane issues every TMA / bulk copy, running ahead of the others
-//                             through full/empty mbarriers.
+//   warps 0-7   "row warps":     own the 128 lanes of tensor memory, two threads per lane (each 32 of
+//                                the 64 logit columns).  Aggregation: online softmax per agent row on
+//                                logits that tcgen05.mma left in tensor memory.  Broadcast: softmax over
+//                                the agents per query row; the normalised row goes to the stencil warps.
+//   warps 8-13  "stencil warps": depthwise 3x3 term (Eq. 6) and the store of O, one tile behind the row
+//                                warps; they also pool and merge together with the row warps.
+//   warp 14     "producer":      one lane issues every TMA / bulk copy, ahead of the others through
+//                                full/empty mbarriers.
+//   warp 15     "MMA issuer":    one lane issues every tcgen05.mma and its commits.
 //
-// Blocks take tasks from a device-side queue (same order and progress argument as the first fused
-// kernel: a task waits only for earlier tasks or for its slab's G siblings, which are adjacent in the
-// queue, and the grid holds at least as many blocks as a slab has G tasks).
-//
-//   G task (slab, range of grid rows): pool Q over the range (complete agent rows), publish, wait for
-//     the siblings, then stream K, V and B1 tiles of 64 tokens through a six-slot TMA ring.  A step
-//     takes two tiles: rows 0-63 of the 128-row MMA work on the first, rows 64-127 on the second
-//     (the agent operand is stacked twice), so all 128 lanes carry useful rows with n <= 64.
-//     Logits: S = (scale1 A) K^T + I B1, i.e. the bias enters through a second K-block whose A operand
-//     is an identity matrix (Eq. 5 inside the contraction).  V_A partial = P V with P written back to
-//     shared memory as the A operand (Eq. 3).  Partial states are merged as in the first kernel.
-//   B task (slab, run of broadcast tiles): per tile of whole grid rows (<= 128 tokens) S = Q A^T by
+// Blocks take tasks from a device-side queue.  Four kinds, ordered so that a task only ever waits for
+// tasks of an EARLIER stage of the queue (no circular waits, any grid size makes progress):
+//   P (slab, range of grid rows): pool Q over the range (complete agent rows; text under Eq. 6).
+//   G (slab, range): stream K, V and B1 tiles of 64 tokens through a six-slot TMA ring.  A step takes
+//     two tiles: rows 0-63 of the 128-row MMA work on the first, rows 64-127 on the second (the agent
+//     operand is stacked twice), and each row is shared by two threads that own 32 tokens each with
+//     their own running maximum and their own accumulator, so no reduction crosses threads.
+//     Logits: S = (scale1 A) K^T + I B1: the bias enters through a second K-block whose A operand is an
+//     identity matrix (Eq. 5 inside the contraction).  V_A partial = P V with P written back to shared
+//     memory as the A operand (Eq. 3).  The range's partial state goes to the workspace.
+//   M (slab): merge the slab's partial states into V_A (fixed order: bit-reproducible).
+//   B (slab, run of broadcast tiles): per tile of whole grid rows (<= 128 tokens) S = Q A^T by
 //     tcgen05.mma, softmax with B2 per query row (Eq. 5), O = P V_A, then the depthwise term on the V
-//     rows that a ring of row slots keeps in shared memory.  The three roles are pipelined over the
-//     run's tiles: loads two tiles ahead, softmax one tile ahead of the stencil.
+//     rows that a ring of row slots keeps in shared memory.  Loads run two tiles ahead, the softmax one
+//     tile ahead of the stencil.
+// Stages interleave groups of slabs (P of group g+3, G of g+2, M of g+1, B of g) sized so that the Q and
+// V of the groups in flight stay in L2.
 //
 // Every wait is bounded (mbarrier waits and flag polls give up, set the status word and a block-wide
 // flag that makes every later wait return at once), so a logic error ends as a status code, not as a
@@ -43,8 +46,11 @@ constexpr int DK = 64;            // head dim
 constexpr int KT = 64;            // tokens per aggregation tile
 constexpr int QT = 128;           // most tokens per broadcast tile
 constexpr int RP = 64;            // agent rows, padded
-constexpr int NCOMP = 256;        // compute threads (row group + stencil group)
-constexpr int NT = NCOMP + 32;    // + producer warp
+constexpr int NR = 256;           // row warps 0-7
+constexpr int NX = 192;           // stencil warps 8-13
+constexpr int NCOMP = NR + NX;    // compute threads
+constexpr int NT = NCOMP + 64;    // + producer warp + MMA issuer warp: 512 threads, 128 registers each
+constexpr int kWarpProd = 14, kWarpMma = 15;
 constexpr int RING = 6;           // aggregation ring slots (one tile each)
 constexpr int MAXW = 64, MINW = 8;
 constexpr int kVTokens = 400;     // V row slots: (2R + 2)(W + 2) tokens at most
@@ -56,8 +62,8 @@ constexpr float kTau = 5.5f;      // a row's reference maximum moves only when e
 // ------------------------------------------------------------------ shared-memory map (bytes)
 constexpr int kTile = KT * 128;                       // swizzled [64][64] tile of 16-bit elements
 constexpr int OFF_W = 0;                              // filter taps [9][64] fp32
-constexpr int OFF_BAR = 2304;                         // mbarriers
-constexpr int kNumBars = 32;
+constexpr int OFF_BAR = 2304;                         // mbarriers (8 bytes each)
+constexpr int kNumBars = 40;
 constexpr int OFF_UNION = 3072;
 // aggregation
 constexpr int G_ASTACK = OFF_UNION;                   // [128][128 B]: scaled agents, twice
@@ -84,24 +90,32 @@ static_assert(OFF_UNION % 1024 == 0 && kTile % 1024 == 0 && B_V % 128 == 0 && B_
 static_assert(kSmemBytes <= 232448, "shared memory per block");
 static_assert(kSmemBytes > 116 * 1024, "one block per SM: each block takes all 512 tensor-memory columns");
 
-// mbarrier indices
-constexpr int BAR_FULL = 0;          // [RING]  tile landed                     (tx)      waiter: row-group leader
-constexpr int BAR_EMPTY = 6;         // [RING]  tile consumed                   (commit)  waiter: producer
-constexpr int BAR_S = 12;            // [2]     logits ready                    (commit)  waiter: row group
-constexpr int BAR_PV = 14;           //         P V product done                (commit)  waiter: row group
-constexpr int BAR_AG = 15;           //         agents (and features) landed    (tx)      waiter: row group
-constexpr int BAR_IN_FULL = 16;      // [2]     Q and B2 tile landed            (tx)      waiter: row-group leader
-constexpr int BAR_IN_EMPTY = 18;     // [2]     Q and B2 tile consumed          (128)     waiter: producer
-constexpr int BAR_PATCH_FULL = 20;   // [2]     normalised rows written         (128)     waiter: stencil group
-constexpr int BAR_PATCH_EMPTY = 22;  // [2]     patch consumed                  (128)     waiter: row group
-constexpr int BAR_V_FULL = 24;       // [2]     V rows of a tile landed         (tx)      waiter: stencil group
-constexpr int BAR_V_EMPTY = 26;      // [2]     V rows of a tile consumed       (128)     waiter: producer
-constexpr int kBarsUsed = 28;
+// mbarrier indices                   count     waiter
+constexpr int BAR_FULL = 0;          // [RING]  tx        MMA issuer      tile landed
+constexpr int BAR_EMPTY = 6;         // [RING]  commit    producer        tile consumed
+constexpr int BAR_S_FULL = 12;       // [2]     commit    row warps       logits ready
+constexpr int BAR_S_EMPTY = 14;      // [2]     256       MMA issuer      logits read
+constexpr int BAR_PG_FULL = 16;      //         256       MMA issuer      aggregation: P of the step written
+constexpr int BAR_PB_FULL = 17;      //         1         MMA issuer      broadcast: P of the tile written
+constexpr int BAR_PV = 18;           //         commit    row warps       P V product done
+constexpr int BAR_AG = 19;           //         tx        MMA issuer      agents (and features) landed
+constexpr int BAR_PREP = 20;         //         1         MMA issuer      identity / plain-load bias tiles written
+constexpr int BAR_IN_FULL = 21;      // [2]     tx        MMA issuer      Q and B2 tile landed
+constexpr int BAR_IN_EMPTY = 23;     // [2]     256       producer        Q and B2 tile consumed
+constexpr int BAR_PATCH_FULL = 25;   // [2]     256       stencil warps   normalised rows written
+constexpr int BAR_PATCH_EMPTY = 27;  // [2]     256       row warps       patch consumed
+constexpr int BAR_V_FULL = 29;       // [2]     tx        stencil warps   V rows of a tile landed
+constexpr int BAR_V_EMPTY = 31;      // [2]     256       producer        V rows of a tile consumed
+constexpr int kBarsUsed = 33;
 static_assert(kBarsUsed <= kNumBars, "barriers");
+__host__ __device__ constexpr uint32_t bar_count(int i) {
+    return ((i >= BAR_S_EMPTY && i <= BAR_PG_FULL) || (i >= BAR_IN_EMPTY && i < BAR_PATCH_EMPTY)) ? (uint32_t)NR
+           : ((i >= BAR_PATCH_EMPTY && i < BAR_V_FULL) || i >= BAR_V_EMPTY) ? (uint32_t)NX : 1u;
+}
 
 // tensor-memory columns (512 allocated)
 constexpr uint32_t TM_GS = 0;        // aggregation logits: 2 buffers x 128 columns (two tiles per step)
-constexpr uint32_t TM_GO = 256;      // aggregation accumulators: rows 0-63 use columns [256, 320), rows 64-127 [320, 384)
+constexpr uint32_t TM_GO = 256;      // aggregation accumulators: 4 x 64 columns, index 2 * (stack half) + (token half)
 constexpr uint32_t TM_BS = 0;        // broadcast logits: 2 x 64
 constexpr uint32_t TM_BO = 128;      // broadcast outputs: 2 x 64
 
@@ -109,7 +123,7 @@ struct Role {
     int* status;          // device status word
     int* dead;            // shared flag: some wait of this block gave up
     uint32_t bars;        // shared address of mbarrier 0
-    uint32_t ph;          // parity to wait for next, one bit per mbarrier (each role tracks the ones it waits on)
+    uint64_t ph;          // parity to wait for next, one bit per mbarrier (each role tracks the ones it waits on)
     uint32_t tmem;
 };
 __device__ __forceinline__ uint32_t bar_addr(const Role& ro, int i) { return ro.bars + 8u * (uint32_t)i; }
@@ -121,19 +135,29 @@ __device__ __forceinline__ unsigned ld_acquire(const unsigned* p) {
 }
 __device__ __forceinline__ int ld_shared_volatile(const int* p) { return *reinterpret_cast<const volatile int*>(p); }
 
-// Bounded wait for the next phase of mbarrier i (this role's parity bit flips either way).
-__device__ __forceinline__ void wait_bar(Role& ro, int i, int code) {
-    const uint32_t parity = (ro.ph >> i) & 1u;
-    ro.ph ^= 1u << i;
+// Bounded wait of ONE thread for the next phase of mbarrier i (this thread's parity bit flips either way).
+__device__ __forceinline__ void wait_bar_one(Role& ro, int i, int code) {
+    const uint32_t parity = (uint32_t)(ro.ph >> i) & 1u;
+    ro.ph ^= 1ull << i;
     if (ld_shared_volatile(ro.dead)) return;
     const uint32_t bar = bar_addr(ro, i);
     for (unsigned tries = 0; tries < kBarLimit; ++tries) {
         if (mbar_try_wait(bar, parity)) return;
-        if (tries > 16) __nanosleep(20);
+        if (tries > 4) __nanosleep(32);
         if ((tries & 255u) == 255u && ld_shared_volatile(ro.dead)) return;
     }
     *reinterpret_cast<volatile int*>(ro.dead) = 1;
     atomicCAS(ro.status, 0, code);
+}
+// The same for a whole (converged) warp: lane 0 polls, so that waiting warps leave the shared-memory
+// pipeline to the working ones; the warp barrier passes the acquired data on to the other lanes.
+__device__ __forceinline__ void wait_bar(Role& ro, int i, int code) {
+    if ((threadIdx.x & 31) == 0) {
+        wait_bar_one(ro, i, code);
+    } else {
+        ro.ph ^= 1ull << i;
+    }
+    __syncwarp();
 }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(bar) : "memory");
@@ -161,9 +185,9 @@ __device__ __forceinline__ void publish_add(unsigned* ctr) {
     __syncthreads();
     if (threadIdx.x == 0) { __threadfence(); atomicAdd(ctr, 1u); }
 }
-__device__ __forceinline__ void sync_rows() { asm volatile("bar.sync 1, 128;\n" ::: "memory"); }      // warps 0-3
-__device__ __forceinline__ void sync_stencil() { asm volatile("bar.sync 2, 128;\n" ::: "memory"); }   // warps 4-7
-__device__ __forceinline__ void sync_compute() { asm volatile("bar.sync 3, 256;\n" ::: "memory"); }   // warps 0-7
+__device__ __forceinline__ void sync_rows() { asm volatile("bar.sync 1, 256;\n" ::: "memory"); }      // warps 0-7
+__device__ __forceinline__ void sync_stencil() { asm volatile("bar.sync 2, %0;\n" ::"n"(NX) : "memory"); }     // warps 8-13
+__device__ __forceinline__ void sync_compute() { asm volatile("bar.sync 3, %0;\n" ::"n"(NCOMP) : "memory"); }  // warps 0-13
 
 __device__ __forceinline__ int swz(int row, int col) {
     return row * 128 + ((((col >> 3) ^ row) & 7) << 4) + (col & 7) * 2;
@@ -188,94 +212,62 @@ template <int H_, int W_, int P_> struct Shape {
 };
 using ShapeAny = Shape<0, 0, 0>;
 
-// ---------------------------------------------------------------------------------- G task
+// Optional per-task timestamps (debug builds only): define AA_FUSED2_TRACE and hand a device buffer to
+// aa_fused2_trace_buffer; record (block, task slot < 32) holds eight values: entries 0-5 are globaltimer
+// marks of thread 0, entry 6 the task kind + 1, entry 7 the task index.
+#ifdef AA_FUSED2_TRACE
+__device__ unsigned long long* g_trace2 = nullptr;
+__device__ __forceinline__ void trace_put(int slot, int entry, unsigned long long v) {
+    if (g_trace2 && slot < 32) g_trace2[((size_t)blockIdx.x * 32 + slot) * 8 + entry] = v;
+}
+__device__ __forceinline__ void trace_mark(int slot, int entry) {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    trace_put(slot, entry, t);
+}
+#define TR(entry) if (threadIdx.x == 0) trace_mark(slot, entry)
+#else
+#define TR(entry)
+#endif
+
+// ---------------------------------------------------------------------------------- P task
+// Pool Q over a range of grid rows that covers whole pooling windows: complete rows of A.  Each window
+// is split over `nsplit` warps (by token index inside the window); the parts meet in shared memory.
 template <typename T, typename SH>
-__device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub, unsigned char* smem, Role& ro) {
-    constexpr int cpr = DK / 8;
-    constexpr int fmt = Elem<T>::kIsBf16 ? 1 : 0;
+__device__ __forceinline__ void run_p_task(const FusedArgs& p, int slab, int sub, unsigned char* smem, int slot) {
+    constexpr int cpr = DK / 8;               // 16-byte chunks per token row
+    constexpr int tpl = 32 / cpr;             // tokens per warp-wide load
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const bool is_prod = warp == 8, is_rows = warp < 4;
-    const int head = slab % p.heads;
     const int H = SH::kFixed ? SH::kH : p.H, W = SH::kFixed ? SH::kW : p.W, P = SH::kFixed ? SH::kP : p.p;
     const int N = H * W, n = SH::kFixed ? SH::kP * SH::kP : p.n;
     const int win_h = H / P, win_w = W / P;
     const int gr0 = sub * p.plan.rows_per_g, gr1 = min(H, gr0 + p.plan.rows_per_g);
-    const int t_begin = gr0 * W, t_end = gr1 * W;
-    const int tiles = (t_end - t_begin + KT - 1) / KT;
-    const int steps = (tiles + 1) >> 1;
-    const bool has_bias = SH::kFixed ? true : (p.b1 != nullptr);
-    const bool bias_tma = has_bias && p.b1_tma;
-
-    const uint32_t ring_u32 = smem_u32(smem + G_RING);
-    const uint32_t astack = smem_u32(smem + G_ASTACK), ident = smem_u32(smem + G_IDENT), sP = smem_u32(smem + G_P);
+    const int ar0 = gr0 / win_h, ar1 = gr1 / win_h;
+    const int nwin = (ar1 - ar0) * P;
+    const int cnt = win_h * win_w;
+    int nsplit = (NCOMP / 32) / nwin;
+    if (nsplit < 1) nsplit = 1;
+    if (nsplit > 8) nsplit = 8;
+    while (nsplit > 1 && tpl * nsplit > cnt) --nsplit;        // at least one load per part
     const T* gQ = static_cast<const T*>(p.q) + (size_t)slab * N * DK;
-    const T* gB = has_bias ? static_cast<const T*>(p.b1) + (size_t)head * n * N : nullptr;
     T* gAg = static_cast<T*>(p.ag_ws) + (size_t)slab * RP * DK;     // scale1 * A, rows >= n zero
     T* gAb = static_cast<T*>(p.ab_ws) + (size_t)slab * RP * DK;     // A, rows >= n zero
-    const uint32_t tile_tx = 2 * kTile + (bias_tma ? kTile : 0);
-
-    auto fill = [&](int t) {              // producer lane: tile t of the range -> its ring slot
-        const int s = t % RING, c0 = t_begin + t * KT;
-        const uint32_t bar = bar_addr(ro, BAR_FULL + s), dst = ring_u32 + s * kSlot;
-        mbar_arrive_expect_tx(bar, tile_tx);
-        tma_load_2d(dst, &p.tm_k, 0, slab * N + c0, bar);
-        tma_load_2d(dst + kTile, &p.tm_v, 0, slab * N + c0, bar);
-        if (bias_tma) tma_load_2d(dst + 2 * kTile, &p.tm_b1, c0, head * n, bar);
-    };
-
-    // ---- phase 0: first ring fills; pooling; identity operand; B1 tiles by plain loads if TMA cannot
-    if (is_prod) {
-        if (lane == 0)
-            for (int t = 0; t < tiles && t < RING; ++t) fill(t);
-        __syncwarp();
-    } else {
-        if (has_bias) {
-            // identity, stacked twice: row r has a one at k = r % 64 (the A operand of the bias K-block)
-            const unsigned short one = Elem<T>::kIsBf16 ? 0x3F80u : 0x3C00u;
-            for (int idx = tid; idx < 128 * 8; idx += NCOMP) {
-                const int row = idx >> 3, c = idx & 7;
-                const int lc = c ^ (row & 7);                 // logical 16-byte chunk: k = 8 lc .. 8 lc + 7
-                uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                const int k = row & 63;
-                if ((k >> 3) == lc) {
-                    const uint32_t w = (uint32_t)one << (16 * (k & 1));
-                    const int wi = (k & 7) >> 1;
-                    if (wi == 0) v.x = w; else if (wi == 1) v.y = w; else if (wi == 2) v.z = w; else v.w = w;
-                }
-                *reinterpret_cast<uint4*>(smem + G_IDENT + row * 128 + c * 16) = v;
-            }
-            if (!bias_tma) {                 // the plan guarantees tiles <= RING here
-                for (int t = 0; t < tiles; ++t) {
-                    unsigned char* sB = smem + G_RING + (t % RING) * kSlot + 2 * kTile;
-                    const int c0 = t_begin + t * KT;
-                    for (int e = tid; e < RP * KT; e += NCOMP) {
-                        const int rr = e / KT, j = e - rr * KT;
-                        const int key = c0 + j;
-                        *reinterpret_cast<T*>(sB + swz(rr, j)) =
-                            (rr < n && key < t_end) ? gB[(size_t)rr * N + key] : Elem<T>::from_f32(0.f);
-                    }
-                }
-            }
-            fence_proxy_async();             // the tensor core reads these through the async proxy
-        }
-        // pool this range of Q: whole windows, i.e. complete rows of A (text under Eq. 6)
-        const int ar0 = gr0 / win_h, ar1 = gr1 / win_h;
-        const int nwin = (ar1 - ar0) * P;
-        const int cnt = win_h * win_w;
-        constexpr int tpl = 32 / cpr;
+    float* sPart = reinterpret_cast<float*>(smem + OFF_UNION);      // [window][part][64]
+    TR(0);
+    if (warp < NCOMP / 32) {
         const int cg = lane % cpr, tsub = lane / cpr;
-        const float inv = 1.f / (float)cnt;
-        for (int wi = warp; wi < nwin; wi += NCOMP / 32) {
+        for (int item = warp; item < nwin * nsplit; item += NCOMP / 32) {
+            const int wi = item / nsplit, part = item - wi * nsplit;
             const int ay = ar0 + wi / P, ax = wi % P;
             const int y0 = ay * win_h, x0 = ax * win_w;
             float acc[8];
 #pragma unroll
             for (int k = 0; k < 8; ++k) acc[k] = 0.f;
-            for (int ib = tsub; ib < cnt; ib += 16 * tpl) {    // sixteen loads in flight per lane
-                uint4 raw[16];
+            for (int ib = tsub + part * tpl; ib < cnt; ib += 8 * tpl * nsplit) {    // eight loads in flight per lane
+                uint4 raw[8];
 #pragma unroll
-                for (int u = 0; u < 16; ++u) {
-                    const int i = ib + u * tpl;
+                for (int u = 0; u < 8; ++u) {
+                    const int i = ib + u * tpl * nsplit;
                     raw[u] = make_uint4(0u, 0u, 0u, 0u);
                     if (i < cnt) {
                         const int wy = i / win_w, wx = i - wy * win_w;
@@ -284,7 +276,7 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
                     }
                 }
 #pragma unroll
-                for (int u = 0; u < 16; ++u) {
+                for (int u = 0; u < 8; ++u) {
                     float f[8];
                     unpack16<T>(raw[u], f);
 #pragma unroll
@@ -297,12 +289,28 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
                 for (int k = 0; k < 8; ++k) acc[k] += __shfl_xor_sync(0xffffffffu, acc[k], o);
             }
             if (tsub == 0) {
-                float sc[8];
-#pragma unroll
-                for (int k = 0; k < 8; ++k) { acc[k] *= inv; sc[k] = acc[k] * p.scale1; }
-                *(reinterpret_cast<uint4*>(gAb + (size_t)(ay * P + ax) * DK) + cg) = pack16<T>(acc);
-                *(reinterpret_cast<uint4*>(gAg + (size_t)(ay * P + ax) * DK) + cg) = pack16<T>(sc);
+                float* d = sPart + ((size_t)wi * nsplit + part) * DK + cg * 8;
+                *reinterpret_cast<float4*>(d) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+                *reinterpret_cast<float4*>(d + 4) = make_float4(acc[4], acc[5], acc[6], acc[7]);
             }
+        }
+        sync_compute();
+        const float inv = 1.f / (float)cnt;
+        for (int e = tid; e < nwin * cpr; e += NCOMP) {
+            const int wi = e / cpr, c8 = e - wi * cpr;
+            float a[8], sc[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) a[k] = 0.f;
+            for (int part = 0; part < nsplit; ++part) {         // fixed order: bit-reproducible
+                const float* d = sPart + ((size_t)wi * nsplit + part) * DK + c8 * 8;
+#pragma unroll
+                for (int k = 0; k < 8; ++k) a[k] += d[k];
+            }
+#pragma unroll
+            for (int k = 0; k < 8; ++k) { a[k] *= inv; sc[k] = a[k] * p.scale1; }
+            const int arow = (ar0 + wi / P) * P + wi % P;
+            *(reinterpret_cast<uint4*>(gAb + (size_t)arow * DK) + c8) = pack16<T>(a);
+            *(reinterpret_cast<uint4*>(gAg + (size_t)arow * DK) + c8) = pack16<T>(sc);
         }
         if (sub == 0)                        // padded agent rows are zero in both copies
             for (int e = tid; e < (RP - n) * cpr; e += NCOMP) {
@@ -310,199 +318,28 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
                 *(reinterpret_cast<uint4*>(gAg + (size_t)n * DK) + e) = make_uint4(0u, 0u, 0u, 0u);
             }
     }
-    // publish these agent rows, wait for the slab's other G tasks
-    publish_add(p.counters + slab);
-    wait_counter_block(ro, p.counters + slab, (unsigned)p.plan.g_tasks, kTimeoutAgents);
+    publish_add(p.counters + slab);        // block barrier, then one release + add
+    fence_proxy_async();
+    __syncthreads();
+    TR(1);
+}
 
-    // ---- phase 1: the loop over the range
-    if (tid == 0) {
-        const uint32_t bar = bar_addr(ro, BAR_AG);
-        mbar_arrive_expect_tx(bar, 2 * kTile);
-        tma_load_2d(astack, &p.tm_ag, 0, slab * RP, bar);
-        tma_load_2d(astack + kTile, &p.tm_ag, 0, slab * RP, bar);
-    }
-    float m_ref = -INFINITY, l = 0.f;
-    bool started = false;
-    const int half = (tid >> 6) & 1;
-    const uint32_t lane_base = ((uint32_t)(32 * (warp & 3))) << 16;
-    const uint32_t tO = ro.tmem + TM_GO + 64 * half + lane_base;
-    if (is_prod) {
-        if (lane == 0) {
-            for (int t = RING; t < tiles; ++t) {
-                wait_bar(ro, BAR_EMPTY + t % RING, kTimeoutRole);
-                fill(t);
-            }
-            for (int t = max(0, tiles - RING); t < tiles; ++t) wait_bar(ro, BAR_EMPTY + t % RING, kTimeoutRole);
-        }
-        __syncwarp();
-    } else if (is_rows) {
-        const uint32_t idK = umma_idesc(fmt, 128, 64, 0), idMN = umma_idesc(fmt, 128, 64, 1);
-        auto issue_S = [&](int j) {          // leader: logits of step j (two tiles) -> buffer j & 1
-            const int nt2 = min(2, tiles - 2 * j);
-            for (int h2 = 0; h2 < nt2; ++h2) wait_bar(ro, BAR_FULL + (2 * j + h2) % RING, kTimeoutTile);
-            tc_fence_after_sync();
-            for (int h2 = 0; h2 < nt2; ++h2) {
-                const uint32_t d = ro.tmem + TM_GS + 128 * (j & 1) + 64 * h2;
-                const uint32_t sK = ring_u32 + ((2 * j + h2) % RING) * kSlot, sB = sK + 2 * kTile;
-#pragma unroll
-                for (int kk = 0; kk < DK / 16; ++kk)
-                    umma_f16(d, umma_desc_sw128(astack + kk * 32), umma_desc_sw128(sK + kk * 32), idK, kk > 0);
-                if (has_bias) {
-#pragma unroll
-                    for (int kk = 0; kk < RP / 16; ++kk)
-                        umma_f16(d, umma_desc_sw128(ident + kk * 32), umma_desc_sw128(sB + kk * 2048), idMN, 1u);
-                }
-            }
-            umma_commit(bar_addr(ro, BAR_S + (j & 1)));
-        };
-        wait_bar(ro, BAR_AG, kTimeoutLoads);
-        if (tid == 0) issue_S(0);
-        for (int j = 0; j < steps; ++j) {
-            const int buf = j & 1;
-            if (tid == 0 && j + 1 < steps) issue_S(j + 1);
-            wait_bar(ro, BAR_S + buf, kTimeoutTile);
-            tc_fence_after_sync();
-            const int t = 2 * j + half;
-            const bool tv = t < tiles;                     // uniform per warp
-            uint32_t pk[32];
-            float corr = 1.f;
-            bool resc = false;
-            if (tv) {
-                const int valid = min(KT, t_end - (t_begin + t * KT));
-                float s[64];
-                {
-                    uint32_t ra[32], rb[32];
-                    const uint32_t ts = ro.tmem + TM_GS + 128 * buf + 64 * half + lane_base;
-                    tmem_ld32(ts, ra);
-                    tmem_ld32(ts + 32, rb);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int k = 0; k < 32; ++k) { s[k] = __uint_as_float(ra[k]); s[32 + k] = __uint_as_float(rb[k]); }
-                }
-                if (valid < KT) {
-#pragma unroll
-                    for (int k = 0; k < 64; ++k) if (k >= valid) s[k] = -INFINITY;
-                }
-                float mx = s[0];
-#pragma unroll
-                for (int k = 1; k < 64; ++k) mx = fmaxf(mx, s[k]);
-                if (mx > m_ref + kTau) {                   // also the first tile of the row (m_ref = -inf)
-                    corr = fast_exp2((m_ref - mx) * kLog2e);
-                    resc = started;
-                    m_ref = mx;
-                    l *= corr;
-                }
-                const float nb = -m_ref * kLog2e;
-                float sum0 = 0.f, sum1 = 0.f;
-#pragma unroll
-                for (int k = 0; k < 32; ++k) {
-                    const float p0 = fast_exp2(fmaf(s[2 * k], kLog2e, nb));       // exp2(-inf) = 0 past the range
-                    const float p1 = fast_exp2(fmaf(s[2 * k + 1], kLog2e, nb));
-                    sum0 += p0; sum1 += p1;
-                    pk[k] = pack2<T>(p0, p1);
-                }
-                l += sum0 + sum1;
-                started = true;
-            }
-            if (j > 0) { wait_bar(ro, BAR_PV, kTimeoutTile); tc_fence_after_sync(); }
-            if (__any_sync(0xffffffffu, resc)) {           // rare: the reference maximum of some row moved
-                uint32_t ra[32];
-#pragma unroll
-                for (int hh = 0; hh < 2; ++hh) {
-                    tmem_ld32(tO + 32 * hh, ra);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int k = 0; k < 32; ++k) ra[k] = __float_as_uint(__uint_as_float(ra[k]) * corr);
-                    tmem_st32(tO + 32 * hh, ra);
-                }
-                tmem_st_wait();
-            }
-            if (tv) {
-#pragma unroll
-                for (int c = 0; c < 8; ++c)
-                    *reinterpret_cast<uint4*>(smem + G_P + tid * 128 + ((c ^ (tid & 7)) << 4)) =
-                        make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
-            }
-            fence_proxy_async();
-            tc_fence_before_sync();
-            sync_rows();
-            if (tid == 0) {
-                tc_fence_after_sync();
-                const int nt2 = min(2, tiles - 2 * j);
-                for (int h2 = 0; h2 < nt2; ++h2) {
-                    const int sl = (2 * j + h2) % RING;
-                    const uint32_t sV = ring_u32 + sl * kSlot + kTile;
-                    const uint32_t d = ro.tmem + TM_GO + 64 * h2;
-#pragma unroll
-                    for (int kk = 0; kk < KT / 16; ++kk)
-                        umma_f16(d, umma_desc_sw128(sP + kk * 32), umma_desc_sw128(sV + kk * 2048), idMN, (j > 0 || kk > 0) ? 1u : 0u);
-                    umma_commit(bar_addr(ro, BAR_EMPTY + sl));
-                }
-                umma_commit(bar_addr(ro, BAR_PV));
-            }
-        }
-        wait_bar(ro, BAR_PV, kTimeoutTile);
-        tc_fence_after_sync();
-    }
-    __syncthreads();                   // the ring is drained: every MMA of the range has completed
-
-    // ---- phase 2: the two stacked halves combine into one partial state of the range
+// ---------------------------------------------------------------------------------- M task
+// All partial states of the slab -> V_A (log-sum-exp merge in the fixed order of the parts).
+template <typename T, typename SH>
+__device__ __forceinline__ void run_m_task(const FusedArgs& p, int slab, Role& ro, int slot) {
+    const int tid = threadIdx.x;
+    const int n = SH::kFixed ? SH::kP * SH::kP : p.n;
     const int parts = p.plan.parts;
     const size_t pf = partial_floats(RP, DK);
-    float* slab_parts = p.partials + (size_t)slab * parts * pf;
-    if (is_rows) {
-        float* sX = reinterpret_cast<float*>(smem + G_RING);        // [64][68]: row, m, l of the upper half
-        float o[64];
-        {
-            uint32_t ra[32], rb[32];
-            tmem_ld32(tO, ra);
-            tmem_ld32(tO + 32, rb);
-            tmem_ld_wait();
-#pragma unroll
-            for (int k = 0; k < 32; ++k) {
-                o[k] = started ? __uint_as_float(ra[k]) : 0.f;
-                o[32 + k] = started ? __uint_as_float(rb[k]) : 0.f;
-            }
-        }
-        tc_fence_before_sync();
-        if (half == 1) {
-            float* x = sX + (tid - 64) * 68;
-#pragma unroll
-            for (int k = 0; k < 16; ++k)
-                *reinterpret_cast<float4*>(x + 4 * k) = make_float4(o[4 * k], o[4 * k + 1], o[4 * k + 2], o[4 * k + 3]);
-            x[64] = m_ref; x[65] = l;
-        }
-        sync_rows();
-        if (half == 0) {
-            const float* x = sX + tid * 68;
-            const float om = x[64], ol = x[65];
-            const float mm = fmaxf(m_ref, om);
-            const float bs = (mm == -INFINITY) ? 0.f : mm;
-            const float wa = fast_exp2((m_ref - bs) * kLog2e), wb = fast_exp2((om - bs) * kLog2e);
-            float* part = slab_parts + (size_t)sub * pf;
-            part[tid] = mm * kLog2e;                       // the merge works in log2 units
-            part[RP + tid] = l * wa + ol * wb;
-            float* pacc = part + 2 * RP + (size_t)tid * DK;
-#pragma unroll
-            for (int k = 0; k < 16; ++k) {
-                const float4 xv = *reinterpret_cast<const float4*>(x + 4 * k);
-                *reinterpret_cast<float4*>(pacc + 4 * k) =
-                    make_float4(o[4 * k] * wa + xv.x * wb, o[4 * k + 1] * wa + xv.y * wb,
-                                o[4 * k + 2] * wa + xv.z * wb, o[4 * k + 3] * wa + xv.w * wb);
-            }
-        }
-    }
-    // when all of the slab's partial states are written, every G task merges its share of the agent
-    // rows (fixed order of the parts: bit-reproducible) and counts itself done on the slab's flag
-    unsigned* arrived = p.counters + p.slabs + slab;
-    publish_add(arrived);
-    wait_counter_block(ro, arrived, (unsigned)p.plan.g_tasks, kTimeoutAgents);
-    if (!is_prod) {
-        const int rows_per = (n + p.plan.g_tasks - 1) / p.plan.g_tasks;
-        const int rb = sub * rows_per, re = min(n, rb + rows_per);
+    const float* slab_parts = p.partials + (size_t)slab * parts * pf;
+    TR(0);
+    wait_counter_block(ro, p.counters + p.slabs + slab, (unsigned)p.plan.g_tasks, kTimeoutAgents);
+    TR(1);
+    if (tid < NCOMP) {
         T* va = static_cast<T*>(p.va2_ws) + (size_t)slab * RP * DK;
-        for (int e = tid; e < (re - rb) * (DK / 4); e += NCOMP) {
-            const int r = rb + e / (DK / 4), c = (e % (DK / 4)) * 4;
+        for (int e = tid; e < n * (DK / 4); e += NCOMP) {
+            const int r = e / (DK / 4), c = (e % (DK / 4)) * 4;
             float mx = -INFINITY, den = 0.f;
             float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll 8
@@ -525,13 +362,297 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
             o.y = pack2<T>(num.z * inv, num.w * inv);
             *reinterpret_cast<uint2*>(va + (size_t)r * DK + c) = o;
         }
-        if (sub == 0)                        // padded feature rows are zero (0 * NaN is not 0)
-            for (int e = tid; e < (RP - n) * cpr; e += NCOMP)
-                *(reinterpret_cast<uint4*>(va + (size_t)n * DK) + e) = make_uint4(0u, 0u, 0u, 0u);
+        // padded feature rows are zero (0 * NaN is not 0)
+        for (int e = tid; e < (RP - n) * (DK / 8); e += NCOMP)
+            *(reinterpret_cast<uint4*>(va + (size_t)n * DK) + e) = make_uint4(0u, 0u, 0u, 0u);
     }
     publish_add(p.counters + 2 * p.slabs + slab);
+    __syncthreads();
+    TR(2);
+}
+
+// ---------------------------------------------------------------------------------- G task
+template <typename T, typename SH>
+__device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub, unsigned char* smem, Role& ro, int slot) {
+    constexpr int fmt = Elem<T>::kIsBf16 ? 1 : 0;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int head = slab % p.heads;
+    const int H = SH::kFixed ? SH::kH : p.H, W = SH::kFixed ? SH::kW : p.W;
+    const int N = H * W, n = SH::kFixed ? SH::kP * SH::kP : p.n;
+    const int gr0 = sub * p.plan.rows_per_g, gr1 = min(H, gr0 + p.plan.rows_per_g);
+    const int t_begin = gr0 * W, t_end = gr1 * W;
+    const int tiles = (t_end - t_begin + KT - 1) / KT;
+    const int steps = (tiles + 1) >> 1;
+    const bool has_bias = SH::kFixed ? true : (p.b1 != nullptr);
+    const bool bias_tma = has_bias && p.b1_tma;
+    const bool prep = has_bias;                    // identity operand (and plain-load bias tiles) to build
+
+    const uint32_t ring_u32 = smem_u32(smem + G_RING);
+    const uint32_t astack = smem_u32(smem + G_ASTACK), ident = smem_u32(smem + G_IDENT), sP = smem_u32(smem + G_P);
+    const size_t pf = partial_floats(RP, DK);
+    TR(0);
+
+    if (warp == kWarpProd) {
+        // ------------------------------------------------------------------ producer
+        if (lane == 0) {
+            const uint32_t tile_tx = 2 * kTile + (bias_tma ? kTile : 0);
+            auto fill = [&](int t) {
+                const int s = t % RING, c0 = t_begin + t * KT;
+                const uint32_t bar = bar_addr(ro, BAR_FULL + s), dst = ring_u32 + s * kSlot;
+                mbar_arrive_expect_tx(bar, tile_tx);
+                tma_load_2d(dst, &p.tm_k, 0, slab * N + c0, bar);
+                tma_load_2d(dst + kTile, &p.tm_v, 0, slab * N + c0, bar);
+                if (bias_tma) tma_load_2d(dst + 2 * kTile, &p.tm_b1, c0, head * n, bar);
+            };
+            for (int t = 0; t < tiles && t < RING; ++t) fill(t);
+            // the slab's agents: every P task of the slab has published its rows
+            poll_counter(ro, p.counters + slab, (unsigned)p.plan.g_tasks, kTimeoutAgents);
+            {
+                const uint32_t bar = bar_addr(ro, BAR_AG);
+                mbar_arrive_expect_tx(bar, 2 * kTile);
+                tma_load_2d(astack, &p.tm_ag, 0, slab * RP, bar);
+                tma_load_2d(astack + kTile, &p.tm_ag, 0, slab * RP, bar);
+            }
+            for (int t = RING; t < tiles; ++t) {
+                wait_bar_one(ro, BAR_EMPTY + t % RING, kTimeoutRole);
+                fill(t);
+            }
+            for (int t = max(0, tiles - RING); t < tiles; ++t) wait_bar_one(ro, BAR_EMPTY + t % RING, kTimeoutRole);
+        }
+        __syncwarp();
+    } else if (warp == kWarpMma) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t idK = umma_idesc(fmt, 128, 64, 0), idMN = umma_idesc(fmt, 128, 64, 1);
+            const uint64_t dA = umma_desc_sw128(astack), dI = umma_desc_sw128(ident), dP = umma_desc_sw128(sP);
+            const uint64_t dRing = umma_desc_sw128(ring_u32);
+            // descriptor start addresses count 16-byte units: + 2 per 32 bytes (one K-step of a K-major
+            // operand), + 128 per 2048 bytes (one K-step of an MN-major operand)
+            auto issue_S = [&](int j) {
+                const int nt2 = min(2, tiles - 2 * j);
+                if (j >= 2) wait_bar_one(ro, BAR_S_EMPTY + (j & 1), kTimeoutRole);
+                for (int h2 = 0; h2 < nt2; ++h2) wait_bar_one(ro, BAR_FULL + (2 * j + h2) % RING, kTimeoutTile);
+                tc_fence_after_sync();
+                for (int h2 = 0; h2 < nt2; ++h2) {
+                    const uint32_t d = ro.tmem + TM_GS + 128 * (j & 1) + 64 * h2;
+                    const uint64_t dK = dRing + (uint64_t)(((2 * j + h2) % RING) * (kSlot >> 4));
+                    const uint64_t dB = dK + (uint64_t)((2 * kTile) >> 4);
+#pragma unroll
+                    for (int kk = 0; kk < DK / 16; ++kk) umma_f16(d, dA + 2 * kk, dK + 2 * kk, idK, kk > 0);
+                    if (has_bias) {
+#pragma unroll
+                        for (int kk = 0; kk < RP / 16; ++kk) umma_f16(d, dI + 2 * kk, dB + 128 * kk, idMN, 1u);
+                    }
+                }
+                umma_commit(bar_addr(ro, BAR_S_FULL + (j & 1)));
+            };
+            if (prep) wait_bar_one(ro, BAR_PREP, kTimeoutRole);
+            wait_bar_one(ro, BAR_AG, kTimeoutLoads);
+            unsigned started = 0u;                    // accumulators that hold a product already
+            issue_S(0);
+            for (int j = 0; j < steps; ++j) {
+                if (j + 1 < steps) issue_S(j + 1);
+                wait_bar_one(ro, BAR_PG_FULL, kTimeoutRole);
+                tc_fence_after_sync();
+                const int nt2 = min(2, tiles - 2 * j);
+                for (int h2 = 0; h2 < nt2; ++h2) {
+                    const int t = 2 * j + h2, sl = t % RING;
+                    const int ntok = min(KT, t_end - (t_begin + t * KT));
+                    const uint64_t dV = dRing + (uint64_t)(sl * (kSlot >> 4)) + (uint64_t)(kTile >> 4);
+                    for (int c = 0; c < 2; ++c) {
+                        if (32 * c >= ntok) break;
+                        const int a = 2 * h2 + c;
+                        const uint32_t d = ro.tmem + TM_GO + 64 * a;
+#pragma unroll
+                        for (int k2 = 0; k2 < 2; ++k2) {
+                            const int kk = 2 * c + k2;
+                            umma_f16(d, dP + 2 * kk, dV + 128 * kk, idMN, (((started >> a) & 1u) || k2 > 0) ? 1u : 0u);
+                        }
+                        started |= 1u << a;
+                    }
+                    umma_commit(bar_addr(ro, BAR_EMPTY + sl));
+                }
+                umma_commit(bar_addr(ro, BAR_PV));
+            }
+            for (int j = max(0, steps - 2); j < steps; ++j) wait_bar_one(ro, BAR_S_EMPTY + (j & 1), kTimeoutRole);
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------------ compute warps
+        if (prep) {
+            // identity, stacked twice: row r has a one at k = r % 64 (the A operand of the bias K-block)
+            const unsigned short one = Elem<T>::kIsBf16 ? 0x3F80u : 0x3C00u;
+            for (int idx = tid; idx < 128 * 8; idx += NCOMP) {
+                const int row = idx >> 3, c = idx & 7;
+                const int lc = c ^ (row & 7);                 // logical 16-byte chunk: k = 8 lc .. 8 lc + 7
+                uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                const int k = row & 63;
+                if ((k >> 3) == lc) {
+                    const uint32_t w = (uint32_t)one << (16 * (k & 1));
+                    const int wi = (k & 7) >> 1;
+                    if (wi == 0) v.x = w; else if (wi == 1) v.y = w; else if (wi == 2) v.z = w; else v.w = w;
+                }
+                *reinterpret_cast<uint4*>(smem + G_IDENT + row * 128 + c * 16) = v;
+            }
+            if (!bias_tma) {                 // the plan guarantees tiles <= RING here
+                const T* gB = static_cast<const T*>(p.b1) + (size_t)head * n * N;
+                for (int t = 0; t < tiles; ++t) {
+                    unsigned char* sB = smem + G_RING + (t % RING) * kSlot + 2 * kTile;
+                    const int c0 = t_begin + t * KT;
+                    for (int e = tid; e < RP * KT; e += NCOMP) {
+                        const int rr = e / KT, j = e - rr * KT;
+                        const int key = c0 + j;
+                        *reinterpret_cast<T*>(sB + swz(rr, j)) =
+                            (rr < n && key < t_end) ? gB[(size_t)rr * N + key] : Elem<T>::from_f32(0.f);
+                    }
+                }
+            }
+            fence_proxy_async();             // the tensor core reads these through the async proxy
+            sync_compute();
+            if (tid == 0) mbar_arrive(bar_addr(ro, BAR_PREP));
+        }
+        if (warp < NR / 32) {
+            // -------------------------------------------------------------- row warps
+            const int row = tid & 127, ch = tid >> 7;          // tensor-memory lane, token half of the tile
+            const int half = row >> 6;                         // stack half: which tile of the step
+            const uint32_t lane_base = ((uint32_t)(32 * (warp & 3))) << 16;
+            const uint32_t tO = ro.tmem + TM_GO + 64 * (2 * half + ch) + lane_base;
+            float m_ref = -INFINITY, l = 0.f;
+            bool started = false;
+            for (int j = 0; j < steps; ++j) {
+                const int buf = j & 1;
+                wait_bar(ro, BAR_S_FULL + buf, kTimeoutTile);
+                tc_fence_after_sync();
+                const int t = 2 * j + half;
+                int valid = 0;
+                if (t < tiles) valid = min(32, t_end - (t_begin + t * KT + 32 * ch));
+                const bool tv = valid > 0;                     // uniform per warp
+                float s[32];
+                {
+                    uint32_t ra[32];
+                    tmem_ld32(ro.tmem + TM_GS + 128 * buf + 64 * half + 32 * ch + lane_base, ra);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int k = 0; k < 32; ++k) s[k] = __uint_as_float(ra[k]);
+                }
+                tc_fence_before_sync();
+                mbar_arrive(bar_addr(ro, BAR_S_EMPTY + buf));
+                uint32_t pk[16];
+                float corr = 1.f;
+                bool resc = false;
+                if (tv) {
+                    if (valid < 32) {
+#pragma unroll
+                        for (int k = 0; k < 32; ++k) if (k >= valid) s[k] = -INFINITY;
+                    }
+                    float mx0 = fmaxf(s[0], s[1]), mx1 = fmaxf(s[2], s[3]), mx2 = fmaxf(s[4], s[5]), mx3 = fmaxf(s[6], s[7]);
+#pragma unroll
+                    for (int k = 8; k < 32; k += 8) {
+                        mx0 = fmaxf(mx0, fmaxf(s[k], s[k + 1]));     mx1 = fmaxf(mx1, fmaxf(s[k + 2], s[k + 3]));
+                        mx2 = fmaxf(mx2, fmaxf(s[k + 4], s[k + 5])); mx3 = fmaxf(mx3, fmaxf(s[k + 6], s[k + 7]));
+                    }
+                    const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+                    if (mx > m_ref + kTau) {                   // also the first tile of the row (m_ref = -inf)
+                        corr = fast_exp2((m_ref - mx) * kLog2e);
+                        resc = started;
+                        m_ref = mx;
+                        l *= corr;
+                    }
+                    const float nb = -m_ref * kLog2e;
+                    float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
+#pragma unroll
+                    for (int k = 0; k < 16; k += 2) {
+                        const float p0 = fast_exp2(fmaf(s[2 * k], kLog2e, nb));       // exp2(-inf) = 0 past the range
+                        const float p1 = fast_exp2(fmaf(s[2 * k + 1], kLog2e, nb));
+                        const float p2 = fast_exp2(fmaf(s[2 * k + 2], kLog2e, nb));
+                        const float p3 = fast_exp2(fmaf(s[2 * k + 3], kLog2e, nb));
+                        sum0 += p0; sum1 += p1; sum2 += p2; sum3 += p3;
+                        pk[k] = pack2<T>(p0, p1);
+                        pk[k + 1] = pack2<T>(p2, p3);
+                    }
+                    l += (sum0 + sum1) + (sum2 + sum3);
+                    started = true;
+                }
+                if (j > 0) { wait_bar(ro, BAR_PV, kTimeoutTile); tc_fence_after_sync(); }
+                if (__any_sync(0xffffffffu, resc)) {           // rare: the reference maximum of some row moved
+                    uint32_t ra[32];
+#pragma unroll
+                    for (int hh = 0; hh < 2; ++hh) {
+                        tmem_ld32(tO + 32 * hh, ra);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int k = 0; k < 32; ++k) ra[k] = __float_as_uint(__uint_as_float(ra[k]) * corr);
+                        tmem_st32(tO + 32 * hh, ra);
+                    }
+                    tmem_st_wait();
+                }
+                if (tv) {
+#pragma unroll
+                    for (int c = 0; c < 4; ++c)
+                        *reinterpret_cast<uint4*>(smem + G_P + row * 128 + (((4 * ch + c) ^ (row & 7)) << 4)) =
+                            make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+                }
+                fence_proxy_async();
+                tc_fence_before_sync();
+                mbar_arrive(bar_addr(ro, BAR_PG_FULL));
+            }
+            wait_bar(ro, BAR_PV, kTimeoutTile);
+            tc_fence_after_sync();
+            TR(1);
+            // the four states of an agent row (stack half x token half) meet in shared memory
+            float* sX = reinterpret_cast<float*>(smem + G_RING);        // [4][64][68]: row, m, l
+            {
+                uint32_t ra[32], rb[32];
+                tmem_ld32(tO, ra);
+                tmem_ld32(tO + 32, rb);
+                tmem_ld_wait();
+                float* x = sX + ((size_t)(2 * half + ch) * 64 + (row & 63)) * 68;
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    *reinterpret_cast<float4*>(x + 4 * k) = started
+                        ? make_float4(__uint_as_float(ra[4 * k]), __uint_as_float(ra[4 * k + 1]), __uint_as_float(ra[4 * k + 2]), __uint_as_float(ra[4 * k + 3]))
+                        : make_float4(0.f, 0.f, 0.f, 0.f);
+                    *reinterpret_cast<float4*>(x + 32 + 4 * k) = started
+                        ? make_float4(__uint_as_float(rb[4 * k]), __uint_as_float(rb[4 * k + 1]), __uint_as_float(rb[4 * k + 2]), __uint_as_float(rb[4 * k + 3]))
+                        : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+                x[64] = m_ref; x[65] = started ? l : 0.f;
+            }
+            tc_fence_before_sync();
+            sync_rows();
+            {
+                const int a = tid & 63, q = tid >> 6;          // agent row, quarter of the channels
+                float mm = -INFINITY;
+#pragma unroll
+                for (int st = 0; st < 4; ++st) mm = fmaxf(mm, sX[((size_t)st * 64 + a) * 68 + 64]);
+                const float bs = (mm == -INFINITY) ? 0.f : mm;
+                float wgt[4], lsum = 0.f;
+#pragma unroll
+                for (int st = 0; st < 4; ++st) {
+                    wgt[st] = fast_exp2((sX[((size_t)st * 64 + a) * 68 + 64] - bs) * kLog2e);     // exp2(-inf) = 0
+                    lsum += sX[((size_t)st * 64 + a) * 68 + 65] * wgt[st];
+                }
+                float* part = p.partials + ((size_t)slab * p.plan.parts + sub) * pf;
+                if (q == 0) { part[a] = mm * kLog2e; part[RP + a] = lsum; }      // the merge works in log2 units
+                float* pacc = part + 2 * RP + (size_t)a * DK + 16 * q;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                    for (int st = 0; st < 4; ++st) {
+                        const float4 xv = *reinterpret_cast<const float4*>(sX + ((size_t)st * 64 + a) * 68 + 16 * q + 4 * k);
+                        acc.x += xv.x * wgt[st]; acc.y += xv.y * wgt[st]; acc.z += xv.z * wgt[st]; acc.w += xv.w * wgt[st];
+                    }
+                    *reinterpret_cast<float4*>(pacc + 4 * k) = acc;
+                }
+            }
+        }
+    }
+    TR(2);
+    publish_add(p.counters + p.slabs + slab);       // block barrier (the ring is drained), release + add
     fence_proxy_async();   // this task's plain shared-memory writes precede the next task's TMA writes
     __syncthreads();
+    TR(3);
 }
 
 // ---------------------------------------------------------------------------------- B task
@@ -541,10 +662,9 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
 // are fetched.
 template <typename T, typename SH>
 __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int run, unsigned char* smem, Role& ro,
-                                           int* s_whead) {
+                                           int* s_whead, float (*s_red)[128], int slot) {
     constexpr int fmt = Elem<T>::kIsBf16 ? 1 : 0;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const bool is_prod = warp == 8, is_rows = warp < 4;
     const int head = slab % p.heads;
     const int H = SH::kFixed ? SH::kH : p.H, W = SH::kFixed ? SH::kW : p.W;
     const int N = H * W, n = SH::kFixed ? SH::kP * SH::kP : p.n;
@@ -560,15 +680,15 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int run
     float* sW = reinterpret_cast<float*>(smem + OFF_W);
     T* sV = reinterpret_cast<T*>(smem + B_V);
     const T* gV = static_cast<const T*>(p.v) + (size_t)slab * N * DK;
-    const unsigned char* b2base = has_b2 ? reinterpret_cast<const unsigned char*>(p.b2) + (size_t)head * N * n * 2 : nullptr;
     const size_t b2_total = (size_t)p.heads * N * n * 2;           // bytes of the whole B2 array
     const size_t b2_head_off = (size_t)head * N * n * 2;
     auto slot_of = [&](int y) { return (y - y_first + 1) % NSLOT; };
+    TR(0);
 
-    if (is_prod) {
+    if (warp == kWarpProd) {
         // ------------------------------------------------------------------ producer
         if (lane == 0) {
-            poll_counter(ro, p.counters + 2 * p.slabs + slab, (unsigned)p.plan.g_tasks, kTimeoutFeatures);
+            poll_counter(ro, p.counters + 2 * p.slabs + slab, 1u, kTimeoutFeatures);     // the slab's M task is done
             {
                 const uint32_t bar = bar_addr(ro, BAR_AG);
                 mbar_arrive_expect_tx(bar, 2 * kTile);
@@ -579,7 +699,7 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int run
                 const int b = i & 1;
                 const int y0 = y_first + i * R, rows = min(R, H - y0);
                 const int q0 = y0 * W, TQ = rows * W;
-                if (i >= 2) wait_bar(ro, BAR_IN_EMPTY + b, kTimeoutRole);
+                if (i >= 2) wait_bar_one(ro, BAR_IN_EMPTY + b, kTimeoutRole);
                 {
                     // B2 rows of the tile: the 16-byte aligned span that covers them, clipped to the array
                     uint32_t nb2 = 0;
@@ -597,7 +717,7 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int run
                     if (nb2) bulk_load_1d(smem_u32(smem + B_B2 + b * kB2Buf), reinterpret_cast<const unsigned char*>(p.b2) + lo, nb2, bar);
                 }
                 if (has_dwc) {
-                    if (i >= 2) wait_bar(ro, BAR_V_EMPTY + b, kTimeoutRole);
+                    if (i >= 2) wait_bar_one(ro, BAR_V_EMPTY + b, kTimeoutRole);
                     int ylo = (i == 0) ? y0 - 1 : y0 + 1, yhi = y0 + rows;
                     if (ylo < 0) ylo = 0;
                     if (yhi > H - 1) yhi = H - 1;
@@ -609,45 +729,60 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int run
                 }
             }
             for (int i = max(0, nt - 2); i < nt; ++i) {
-                wait_bar(ro, BAR_IN_EMPTY + (i & 1), kTimeoutRole);
-                if (has_dwc) wait_bar(ro, BAR_V_EMPTY + (i & 1), kTimeoutRole);
+                wait_bar_one(ro, BAR_IN_EMPTY + (i & 1), kTimeoutRole);
+                if (has_dwc) wait_bar_one(ro, BAR_V_EMPTY + (i & 1), kTimeoutRole);
             }
         }
         __syncwarp();
-    } else if (is_rows) {
-        // ------------------------------------------------------------------ row group
-        const uint32_t lane_base = ((uint32_t)(32 * (warp & 3))) << 16;
-        const uint32_t idK = umma_idesc(fmt, 128, 64, 0), idMN = umma_idesc(fmt, 128, 64, 1);
-        const uint32_t sA = smem_u32(smem + B_A), sVA = smem_u32(smem + B_VA), sP = smem_u32(smem + B_P);
-        auto issue_S = [&](int i) {
-            const int b = i & 1;
-            wait_bar(ro, BAR_IN_FULL + b, kTimeoutLoads);
-            tc_fence_after_sync();
-            const uint32_t sQ = smem_u32(smem + B_Q + b * 2 * kTile);
+    } else if (warp == kWarpMma) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t idK = umma_idesc(fmt, 128, 64, 0), idMN = umma_idesc(fmt, 128, 64, 1);
+            const uint64_t dA = umma_desc_sw128(smem_u32(smem + B_A)), dVA = umma_desc_sw128(smem_u32(smem + B_VA));
+            const uint64_t dP = umma_desc_sw128(smem_u32(smem + B_P)), dQ0 = umma_desc_sw128(smem_u32(smem + B_Q));
+            auto issue_S = [&](int i) {
+                const int b = i & 1;
+                if (i >= 2) wait_bar_one(ro, BAR_S_EMPTY + b, kTimeoutRole);
+                wait_bar_one(ro, BAR_IN_FULL + b, kTimeoutLoads);
+                tc_fence_after_sync();
+                const uint64_t dQ = dQ0 + (uint64_t)(b * ((2 * kTile) >> 4));
 #pragma unroll
-            for (int kk = 0; kk < DK / 16; ++kk)
-                umma_f16(ro.tmem + TM_BS + 64 * b, umma_desc_sw128(sQ + kk * 32), umma_desc_sw128(sA + kk * 32), idK, kk > 0);
-            umma_commit(bar_addr(ro, BAR_S + b));
-        };
-        wait_bar(ro, BAR_AG, kTimeoutLoads);
-        if (tid == 0) issue_S(0);
+                for (int kk = 0; kk < DK / 16; ++kk) umma_f16(ro.tmem + TM_BS + 64 * b, dQ + 2 * kk, dA + 2 * kk, idK, kk > 0);
+                umma_commit(bar_addr(ro, BAR_S_FULL + b));
+            };
+            wait_bar_one(ro, BAR_AG, kTimeoutLoads);
+            issue_S(0);
+            for (int i = 0; i < nt; ++i) {
+                if (i + 1 < nt) issue_S(i + 1);
+                wait_bar_one(ro, BAR_PB_FULL, kTimeoutRole);
+                tc_fence_after_sync();
+                for (int kk = 0; kk < n16; ++kk) umma_f16(ro.tmem + TM_BO + 64 * (i & 1), dP + 2 * kk, dVA + 128 * kk, idMN, kk > 0);
+                umma_commit(bar_addr(ro, BAR_PV));
+            }
+            for (int i = max(0, nt - 2); i < nt; ++i) wait_bar_one(ro, BAR_S_EMPTY + (i & 1), kTimeoutRole);
+        }
+        __syncwarp();
+    } else if (warp < NR / 32) {
+        // ------------------------------------------------------------------ row warps
+        const int row = tid & 127, ch = tid >> 7;              // query row of the tile, half of the agent columns
+        const uint32_t lane_base = ((uint32_t)(32 * (warp & 3))) << 16;
+        const int c0 = 32 * ch;
         for (int i = 0; i < nt; ++i) {
             const int b = i & 1;
             const int y0 = y_first + i * R, rows = min(R, H - y0);
             const int q0 = y0 * W, TQ = rows * W;
-            if (tid == 0 && i + 1 < nt) issue_S(i + 1);
-            wait_bar(ro, BAR_S + b, kTimeoutLoads);
+            wait_bar(ro, BAR_S_FULL + b, kTimeoutLoads);
             tc_fence_after_sync();
-            float s[64];
+            float s[32];
             {
-                uint32_t ra[32], rb[32];
-                const uint32_t ts = ro.tmem + TM_BS + 64 * b + lane_base;
-                tmem_ld32(ts, ra);
-                tmem_ld32(ts + 32, rb);
+                uint32_t ra[32];
+                tmem_ld32(ro.tmem + TM_BS + 64 * b + c0 + lane_base, ra);
                 tmem_ld_wait();
 #pragma unroll
-                for (int k = 0; k < 32; ++k) { s[k] = __uint_as_float(ra[k]); s[32 + k] = __uint_as_float(rb[k]); }
+                for (int k = 0; k < 32; ++k) s[k] = __uint_as_float(ra[k]);
             }
+            tc_fence_before_sync();
+            mbar_arrive(bar_addr(ro, BAR_S_EMPTY + b));
             // logits in natural units: t = scale2 * q.a + b2; columns >= n are not agents
             float mx = -INFINITY;
             if (has_b2) {
@@ -662,36 +797,39 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int run
                             *reinterpret_cast<const unsigned short*>(reinterpret_cast<const unsigned char*>(p.b2) + g);
                     sync_rows();
                 }
-                // element index of this row's first bias value inside the buffer (the copy starts at a 16-byte boundary)
-                const uint32_t e0 = (uint32_t)(((b2_head_off + (size_t)q0 * n * 2) & 15) >> 1) + (uint32_t)tid * n;
+                // element index of this thread's first bias value inside the buffer (the copy starts at a 16-byte boundary)
+                const uint32_t e0 = (uint32_t)((beg & 15) >> 1) + (uint32_t)row * n + c0;
                 const uint32_t* w32 = reinterpret_cast<const uint32_t*>(smem + B_B2 + b * kB2Buf) + (e0 >> 1);
                 const int sh = (e0 & 1) * 16;
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    if (2 * j < n) {
+                for (int j = 0; j < 16; ++j) {
+                    if (c0 + 2 * j < n) {
                         const float2 bb = unpack2<T>(__funnelshift_r(w32[j], w32[j + 1], sh));
                         s[2 * j] = fmaf(s[2 * j], p.scale2, bb.x);
-                        s[2 * j + 1] = (2 * j + 1 < n) ? fmaf(s[2 * j + 1], p.scale2, bb.y) : -INFINITY;
+                        s[2 * j + 1] = (c0 + 2 * j + 1 < n) ? fmaf(s[2 * j + 1], p.scale2, bb.y) : -INFINITY;
                         mx = fmaxf(mx, fmaxf(s[2 * j], s[2 * j + 1]));
                     }
                 }
             } else {
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    if (2 * j < n) {
+                for (int j = 0; j < 16; ++j) {
+                    if (c0 + 2 * j < n) {
                         s[2 * j] = s[2 * j] * p.scale2;
-                        s[2 * j + 1] = (2 * j + 1 < n) ? s[2 * j + 1] * p.scale2 : -INFINITY;
+                        s[2 * j + 1] = (c0 + 2 * j + 1 < n) ? s[2 * j + 1] * p.scale2 : -INFINITY;
                         mx = fmaxf(mx, fmaxf(s[2 * j], s[2 * j + 1]));
                     }
                 }
             }
-            mbar_arrive(bar_addr(ro, BAR_IN_EMPTY + b));     // the Q tile and this row's bias values are consumed
+            mbar_arrive(bar_addr(ro, BAR_IN_EMPTY + b));     // the Q tile and this thread's bias values are consumed
+            s_red[ch][row] = mx;
+            sync_rows();
+            mx = fmaxf(mx, s_red[ch ^ 1][row]);
             const float nm = -mx * kLog2e;
             float l0 = 0.f, l1 = 0.f;
-            uint32_t pk[32];
+            uint32_t pk[16];
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                if (2 * j < n) {
+            for (int j = 0; j < 16; ++j) {
+                if (c0 + 2 * j < n) {
                     const float p0 = fast_exp2(fmaf(s[2 * j], kLog2e, nm));
                     const float p1 = fast_exp2(fmaf(s[2 * j + 1], kLog2e, nm));      // exp2(-inf) = 0 past the last agent
                     pk[j] = pack2<T>(p0, p1);
@@ -701,61 +839,51 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int run
                     pk[j] = 0u;
                 }
             }
+            s_red[2 + ch][row] = l0 + l1;
 #pragma unroll
-            for (int c = 0; c < 8; ++c)
-                *reinterpret_cast<uint4*>(smem + B_P + tid * 128 + ((c ^ (tid & 7)) << 4)) =
+            for (int c = 0; c < 4; ++c)
+                *reinterpret_cast<uint4*>(smem + B_P + row * 128 + (((4 * ch + c) ^ (row & 7)) << 4)) =
                     make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
             fence_proxy_async();
-            tc_fence_before_sync();
             sync_rows();
-            if (tid == 0) {
-                tc_fence_after_sync();
-                for (int kk = 0; kk < n16; ++kk)
-                    umma_f16(ro.tmem + TM_BO + 64 * b, umma_desc_sw128(sP + kk * 32), umma_desc_sw128(sVA + kk * 2048), idMN, kk > 0);
-                umma_commit(bar_addr(ro, BAR_PV));
-            }
+            if (tid == 0) mbar_arrive(bar_addr(ro, BAR_PB_FULL));
+            const float inv = 1.f / (l0 + l1 + s_red[2 + (ch ^ 1)][row]);
             wait_bar(ro, BAR_PV, kTimeoutLoads);
             tc_fence_after_sync();
             if (i >= 2) wait_bar(ro, BAR_PATCH_EMPTY + b, kTimeoutRole);
             {
-                const float inv = 1.f / (l0 + l1);
-                float* prow = reinterpret_cast<float*>(smem + B_PATCH + b * kPatch) + tid * PO;
-                uint32_t ra[32], rb[32];
-                const uint32_t to = ro.tmem + TM_BO + 64 * b + lane_base;
-                tmem_ld32(to, ra);
-                tmem_ld32(to + 32, rb);
+                float* prow = reinterpret_cast<float*>(smem + B_PATCH + b * kPatch) + row * PO + c0;
+                uint32_t ra[32];
+                tmem_ld32(ro.tmem + TM_BO + 64 * b + c0 + lane_base, ra);
                 tmem_ld_wait();
-                if (tid < TQ) {
+                if (row < TQ) {
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) {
+                    for (int k = 0; k < 8; ++k)
                         *reinterpret_cast<float4*>(prow + 4 * k) =
                             make_float4(__uint_as_float(ra[4 * k]) * inv, __uint_as_float(ra[4 * k + 1]) * inv,
                                         __uint_as_float(ra[4 * k + 2]) * inv, __uint_as_float(ra[4 * k + 3]) * inv);
-                        *reinterpret_cast<float4*>(prow + 32 + 4 * k) =
-                            make_float4(__uint_as_float(rb[4 * k]) * inv, __uint_as_float(rb[4 * k + 1]) * inv,
-                                        __uint_as_float(rb[4 * k + 2]) * inv, __uint_as_float(rb[4 * k + 3]) * inv);
-                    }
                 }
                 tc_fence_before_sync();
             }
             mbar_arrive(bar_addr(ro, BAR_PATCH_FULL + b));
         }
+        TR(1);
         for (int i = max(0, nt - 2); i < nt; ++i) wait_bar(ro, BAR_PATCH_EMPTY + (i & 1), kTimeoutRole);
     } else {
-        // ------------------------------------------------------------------ stencil group
-        const int t2 = tid - 128;
+        // ------------------------------------------------------------------ stencil warps
+        const int t2 = tid - NR;
         if (has_dwc) {
             // zero columns x = -1 and x = W of every slot; the row above the grid if the run starts the slab
-            for (int e = t2; e < NSLOT * 2 * (DK / 8); e += 128) {
+            for (int e = t2; e < NSLOT * 2 * (DK / 8); e += NX) {
                 const int sl = e / (2 * (DK / 8)), rest = e - sl * 2 * (DK / 8);
                 const int side = rest / (DK / 8), c = rest - side * (DK / 8);
                 *(reinterpret_cast<uint4*>(sV + ((size_t)sl * HP + (side ? W + 1 : 0)) * DK) + c) = make_uint4(0, 0, 0, 0);
             }
             if (y_first == 0)
-                for (int e = t2; e < W * (DK / 8); e += 128) *(reinterpret_cast<uint4*>(sV + DK) + e) = make_uint4(0, 0, 0, 0);
+                for (int e = t2; e < W * (DK / 8); e += NX) *(reinterpret_cast<uint4*>(sV + DK) + e) = make_uint4(0, 0, 0, 0);
             if (ld_shared_volatile(s_whead) != head) {       // filter taps change only with the head
                 const T* w = static_cast<const T*>(p.dwc_w) + (size_t)head * DK * 9;
-                for (int e = t2; e < 9 * DK; e += 128) {
+                for (int e = t2; e < 9 * DK; e += NX) {
                     const int c = e / 9, tap = e - c * 9;
                     sW[tap * DK + c] = Elem<T>::to_f32(w[e]);
                 }
@@ -771,7 +899,7 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int run
                 wait_bar(ro, BAR_V_FULL + b, kTimeoutLoads);
                 if (y0 + rows >= H) {            // the row below the grid
                     T* z = sV + ((size_t)slot_of(H) * HP + 1) * DK;
-                    for (int e = t2; e < W * (DK / 8); e += 128) *(reinterpret_cast<uint4*>(z) + e) = make_uint4(0, 0, 0, 0);
+                    for (int e = t2; e < W * (DK / 8); e += NX) *(reinterpret_cast<uint4*>(z) + e) = make_uint4(0, 0, 0, 0);
                     sync_stencil();
                 }
             }
@@ -781,12 +909,12 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int run
                 constexpr int NCQ = DK / 4;
                 const float* sPatch = reinterpret_cast<const float*>(smem + B_PATCH + b * kPatch);
                 const int npairs = rows * NCQ;
-                int nseg = 128 / npairs;
+                int nseg = NX / npairs;
                 if (nseg < 1) nseg = 1;
                 if (nseg > W) nseg = W;
                 const int seg_len = (W + nseg - 1) / nseg;
                 T* gO = static_cast<T*>(p.out) + ((size_t)slab * N + q0) * DK;
-                for (int item = t2; item < npairs * nseg; item += 128) {
+                for (int item = t2; item < npairs * nseg; item += NX) {
                     const int pair = item % npairs, seg = item / npairs;
                     const int r = pair / NCQ, cq = pair - r * NCQ;
                     const int x0 = seg * seg_len, x1 = min(W, x0 + seg_len);
@@ -855,30 +983,33 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int run
             mbar_arrive(bar_addr(ro, BAR_PATCH_EMPTY + b));
         }
     }
+    TR(2);
     fence_proxy_async();   // this task's plain shared-memory writes precede the next task's TMA writes
     __syncthreads();       // shared memory is free for the next task
+    TR(3);
 }
 
 // ---------------------------------------------------------------------------------- kernel
+// Queue order: stage t holds the B tasks of slab group t-3, the M tasks of group t-2, the G tasks of
+// group t-1 and the P tasks of group t (groups of plan.lag slabs), so every task's inputs come from an
+// earlier stage.
 template <typename T, typename SH>
 __global__ void __launch_bounds__(NT, 1) fused2_kernel(const __grid_constant__ FusedArgs p) {
     extern __shared__ unsigned char smem_raw[];
-    __shared__ int s_task, s_whead, s_dead;
+    __shared__ int s_info[4], s_whead, s_dead;
     __shared__ uint32_t s_tmem;
+    __shared__ float s_red[4][128];     // per query row: maxima and sums of the two column halves
     unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     const int tid = threadIdx.x;
     Role ro;
     ro.status = p.status;
     ro.dead = &s_dead;
     ro.bars = smem_u32(smem + OFF_BAR);
-    ro.ph = 0u;
+    ro.ph = 0ull;
     if (tid == 0) {
         s_whead = -1;
         s_dead = 0;
-        for (int i = 0; i < kBarsUsed; ++i) {
-            const bool many = (i >= BAR_IN_EMPTY && i < BAR_V_FULL) || i >= BAR_V_EMPTY;   // arrivals by a whole group
-            mbar_init(ro.bars + 8 * i, many ? 128u : 1u);
-        }
+        for (int i = 0; i < kBarsUsed; ++i) mbar_init(ro.bars + 8 * i, bar_count(i));
         mbar_fence_init();
     }
     if (tid < 32) tmem_alloc<512>(smem_u32(&s_tmem));
@@ -887,33 +1018,42 @@ __global__ void __launch_bounds__(NT, 1) fused2_kernel(const __grid_constant__ F
     tc_fence_after_sync();
     ro.tmem = s_tmem;
     const int G = p.plan.g_tasks, B = p.plan.b_tasks, Lg = p.plan.lag, S = p.slabs;
-    const int count0 = Lg * G, count1 = (S - Lg) * (G + B);
-    const int total = S * (G + B);
+    const int NG = (S + Lg - 1) / Lg;
+    const int total = S * (2 * G + 1 + B);
     unsigned* queue = p.counters + 3 * (size_t)S;
+    int slot = 0;
     for (;;) {
-        if (tid == 0) s_task = (int)atomicAdd(queue, 1u);
-        __syncthreads();
-        const int task = s_task;
-        __syncthreads();
-        if (task >= total) break;
-        // queue order: step i holds the G tasks of slab i (i < S) and the B tasks of slab i - lag (i >= lag)
-        int slab, sub;
-        bool is_g;
-        if (task < count0) {
-            slab = task / G; sub = task - slab * G; is_g = true;
-        } else if (task - count0 < count1) {
-            const int t = task - count0;
-            const int step = t / (G + B), r = t - step * (G + B);
-            is_g = r < G;
-            slab = is_g ? (Lg + step) : step;
-            sub = is_g ? r : (r - G);
-        } else {
-            const int t = task - count0 - count1;
-            const int step = t / B;
-            slab = S - Lg + step; sub = t - step * B; is_g = false;
+        if (tid == 0) {
+            int idx = (int)atomicAdd(queue, 1u);
+            int kind = -1, slab = 0, sub = 0;
+            if (idx < total) {
+                for (int t = 0; t < NG + 3 && kind < 0; ++t) {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {           // B, M, G, P
+                        const int g = t - 3 + k;
+                        if (kind >= 0 || g < 0 || g >= NG) continue;
+                        const int ns = min(Lg, S - g * Lg);
+                        const int per = k == 0 ? B : (k == 1 ? 1 : G);
+                        const int cnt = ns * per;
+                        if (idx < cnt) { kind = 3 - k; slab = g * Lg + idx / per; sub = idx % per; }
+                        else idx -= cnt;
+                    }
+                }
+            }
+            s_info[0] = kind; s_info[1] = slab; s_info[2] = sub;
         }
-        if (is_g) run_g_task<T, SH>(p, slab, sub, smem, ro);
-        else      run_b_task<T, SH>(p, slab, sub, smem, ro, &s_whead);
+        __syncthreads();
+        const int kind = s_info[0], slab = s_info[1], sub = s_info[2];
+        __syncthreads();
+        if (kind < 0) break;
+        if (kind == 0) run_p_task<T, SH>(p, slab, sub, smem, slot);
+        else if (kind == 1) run_g_task<T, SH>(p, slab, sub, smem, ro, slot);
+        else if (kind == 2) run_m_task<T, SH>(p, slab, ro, slot);
+        else run_b_task<T, SH>(p, slab, sub, smem, ro, &s_whead, s_red, slot);
+#ifdef AA_FUSED2_TRACE
+        if (tid == 0) { trace_put(slot, 6, (unsigned long long)(kind + 1)); trace_put(slot, 7, (unsigned long long)(slab * 64 + sub)); }
+#endif
+        ++slot;
     }
     tc_fence_before_sync();
     __syncthreads();

@@ -17,6 +17,9 @@ cudaError_t launch_fused2_s56(int dtype, const FusedArgs& a, cudaStream_t st);
 cudaError_t launch_fused2_s14(int dtype, const FusedArgs& a, cudaStream_t st);
 
 static int fused2_spec_of(int H, int W, int n_agents) {
+#ifdef AA_FUSED2_TRACE
+    return 0;                      // debug builds trace the generic kernel
+#endif
     if (H == 56 && W == 56 && n_agents == 49) return 1;
     if (H == 14 && W == 14 && n_agents == 49) return 2;
     return 0;
@@ -66,23 +69,21 @@ FusedPlan plan_fused2(int dtype, int slabs, int H, int W, int d, int n_agents, i
     if (!fused2_prepare_dt<ShapeAny>(dtype)) return pl;
     if (pl.spec == 1 && !fused2_prepare_s56(dtype)) return pl;
     if (pl.spec == 2 && !fused2_prepare_s14(dtype)) return pl;
-    const long long total = (long long)slabs * (pl.g_tasks + pl.b_tasks);
+    const long long total = (long long)slabs * (2 * pl.g_tasks + 1 + pl.b_tasks);
+    if (total > 0x3fffffffLL) return pl;
     long long grid = sm_count;                     // one block per SM: a block takes all of its tensor memory
     if (grid > total) grid = total;
     pl.grid = (int)grid;
-    if (pl.grid < pl.g_tasks) return pl;           // progress needs a resident block per G sibling
-    // The aggregation runs ahead of the broadcast by `lag` slabs: far enough that B tasks rarely wait
-    // for their slab's flag, close enough that the Q and V of the slabs in between stay in L2
-    // (budget: half of a 126 MB L2 for those re-reads).
+    // Slabs are processed in groups: pooling, aggregation, merge and broadcast of consecutive groups
+    // overlap in the queue, and a group is small enough that the Q and V of the groups in flight stay
+    // in L2 between their first and second reads (budget: half of a 126 MB L2).
     const long long slab_qv_bytes = 2LL * H * W * d * 2;
-    long long lag_l2 = (64LL << 20) / slab_qv_bytes;
-    int lag = (5 * pl.grid / 2 + pl.g_tasks + pl.b_tasks - 1) / (pl.g_tasks + pl.b_tasks) + 2;
-    if (lag_l2 > lag) lag = (int)(lag_l2 > 1000000 ? 1000000 : lag_l2);
+    long long lag = (64LL << 20) / (3 * slab_qv_bytes);
     const char* env_lag = getenv("AGENT_ATTN_FUSED2_LAG");
     if (env_lag && atoi(env_lag) > 0) lag = atoi(env_lag);
-    if (lag > slabs) lag = slabs;
+    if (3 * lag >= slabs) lag = slabs;             // everything fits: one group, phase after phase
     if (lag < 1) lag = 1;
-    pl.lag = lag;
+    pl.lag = (int)lag;
     pl.smem = kSmemBytes;
     pl.v2 = 1;
     pl.ok = true;
@@ -118,3 +119,9 @@ cudaError_t launch_fused2(int dtype, const FusedArgs& a, cudaStream_t st) {
 }
 
 }  // namespace aa
+
+#ifdef AA_FUSED2_TRACE
+extern "C" int aa_fused2_trace_buffer(void* device_buffer) {
+    return (int)cudaMemcpyToSymbol(aa::f2::g_trace2, &device_buffer, sizeof(void*));
+}
+#endif
