@@ -21,8 +21,6 @@ struct agent_attn_handle {
     int launches;
     int fused_key[3];       // (grid_h, grid_w, n_agents) that fused_plan was made for
     FusedPlan fused_plan;
-    int fused2_key[4];      // (grid_h, grid_w, n_agents, has_b1) that fused2_plan was made for
-    FusedPlan fused2_plan;
     char err[512];
 };
 
@@ -55,7 +53,7 @@ AggPlan plan_for(const agent_attn_handle* h, int n_tokens, int n_agents) {
 
 // Workspace layout: [A | V_A | partials | tickets], each region 256-byte aligned.
 struct WsLayout {
-    size_t a_off, va_off, part_off, ticket_off, pad_off, pad_bytes, total;
+    size_t a_off, va_off, part_off, ticket_off, total;
 };
 WsLayout ws_layout(const agent_attn_handle* h, int n_tokens, int n_agents, int grid_h = 0, int grid_w = 0) {
     const size_t slabs = (size_t)h->cfg.batch * h->cfg.heads;
@@ -73,11 +71,7 @@ WsLayout ws_layout(const agent_attn_handle* h, int n_tokens, int n_agents, int g
         if (part_floats < fused_floats) part_floats = fused_floats;
     }
     w.ticket_off = w.part_off + align_up(part_floats * sizeof(float), 256);
-    // three regions of 64 padded rows per slab for the role-specialised fused kernel
-    w.pad_off = w.ticket_off + align_up(fused_counter_words((int)slabs) * sizeof(unsigned), 256);
-    w.pad_bytes = (grid_h > 0 && h->cfg.path == AA_PATH_AUTO && h->cfg.dtype != AA_F32 && n_agents <= 64)
-                      ? align_up(fused2_pad_bytes((int)slabs, h->cfg.head_dim), 256) : 0;
-    w.total = w.pad_off + 3 * w.pad_bytes;
+    w.total = w.ticket_off + align_up(fused_counter_words((int)slabs) * sizeof(unsigned), 256);
     return w;
 }
 
@@ -311,31 +305,6 @@ int agent_attn_forward(agent_attn_handle* h, const void* Q, const void* K, const
             h->fused_plan = plan_fused(h->cfg.dtype, h->cfg.batch * h->cfg.heads, grid_h, grid_w, h->cfg.head_dim,
                                        n_agents, h->sm_count);
             h->fused_key[0] = grid_h; h->fused_key[1] = grid_w; h->fused_key[2] = n_agents;
-        }
-        if (h->fused2_key[0] != grid_h || h->fused2_key[1] != grid_w || h->fused2_key[2] != n_agents ||
-            h->fused2_key[3] != (b1 ? 1 : 0)) {
-            h->fused2_plan = plan_fused2(h->cfg.dtype, h->cfg.batch * h->cfg.heads, grid_h, grid_w, h->cfg.head_dim,
-                                         n_agents, h->sm_count, b1 != nullptr);
-            h->fused2_key[0] = grid_h; h->fused2_key[1] = grid_w; h->fused2_key[2] = n_agents; h->fused2_key[3] = b1 ? 1 : 0;
-        }
-        if (h->fused2_plan.ok && w.pad_bytes) {
-            const int slabs = h->cfg.batch * h->cfg.heads;
-            unsigned* counters = reinterpret_cast<unsigned*>(ws + w.ticket_off);
-            cudaError_t e = cudaMemsetAsync(counters, 0, fused_counter_words(slabs) * sizeof(unsigned), st);
-            if (e != cudaSuccess) return fail(h, AA_ERR_CUDA, "counter reset failed: %s", cudaGetErrorString(e));
-            FusedArgs fa;
-            memset(&fa, 0, sizeof(fa));
-            fa.q = Q; fa.k = K; fa.v = V; fa.b1 = b1; fa.b2 = b2; fa.dwc_w = dwc_weight; fa.out = out;
-            fa.ag_ws = ws + w.pad_off; fa.ab_ws = ws + w.pad_off + w.pad_bytes; fa.va2_ws = ws + w.pad_off + 2 * w.pad_bytes;
-            fa.partials = reinterpret_cast<float*>(ws + w.part_off);
-            fa.counters = counters; fa.status = h->d_status;
-            fa.slabs = slabs; fa.heads = h->cfg.heads; fa.H = grid_h; fa.W = grid_w; fa.d = h->cfg.head_dim;
-            fa.n = n_agents; fa.p = p; fa.scale1 = h->scale1; fa.scale2 = h->scale2; fa.plan = h->fused2_plan;
-            if (!fused2_make_maps(&fa)) return fail(h, AA_ERR_CUDA, "tensor map encoding failed");
-            e = launch_fused2(h->cfg.dtype, fa, st);
-            if (e != cudaSuccess) return fail(h, AA_ERR_CUDA, "fused launch failed: %s", cudaGetErrorString(e));
-            h->launches = 1;
-            return AA_OK;
         }
         if (h->fused_plan.ok) {
             const int slabs = h->cfg.batch * h->cfg.heads;

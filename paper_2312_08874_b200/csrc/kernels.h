@@ -86,9 +86,6 @@ struct FusedPlan {
     int parts;          // partial states per slab
     int spec;           // 0 = generic kernel, else index of a kernel specialised for this shape
     size_t smem;        // dynamic shared memory per block
-    int v2;             // role-specialised kernel (fused2_kernel.cuh): b_tasks counts runs of tb tiles
-    int tb;             // v2: broadcast tiles per B task
-    int b_tiles;        // v2: broadcast tiles per slab
 };
 struct FusedArgs {
     const void *q, *k, *v, *b1, *b2, *dwc_w;
@@ -106,21 +103,11 @@ struct FusedArgs {
     int b1_tma;           // B1 tiles come through TMA (needs N % 8 == 0 and 8-aligned task ranges)
     alignas(64) CUtensorMap tm_k, tm_v, tm_b1, tm_a, tm_va;
     alignas(64) CUtensorMap tm_q;     // Q as [slabs*N][d] with 128-row boxes (A operand of the broadcast MMA)
-    // role-specialised kernel: agents and features padded to 64 rows per slab (rows >= n zero)
-    void* ag_ws;          // [slabs][64][d]  scale1 * A
-    void* ab_ws;          // [slabs][64][d]  A
-    void* va2_ws;         // [slabs][64][d]  V_A
-    alignas(64) CUtensorMap tm_ag, tm_ab, tm_va2;     // [slabs*64][d] with 64-row boxes
 };
 FusedPlan plan_fused(int dtype, int slabs, int H, int W, int d, int n_agents, int sm_count);
 bool fused_make_maps(FusedArgs* a);     // encode the tensor maps from a's pointers and shape
 cudaError_t launch_fused(int dtype, const FusedArgs& a, cudaStream_t st);
 int fused_parts_per_slab(int dtype, int H, int W, int d, int n_agents);   // 0 if the shape is not eligible
 inline size_t fused_counter_words(int slabs) { return 3 * (size_t)slabs + 4; }
-// role-specialised kernel
-FusedPlan plan_fused2(int dtype, int slabs, int H, int W, int d, int n_agents, int sm_count, bool has_b1);
-bool fused2_make_maps(FusedArgs* a);
-cudaError_t launch_fused2(int dtype, const FusedArgs& a, cudaStream_t st);
-inline size_t fused2_pad_bytes(int slabs, int d) { return (size_t)slabs * 64 * d * 2; }   // one padded region
 
 }  // namespace aa
