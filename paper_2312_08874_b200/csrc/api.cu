@@ -45,8 +45,17 @@ bool use_simt(const agent_attn_handle* h) {
     return h->cfg.dtype == AA_F32 || h->cfg.path == AA_PATH_SIMT;
 }
 
+// Large agent counts go to the tensor-memory kernel (the shape rule does not depend on the bias, so
+// that the workspace size is the same with and without one).
+bool use_umma(const agent_attn_handle* h, int n_tokens, int n_agents) {
+    return !use_simt(h) && h->cfg.path == AA_PATH_AUTO &&
+           aggregate_umma_eligible(h->cfg.dtype, n_agents, n_tokens, h->cfg.head_dim, true);
+}
+
 AggPlan plan_for(const agent_attn_handle* h, int n_tokens, int n_agents) {
     const int slabs = h->cfg.batch * h->cfg.heads;
+    if (use_umma(h, n_tokens, n_agents))
+        return plan_aggregate_umma(slabs, n_agents, n_tokens, h->cfg.head_dim, h->sm_count);
     return use_simt(h) ? plan_aggregate_simt(slabs, n_agents, n_tokens, h->cfg.head_dim, h->sm_count)
                        : plan_aggregate_mma(slabs, n_agents, n_tokens, h->cfg.head_dim, h->sm_count);
 }
@@ -113,8 +122,10 @@ int do_aggregate(agent_attn_handle* h, const void* A, const void* K, const void*
     a.slabs = h->cfg.batch * h->cfg.heads; a.heads = h->cfg.heads;
     a.rows = n; a.cols = N; a.d = h->cfg.head_dim;
     a.scale = h->scale1; a.splits = pl.splits;
-    e = use_simt(h) ? launch_aggregate_simt(h->cfg.dtype, a, pl, st)
-                    : launch_aggregate_mma(h->cfg.dtype, a, pl, st);
+    a.status = h->d_status;
+    e = use_umma(h, N, n) ? launch_aggregate_umma(h->cfg.dtype, a, pl, st)
+        : use_simt(h)     ? launch_aggregate_simt(h->cfg.dtype, a, pl, st)
+                          : launch_aggregate_mma(h->cfg.dtype, a, pl, st);
     if (e != cudaSuccess) return fail(h, AA_ERR_CUDA, "aggregation launch failed: %s", cudaGetErrorString(e));
     h->launches++;
     return AA_OK;

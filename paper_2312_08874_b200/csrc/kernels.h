@@ -51,6 +51,7 @@ struct AttnArgs {
     const void* dwc_v;    // broadcast only: V [slabs][H*W][d] or nullptr
     const void* dwc_w;    // broadcast only: [heads][d][3][3] or nullptr
     int H, W;             // broadcast only: token grid
+    int* status;          // device status word for bounded waits (tensor-memory kernels), may be null
 };
 
 // Plan of the aggregation launch for a problem shape (used for workspace sizing too).
@@ -69,6 +70,10 @@ cudaError_t launch_aggregate_simt(int dtype, const AttnArgs& p, const AggPlan& p
 cudaError_t launch_broadcast_simt(int dtype, const AttnArgs& p, cudaStream_t st);
 cudaError_t launch_aggregate_mma(int dtype, const AttnArgs& p, const AggPlan& plan, cudaStream_t st);
 cudaError_t launch_broadcast_mma(int dtype, const AttnArgs& p, cudaStream_t st);
+// tensor-memory (tcgen05) kernels for large agent counts (aggregate_umma.cu)
+bool aggregate_umma_eligible(int dtype, int n_agents, int n_tokens, int d, bool has_bias);
+AggPlan plan_aggregate_umma(int slabs, int n_agents, int n_tokens, int d, int sm_count);
+cudaError_t launch_aggregate_umma(int dtype, const AttnArgs& p, const AggPlan& plan, cudaStream_t st);
 
 // Whole module (Eq. 6) in one persistent kernel for small agent counts (n <= 64, d = 64,
 // block pooling, W <= 64).  Blocks take tasks from a device-side queue: "G" tasks pool their token
