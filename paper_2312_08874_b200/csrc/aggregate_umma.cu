@@ -14,7 +14,8 @@
 //                        A row's reference maximum moves only when exceeded by a margin; then the thread
 //                        rescales its accumulator row in tensor memory.
 // At the end the two token halves of a row meet in shared memory and the block writes one partial state;
-// the last block of the slab merges all partials in a fixed order (merge.cuh).
+// a second small kernel merges the slab's partials in a fixed order, spread over many blocks (a merge by
+// the slab's last block alone took longer than the streaming part).
 // Every wait is bounded (pipe.cuh).  No TMA multicast, no clusters.
 #include "common.cuh"
 #include "kernels.h"
@@ -66,7 +67,7 @@ struct UmmaAggArgs {
 template <typename T>
 __global__ void __launch_bounds__(NT, 1) aggregate_umma_kernel(const __grid_constant__ UmmaAggArgs g) {
     extern __shared__ unsigned char smem_raw[];
-    __shared__ int s_flag, s_dead;
+    __shared__ int s_dead;
     __shared__ uint32_t s_tmem;
     unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     constexpr int fmt = Elem<T>::kIsBf16 ? 1 : 0;
@@ -74,7 +75,7 @@ __global__ void __launch_bounds__(NT, 1) aggregate_umma_kernel(const __grid_cons
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int split = blockIdx.x, slab = blockIdx.y;
     const int head = slab % p.heads;
-    const int n = p.rows, N = p.cols, d = p.d;
+    const int n = p.rows, N = p.cols;
     const int MB = g.rows_pad >> 7;                       // 128-row agent blocks
     const bool has_bias = p.bias != nullptr;
     const int tiles_all = (N + KT - 1) / KT;
@@ -303,12 +304,44 @@ __global__ void __launch_bounds__(NT, 1) aggregate_umma_kernel(const __grid_cons
             }
         }
     }
-    const bool last = arrive_is_last(p.tickets + slab, gridDim.x, &s_flag);
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 0) tmem_dealloc<512>(pp.tmem);
-    if (last)
-        merge_partials<T>(slab_parts, (int)gridDim.x, g.rows_pad, 64, n, d, static_cast<T*>(p.out) + (size_t)slab * n * d);
+}
+
+// Merge of the slab's partial states into V_A, spread over many blocks: grid (row chunks, slabs), a
+// thread per (agent row, four channels), the parts in their fixed order (bit-reproducible).
+template <typename T>
+__global__ void __launch_bounds__(256) merge_umma_kernel(const float* __restrict__ partials, int parts, int rows_pad,
+                                                         int n, int d, T* __restrict__ out) {
+    const int slab = blockIdx.y;
+    const size_t pf = partial_floats(rows_pad, 64);
+    const float* base = partials + (size_t)slab * parts * pf;
+    const int groups = d >> 2;                             // d is a multiple of 8
+    const int rows_per_block = 256 / 16;
+    const int r = blockIdx.x * rows_per_block + (threadIdx.x >> 4), cg = threadIdx.x & 15;
+    if (r >= n || cg >= groups) return;
+    float mx = -INFINITY, den = 0.f;
+    float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
+    for (int q = 0; q < parts; ++q) {
+        const float* pq = base + q * pf;
+        const float mq = __ldcg(pq + r);
+        const float lq = __ldcg(pq + rows_pad + r);
+        const float4 a = __ldcg(reinterpret_cast<const float4*>(pq + 2 * (size_t)rows_pad + (size_t)r * 64 + 4 * cg));
+        const float mn = fmaxf(mx, mq);
+        const float bs = (mn == -INFINITY) ? 0.f : mn;
+        const float c0 = exp2f(mx - bs), c1 = exp2f(mq - bs);
+        den = den * c0 + lq * c1;
+        num.x = num.x * c0 + a.x * c1; num.y = num.y * c0 + a.y * c1;
+        num.z = num.z * c0 + a.z * c1; num.w = num.w * c0 + a.w * c1;
+        mx = mn;
+    }
+    const float inv = 1.f / den;
+    uint2 o;
+    o.x = pack2<T>(num.x * inv, num.y * inv);
+    o.y = pack2<T>(num.z * inv, num.w * inv);
+    *reinterpret_cast<uint2*>(out + ((size_t)slab * n + r) * d + 4 * cg) = o;
 }
 
 // ------------------------------------------------------------------------------------- host
@@ -344,6 +377,10 @@ static cudaError_t launch_umma_t(const UmmaAggArgs& g, cudaStream_t st) {
     if (e != cudaSuccess) return e;
     dim3 grid(g.a.splits, g.a.slabs);
     kern<<<grid, NT, kSmemBytes, st>>>(g);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    dim3 mgrid((g.a.rows + 15) / 16, g.a.slabs);
+    merge_umma_kernel<T><<<mgrid, 256, 0, st>>>(g.a.partials, g.a.splits, g.rows_pad, g.a.rows, g.a.d, static_cast<T*>(g.a.out));
     return cudaGetLastError();
 }
 

@@ -127,7 +127,7 @@ int do_aggregate(agent_attn_handle* h, const void* A, const void* K, const void*
         : use_simt(h)     ? launch_aggregate_simt(h->cfg.dtype, a, pl, st)
                           : launch_aggregate_mma(h->cfg.dtype, a, pl, st);
     if (e != cudaSuccess) return fail(h, AA_ERR_CUDA, "aggregation launch failed: %s", cudaGetErrorString(e));
-    h->launches++;
+    h->launches += use_umma(h, N, n) ? 2 : 1;      // the tensor-memory path merges in a second kernel
     return AA_OK;
 }
 
@@ -140,8 +140,12 @@ int do_broadcast(agent_attn_handle* h, const void* Q, const void* A, const void*
     a.rows = gh * gw; a.cols = n; a.d = h->cfg.head_dim;
     a.scale = h->scale2; a.splits = 1;
     a.dwc_v = wd ? V : nullptr; a.dwc_w = wd; a.H = gh; a.W = gw;
-    cudaError_t e = use_simt(h) ? launch_broadcast_simt(h->cfg.dtype, a, st)
-                                : launch_broadcast_mma(h->cfg.dtype, a, st);
+    a.status = h->d_status;
+    const bool umma = !use_simt(h) && h->cfg.path == AA_PATH_AUTO &&
+                      broadcast_umma_eligible(h->cfg.dtype, n, gh * gw, h->cfg.head_dim);
+    cudaError_t e = umma          ? launch_broadcast_umma(h->cfg.dtype, a, h->sm_count, st)
+                    : use_simt(h) ? launch_broadcast_simt(h->cfg.dtype, a, st)
+                                  : launch_broadcast_mma(h->cfg.dtype, a, st);
     if (e != cudaSuccess) return fail(h, AA_ERR_CUDA, "broadcast launch failed: %s", cudaGetErrorString(e));
     h->launches++;
     return AA_OK;

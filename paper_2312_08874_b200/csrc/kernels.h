@@ -74,6 +74,8 @@ cudaError_t launch_broadcast_mma(int dtype, const AttnArgs& p, cudaStream_t st);
 bool aggregate_umma_eligible(int dtype, int n_agents, int n_tokens, int d, bool has_bias);
 AggPlan plan_aggregate_umma(int slabs, int n_agents, int n_tokens, int d, int sm_count);
 cudaError_t launch_aggregate_umma(int dtype, const AttnArgs& p, const AggPlan& plan, cudaStream_t st);
+bool broadcast_umma_eligible(int dtype, int n_agents, int n_tokens, int d);
+cudaError_t launch_broadcast_umma(int dtype, const AttnArgs& p, int sm_count, cudaStream_t st);
 
 // Whole module (Eq. 6) in one persistent kernel for small agent counts (n <= 64, d = 64,
 // block pooling, W <= 64).  Blocks take tasks from a device-side queue: "G" tasks pool their token
