@@ -298,29 +298,39 @@ __global__ void __launch_bounds__(NT, 1) broadcast_umma_kernel(const __grid_cons
                 pipe_arrive(pp, BAR_P_FULL);
             }
             // depthwise 3x3 term for this thread's 16 channels of its token, while the last product is in flight
-            float dw[16];
+            float2 dw[8];
 #pragma unroll
-            for (int k = 0; k < 16; ++k) dw[k] = 0.f;
-            if (has_dwc && tok < N && nch > 0) {
-                const int y = tok / W, x = tok - y * W;
+            for (int k = 0; k < 8; ++k) dw[k] = make_float2(0.f, 0.f);
+            if (has_dwc) {
+                // all taps of a grid row are fetched before they are used (loads outside the grid or past the
+                // head dim become zeros, from a clamped address), so the L2 latency is paid once per row
+                const int tk = min(tok, N - 1);
+                const int y = tk / W, x = tk - y * W;
+                const bool live = tok < N && nch > 0;
 #pragma unroll
                 for (int u = 0; u < 3; ++u) {
                     const int yy = y + u - 1;
-                    if (yy < 0 || yy >= H) continue;
+                    const bool rowok = live && yy >= 0 && yy < H;
+                    uint4 raw[3][2];
 #pragma unroll
                     for (int v = 0; v < 3; ++v) {
                         const int xx = x + v - 1;
-                        if (xx < 0 || xx >= W) continue;
-                        const T* src = gV + ((size_t)yy * W + xx) * d + c0;
-                        const float* wt = sW + (u * 3 + v) * 64 + c0;
-                        float f[8];
-                        unpack16<T>(__ldg(reinterpret_cast<const uint4*>(src)), f);
+                        const bool ok = rowok && xx >= 0 && xx < W;
+                        const uint4* src = reinterpret_cast<const uint4*>(gV + (ok ? ((size_t)yy * W + xx) * d + c0 : (size_t)0));
+                        raw[v][0] = ok ? __ldg(src) : make_uint4(0u, 0u, 0u, 0u);
+                        raw[v][1] = (ok && nch > 8) ? __ldg(src + 1) : make_uint4(0u, 0u, 0u, 0u);
+                    }
 #pragma unroll
-                        for (int k = 0; k < 8; ++k) dw[k] = fmaf(wt[k], f[k], dw[k]);
-                        if (nch > 8) {
-                            unpack16<T>(__ldg(reinterpret_cast<const uint4*>(src) + 1), f);
+                    for (int v = 0; v < 3; ++v) {
+                        const float4* wt = reinterpret_cast<const float4*>(sW + (u * 3 + v) * 64 + c0);
 #pragma unroll
-                            for (int k = 0; k < 8; ++k) dw[8 + k] = fmaf(wt[8 + k], f[k], dw[8 + k]);
+                        for (int hh = 0; hh < 2; ++hh) {
+                            const float4 w0 = wt[2 * hh], w1 = wt[2 * hh + 1];
+                            const uint4 r = raw[v][hh];
+                            dw[4 * hh + 0] = ffma2(make_float2(w0.x, w0.y), unpack2<T>(r.x), dw[4 * hh + 0]);
+                            dw[4 * hh + 1] = ffma2(make_float2(w0.z, w0.w), unpack2<T>(r.y), dw[4 * hh + 1]);
+                            dw[4 * hh + 2] = ffma2(make_float2(w1.x, w1.y), unpack2<T>(r.z), dw[4 * hh + 2]);
+                            dw[4 * hh + 3] = ffma2(make_float2(w1.z, w1.w), unpack2<T>(r.w), dw[4 * hh + 3]);
                         }
                     }
                 }
@@ -358,11 +368,11 @@ __global__ void __launch_bounds__(NT, 1) broadcast_umma_kernel(const __grid_cons
                 if (tok < N && nch > 0) {
                     float o8[8];
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) o8[k] = fmaf(acc[k], inv, dw[k]);
+                    for (int k = 0; k < 8; ++k) o8[k] = fmaf(acc[k], inv, (k & 1) ? dw[k >> 1].y : dw[k >> 1].x);
                     *reinterpret_cast<uint4*>(gO + (size_t)tok * d + c0) = pack16<T>(o8);
                     if (nch > 8) {
 #pragma unroll
-                        for (int k = 0; k < 8; ++k) o8[k] = fmaf(acc[8 + k], inv, dw[8 + k]);
+                        for (int k = 0; k < 8; ++k) o8[k] = fmaf(acc[8 + k], inv, (k & 1) ? dw[4 + (k >> 1)].y : dw[4 + (k >> 1)].x);
                         *(reinterpret_cast<uint4*>(gO + (size_t)tok * d + c0) + 1) = pack16<T>(o8);
                     }
                 }
