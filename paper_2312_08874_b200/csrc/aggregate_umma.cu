@@ -1,12 +1,13 @@
 // Agent aggregation V_A = softmax(scale1 * A K^T + B1) V (Eq. 3, Eq. 5) for large agent counts
 // (64 < n <= 256, d <= 64, 16-bit elements) on the 5th-generation tensor cores.
 //
-// Grid: (splits, slabs), one block of 18 warps per SM.  A block keeps the slab's agents resident (up to
+// Grid: (splits, slabs), one block of 19 warps per SM.  A block keeps the slab's agents resident (up to
 // two 128-row operand blocks) and streams its share of the slab's 64-token tiles (K, V and the matching
 // B1 columns) through a three-stage TMA ring.
 //   warp 16 "producer":  one lane issues every TMA copy, ahead of the others through full/empty mbarriers.
 //   warp 17 "MMA issuer": one lane issues S = A K^T (tcgen05.mma, accumulator in tensor memory) one tile
-//                        ahead, and the products P V once the probabilities of a tile are written.
+//                        ahead; warp 18 issues the products P V once the probabilities of a tile are written
+//                        (two issuing threads, so that neither instruction stream delays the other).
 //   warps 0-15 "row warps": thread (agent row, token half): reads its 32 logits of the tile from tensor
 //                        memory, adds scale and bias, keeps its own running maximum / sum (no reduction
 //                        crosses threads: each token half has its own accumulator in tensor memory),
@@ -29,7 +30,7 @@ namespace aa {
 namespace {
 constexpr int KT = 64;                 // tokens per tile
 constexpr int NROW = 512;              // row-warp threads
-constexpr int NT = NROW + 64;          // + producer warp + MMA issuer warp
+constexpr int NT = NROW + 96;          // + producer warp + two MMA issuer warps (logits, products)
 constexpr int STAGES = 3;
 constexpr int kTile = 64 * 128;        // swizzled [64][64] tile of 16-bit elements
 constexpr float kTau = 5.5f;           // margin (natural units) before a row's reference maximum moves
@@ -124,48 +125,56 @@ __global__ void __launch_bounds__(NT, 1) aggregate_umma_kernel(const __grid_cons
         }
         __syncwarp();
     } else if (warp == 17) {
-        // ------------------------------------------------------------------ MMA issuer
+        // ------------------------------------------------------------------ MMA issuer: logits, one tile ahead
         if (lane == 0) {
-            const uint32_t idK = umma_idesc(fmt, 128, 64, 0), idMN = umma_idesc(fmt, 128, 64, 1);
-            const uint64_t dA = umma_desc_sw128(sA), dP = umma_desc_sw128(sP), dRing = umma_desc_sw128(ring);
+            const uint32_t idK = umma_idesc(fmt, 128, 64, 0);
+            const uint64_t dA = umma_desc_sw128(sA), dRing = umma_desc_sw128(ring);
             // descriptor start addresses count 16-byte units: + 2 per K-step of a K-major operand (32 bytes),
-            // + 128 per K-step of an MN-major operand (16 rows of 128 bytes), + 1024 per 128-row block
-            auto issue_S = [&](int t) {
+            // + 1024 per 128-row block
+            pipe_wait_one(pp, BAR_AG, kTimeoutLoads);
+            for (int t = 0; t < tiles; ++t) {
                 const int b = t & 1, s = t % STAGES;
                 if (t >= 2) pipe_wait_one(pp, BAR_S_EMPTY + b, kTimeoutRole);
                 pipe_wait_one(pp, BAR_FULL + s, kTimeoutTile);
                 tc_fence_after_sync();
                 const uint64_t dK = dRing + (uint64_t)(s * (kStage >> 4));
                 for (int mb = 0; mb < MB; ++mb) {
-#pragma unroll
-                    for (int kk = 0; kk < 4; ++kk)
-                        umma_f16(pp.tmem + TM_S + 128 * b + 64 * mb, dA + 1024 * mb + 2 * kk, dK + 2 * kk, idK, kk > 0);
+                    const uint32_t dd = pp.tmem + TM_S + 128 * b + 64 * mb;
+                    const uint64_t da = dA + 1024 * mb;
+                    umma_f16_c<0>(dd, da, dK, idK);
+                    umma_f16_c<1>(dd, da + 2, dK + 2, idK);
+                    umma_f16_c<1>(dd, da + 4, dK + 4, idK);
+                    umma_f16_c<1>(dd, da + 6, dK + 6, idK);
                 }
                 umma_commit(pipe_bar(pp, BAR_S_FULL + b));
-            };
-            pipe_wait_one(pp, BAR_AG, kTimeoutLoads);
-            issue_S(0);
+            }
+            for (int t = max(0, tiles - 2); t < tiles; ++t) pipe_wait_one(pp, BAR_S_EMPTY + (t & 1), kTimeoutRole);
+        }
+        __syncwarp();
+    } else if (warp == 18) {
+        // ------------------------------------------------------------------ MMA issuer: products P V
+        if (lane == 0) {
+            const uint32_t idMN = umma_idesc(fmt, 128, 64, 1);
+            const uint64_t dP = umma_desc_sw128(sP), dRing = umma_desc_sw128(ring);
+            // + 128 per K-step of an MN-major operand (16 rows of 128 bytes)
             for (int t = 0; t < tiles; ++t) {
-                if (t + 1 < tiles) issue_S(t + 1);
+                const int s = t % STAGES;
+                pipe_wait_one(pp, BAR_FULL + s, kTimeoutTile);          // long done: the logits of the tile used this stage
                 pipe_wait_one(pp, BAR_P_FULL, kTimeoutRole);
                 tc_fence_after_sync();
-                const int s = t % STAGES;
                 const int ntok = min(KT, N - (t0 + t) * KT);
                 const uint64_t dV = dRing + (uint64_t)(s * (kStage >> 4)) + (uint64_t)(kTile >> 4);
                 for (int mb = 0; mb < MB; ++mb)
                     for (int c = 0; c < 2; ++c) {
                         if (32 * c >= ntok) break;
-#pragma unroll
-                        for (int k2 = 0; k2 < 2; ++k2) {
-                            const int kk = 2 * c + k2;
-                            umma_f16(pp.tmem + TM_O + 64 * (2 * mb + c), dP + 1024 * mb + 2 * kk, dV + 128 * kk, idMN,
-                                     (t > 0 || k2 > 0) ? 1u : 0u);
-                        }
+                        const uint32_t dd = pp.tmem + TM_O + 64 * (2 * mb + c);
+                        const uint64_t da = dP + 1024 * mb + 4 * c, db = dV + 256 * c;
+                        if (t > 0) umma_f16_c<1>(dd, da, db, idMN); else umma_f16_c<0>(dd, da, db, idMN);
+                        umma_f16_c<1>(dd, da + 2, db + 128, idMN);
                     }
                 umma_commit(pipe_bar(pp, BAR_EMPTY + s));
                 umma_commit(pipe_bar(pp, BAR_PV));
             }
-            for (int t = max(0, tiles - 2); t < tiles; ++t) pipe_wait_one(pp, BAR_S_EMPTY + (t & 1), kTimeoutRole);
         }
         __syncwarp();
     } else if ((warp >> 2 & 1) < MB) {
@@ -186,20 +195,21 @@ __global__ void __launch_bounds__(NT, 1) aggregate_umma_kernel(const __grid_cons
                 uint32_t ra[32];
                 tmem_ld32(pp.tmem + TM_S + 128 * b + 64 * mb + 32 * c + lane_base, ra);
                 tmem_ld_wait();
+                tc_fence_before_sync();
+                pipe_arrive(pp, BAR_S_EMPTY + b);
+                if (has_bias) {                              // logits in natural units: scale1 * a.k + b1
+                    const unsigned char* sB = smem + OFF_RING + s * kStage + 2 * kTile + row * 128;
 #pragma unroll
-                for (int k = 0; k < 32; ++k) sv[k] = __uint_as_float(ra[k]) * p.scale;
-            }
-            tc_fence_before_sync();
-            pipe_arrive(pp, BAR_S_EMPTY + b);
-            if (has_bias) {
-                const unsigned char* sB = smem + OFF_RING + s * kStage + 2 * kTile + row * 128;
+                    for (int j = 0; j < 4; ++j) {
+                        const uint4 raw = *reinterpret_cast<const uint4*>(sB + (((4 * c + j) ^ (row & 7)) << 4));
+                        float f[8];
+                        unpack16<T>(raw, f);
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const uint4 raw = *reinterpret_cast<const uint4*>(sB + (((4 * c + j) ^ (row & 7)) << 4));
-                    float f[8];
-                    unpack16<T>(raw, f);
+                        for (int k = 0; k < 8; ++k) sv[8 * j + k] = fmaf(__uint_as_float(ra[8 * j + k]), p.scale, f[k]);
+                    }
+                } else {
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) sv[8 * j + k] += f[k];
+                    for (int k = 0; k < 32; ++k) sv[k] = __uint_as_float(ra[k]) * p.scale;
                 }
             }
             uint32_t pk[16];
@@ -323,7 +333,7 @@ __global__ void __launch_bounds__(256) merge_umma_kernel(const float* __restrict
     if (r >= n || cg >= groups) return;
     float mx = -INFINITY, den = 0.f;
     float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 4
+#pragma unroll 16
     for (int q = 0; q < parts; ++q) {
         const float* pq = base + q * pf;
         const float mq = __ldcg(pq + r);

@@ -1,12 +1,13 @@
 // Agent broadcast O = softmax(scale2 * Q A^T + B2) V_A + DWC(V) (Eq. 3, Eq. 5, Eq. 6) for large agent
 // counts (64 < n <= 256, d <= 64, 16-bit elements) on the 5th-generation tensor cores.
 //
-// Grid: (splits, slabs), one block of 18 warps per SM.  The slab's agents A and agent features V_A stay
+// Grid: (splits, slabs), one block of 19 warps per SM.  The slab's agents A and agent features V_A stay
 // resident in shared memory; a block walks its share of the slab's 128-token tiles.  Per tile the agents
 // are taken in blocks of 128 ("steps"): S = Q A_block^T by tcgen05.mma into tensor memory, one step ahead.
 //   warp 16 "producer":   one lane issues every TMA copy (Q tiles, B2 tiles) through full/empty mbarriers.
-//   warp 17 "MMA issuer": one lane issues the logits and, once the probabilities of a step are written,
-//                         the products P V_A.
+//   warp 17 "MMA issuer": one lane issues the logits; warp 18 issues the products P V_A once the
+//                         probabilities of a step are written (two issuing threads, so that neither
+//                         instruction stream delays the other).
 //   warps 0-15 "row warps": thread (query row, agent group g of 32 columns per step): online softmax over
 //                         the steps with its own running maximum, sum and accumulator O_g in tensor memory
 //                         (no reduction crosses threads inside the loop).  At the end of a tile the four
@@ -25,7 +26,7 @@ namespace aa {
 namespace {
 constexpr int QT = 128;                // query rows per tile
 constexpr int NROW = 512;              // row-warp threads
-constexpr int NT = NROW + 64;          // + producer warp + MMA issuer warp
+constexpr int NT = NROW + 96;          // + producer warp + two MMA issuer warps (logits, products)
 constexpr int kTile = 64 * 128;        // swizzled [64][64] tile of 16-bit elements
 constexpr float kTau = 5.5f;
 constexpr int kTimeoutTile = 3, kTimeoutLoads = 4, kTimeoutRole = 6;
@@ -136,48 +137,58 @@ __global__ void __launch_bounds__(NT, 1) broadcast_umma_kernel(const __grid_cons
         }
         __syncwarp();
     } else if (warp == 17) {
-        // ------------------------------------------------------------------ MMA issuer
+        // ------------------------------------------------------------------ MMA issuer: logits, one step ahead
         if (lane == 0) {
-            const uint32_t idS = umma_idesc(fmt, 128, 128, 0), idMN = umma_idesc(fmt, 128, 64, 1);
-            const uint64_t dA = umma_desc_sw128(sA), dVA = umma_desc_sw128(sVA), dP = umma_desc_sw128(sP), dQ = umma_desc_sw128(sQ);
+            const uint32_t idS = umma_idesc(fmt, 128, 128, 0);
+            const uint64_t dA = umma_desc_sw128(sA), dQ = umma_desc_sw128(sQ);
             // descriptor start addresses count 16-byte units: + 2 per K-step of a K-major operand (32 bytes),
-            // + 128 per K-step of an MN-major operand (16 rows of 128 bytes), + 1024 per 16 KB
-            auto issue_S = [&](int j) {
+            // + 1024 per 16 KB
+            pipe_wait_one(pp, BAR_PREP, kTimeoutLoads);
+            for (int j = 0; j < steps; ++j) {
                 const int i = j / MB, a = j - i * MB, b = j & 1;
                 if (j >= 2) pipe_wait_one(pp, BAR_S_EMPTY + b, kTimeoutRole);
                 if (a == 0) pipe_wait_one(pp, BAR_Q_FULL + (i & 1), kTimeoutLoads);
                 tc_fence_after_sync();
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk)
-                    umma_f16(pp.tmem + TM_S + 128 * b, dQ + 1024 * (i & 1) + 2 * kk, dA + 1024 * a + 2 * kk, idS, kk > 0);
+                const uint32_t dd = pp.tmem + TM_S + 128 * b;
+                const uint64_t da = dQ + 1024 * (i & 1), db = dA + 1024 * a;
+                umma_f16_c<0>(dd, da, db, idS);
+                umma_f16_c<1>(dd, da + 2, db + 2, idS);
+                umma_f16_c<1>(dd, da + 4, db + 4, idS);
+                umma_f16_c<1>(dd, da + 6, db + 6, idS);
                 if (a == MB - 1) umma_commit(pipe_bar(pp, BAR_Q_EMPTY + (i & 1)));
                 umma_commit(pipe_bar(pp, BAR_S_FULL + b));
-            };
+            }
+            for (int j = max(0, steps - 2); j < steps; ++j) pipe_wait_one(pp, BAR_S_EMPTY + (j & 1), kTimeoutRole);
+        }
+        __syncwarp();
+    } else if (warp == 18) {
+        // ------------------------------------------------------------------ MMA issuer: products P V_A
+        if (lane == 0) {
+            const uint32_t idMN = umma_idesc(fmt, 128, 64, 1);
+            const uint64_t dVA = umma_desc_sw128(sVA), dP = umma_desc_sw128(sP);
+            // + 128 per K-step of an MN-major operand (16 rows of 128 bytes)
             pipe_wait_one(pp, BAR_PREP, kTimeoutLoads);
-            issue_S(0);
             unsigned started = 0u;
             for (int j = 0; j < steps; ++j) {
-                if (j + 1 < steps) issue_S(j + 1);
                 const int a = j % MB;
                 if (a == 0) started = 0u;
                 pipe_wait_one(pp, BAR_P_FULL, kTimeoutRole);
                 tc_fence_after_sync();
                 for (int gq = 0; gq < 4; ++gq) {
                     if (128 * a + 32 * gq >= n) break;
-#pragma unroll
-                    for (int k2 = 0; k2 < 2; ++k2)
-                        umma_f16(pp.tmem + TM_O + 64 * gq, dP + 1024 * (gq >> 1) + 2 * ((gq & 1) * 2 + k2),
-                                 dVA + 128 * (8 * a + 2 * gq + k2), idMN, (((started >> gq) & 1u) || k2 > 0) ? 1u : 0u);
+                    const uint32_t dd = pp.tmem + TM_O + 64 * gq;
+                    const uint64_t da = dP + 1024 * (gq >> 1) + 4 * (gq & 1), db = dVA + 128 * (8 * a + 2 * gq);
+                    if ((started >> gq) & 1u) umma_f16_c<1>(dd, da, db, idMN); else umma_f16_c<0>(dd, da, db, idMN);
+                    umma_f16_c<1>(dd, da + 2, db + 128, idMN);
                     started |= 1u << gq;
                 }
                 umma_commit(pipe_bar(pp, BAR_PV));
             }
-            for (int j = max(0, steps - 2); j < steps; ++j) pipe_wait_one(pp, BAR_S_EMPTY + (j & 1), kTimeoutRole);
         }
         __syncwarp();
     } else {
         // ------------------------------------------------------------------ row warps
-        const int gq = warp >> 2;                              // agent group: 32 columns of every step
+        const int gq = (warp >> 2) & 3;                        // agent group: 32 columns of every step
         const int row = 32 * (warp & 3) + lane;                // query row of the tile = tensor-memory lane
         const uint32_t lane_base = ((uint32_t)(32 * (warp & 3))) << 16;
         const uint32_t tO = pp.tmem + TM_O + 64 * gq + lane_base;
@@ -218,23 +229,24 @@ __global__ void __launch_bounds__(NT, 1) broadcast_umma_kernel(const __grid_cons
                     uint32_t ra[32];
                     tmem_ld32(pp.tmem + TM_S + 128 * b + 32 * gq + lane_base, ra);
                     tmem_ld_wait();
+                    tc_fence_before_sync();
+                    pipe_arrive(pp, BAR_S_EMPTY + b);
+                    if (has_b2) {                            // logits in natural units: scale2 * q.a + b2
+                        pipe_wait(pp, BAR_B_FULL + b, kTimeoutLoads);
+                        const unsigned char* sB = smem + OFF_B2 + b * 4 * kTile + (gq >> 1) * 2 * kTile + row * 128;
 #pragma unroll
-                    for (int k = 0; k < 32; ++k) sv[k] = __uint_as_float(ra[k]) * p.scale;
-                }
-                tc_fence_before_sync();
-                pipe_arrive(pp, BAR_S_EMPTY + b);
-                if (has_b2) {
-                    pipe_wait(pp, BAR_B_FULL + b, kTimeoutLoads);
-                    const unsigned char* sB = smem + OFF_B2 + b * 4 * kTile + (gq >> 1) * 2 * kTile + row * 128;
+                        for (int jj = 0; jj < 4; ++jj) {
+                            const uint4 raw = *reinterpret_cast<const uint4*>(sB + (((4 * (gq & 1) + jj) ^ (row & 7)) << 4));
+                            float f[8];
+                            unpack16<T>(raw, f);
 #pragma unroll
-                    for (int jj = 0; jj < 4; ++jj) {
-                        const uint4 raw = *reinterpret_cast<const uint4*>(sB + (((4 * (gq & 1) + jj) ^ (row & 7)) << 4));
-                        float f[8];
-                        unpack16<T>(raw, f);
+                            for (int k = 0; k < 8; ++k) sv[8 * jj + k] = fmaf(__uint_as_float(ra[8 * jj + k]), p.scale, f[k]);
+                        }
+                        pipe_arrive(pp, BAR_B_EMPTY + b);
+                    } else {
 #pragma unroll
-                        for (int k = 0; k < 8; ++k) sv[8 * jj + k] += f[k];
+                        for (int k = 0; k < 32; ++k) sv[k] = __uint_as_float(ra[k]) * p.scale;
                     }
-                    pipe_arrive(pp, BAR_B_EMPTY + b);
                 }
                 uint32_t pk[16];
                 float corr = 1.f;
@@ -267,8 +279,7 @@ __global__ void __launch_bounds__(NT, 1) broadcast_umma_kernel(const __grid_cons
                         const float p3 = fast_exp2(fmaf(sv[2 * k + 3], kLog2e, nb));
                         pk[k] = pack2<T>(p0, p1);
                         pk[k + 1] = pack2<T>(p2, p3);
-                        const float2 q0 = unpack2<T>(pk[k]), q1 = unpack2<T>(pk[k + 1]);   // the normaliser sums the rounded weights
-                        sum0 += q0.x; sum1 += q0.y; sum2 += q1.x; sum3 += q1.y;
+                        sum0 += p0; sum1 += p1; sum2 += p2; sum3 += p3;
                     }
                     l += (sum0 + sum1) + (sum2 + sum3);
                     started = true;
@@ -316,7 +327,7 @@ __global__ void __launch_bounds__(NT, 1) broadcast_umma_kernel(const __grid_cons
                     for (int v = 0; v < 3; ++v) {
                         const int xx = x + v - 1;
                         const bool ok = rowok && xx >= 0 && xx < W;
-                        const uint4* src = reinterpret_cast<const uint4*>(gV + (ok ? ((size_t)yy * W + xx) * d + c0 : (size_t)0));
+                        const uint4* src = reinterpret_cast<const uint4*>(gV + (ok ? (yy * W + xx) * d + c0 : 0));
                         raw[v][0] = ok ? __ldg(src) : make_uint4(0u, 0u, 0u, 0u);
                         raw[v][1] = (ok && nch > 8) ? __ldg(src + 1) : make_uint4(0u, 0u, 0u, 0u);
                     }
