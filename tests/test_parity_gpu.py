@@ -78,6 +78,11 @@ SWEEP = [
     (7, 3, 14, 14, 64, 7, "f16", True, True),       # fused path: one G task per slab, odd-head bias misaligned
     (2, 1, 3, 3, 16, 1, "bf16", True, True),        # one agent, nine tokens
     (1, 1, 1, 1, 64, 1, "bf16", True, True),        # a single token
+    (2, 2, 36, 36, 64, 12, "bf16", True, True),     # tensor-memory kernels: n = 144 (two agent blocks, second ragged), ragged last tiles
+    (1, 2, 48, 32, 40, 16, "f16", True, True),      # tensor-memory kernels: n = 256, d = 40 zero-filled to 64, bias and DWC
+    (1, 3, 40, 40, 64, 10, "bf16", True, False),    # n = 100: one agent block on tcgen05 for the aggregation, n % 8 != 0 for the broadcast
+    (2, 1, 27, 27, 64, 9, "bf16", True, True),      # n = 81 with odd N: stays on the mma.sync kernels
+    (1, 1, 32, 32, 64, 16, "bf16", False, False),   # tensor-memory kernels without bias and DWC
 ]
 
 
