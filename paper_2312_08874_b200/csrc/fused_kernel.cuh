@@ -215,7 +215,40 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
         constexpr int tpl = 32 / cpr;
         const int cg = lane % cpr, tsub = lane / cpr;
         const float inv = 1.f / (float)cnt;
-        for (int wi = warp; wi < nwin; wi += NT / 32) {
+        // windows of at most four tokens (one load per lane): eight windows of the warp in flight at once,
+        // so that their load latencies overlap instead of adding up
+        for (int w0 = warp; cnt <= tpl && w0 < nwin; w0 += 8 * (NT / 32)) {
+            uint4 raw[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int wi = w0 + u * (NT / 32);
+                raw[u] = make_uint4(0u, 0u, 0u, 0u);
+                if (wi < nwin && tsub < cnt) {
+                    const int ay = ar0 + wi / P, ax = wi % P;
+                    const int wy = tsub / win_w, wx = tsub - wy * win_w;
+                    const size_t tok = (size_t)(ay * win_h + wy) * W + (ax * win_w + wx);
+                    raw[u] = __ldg(reinterpret_cast<const uint4*>(gQ + tok * DK) + cg);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int wi = w0 + u * (NT / 32);
+                if (wi >= nwin) break;                       // uniform over the warp
+                float acc[8];
+                unpack16<T>(raw[u], acc);
+#pragma unroll
+                for (int o = cpr; o < 32; o <<= 1) {
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) acc[k] += __shfl_xor_sync(0xffffffffu, acc[k], o);
+                }
+                if (tsub == 0) {
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) acc[k] *= inv;
+                    *(reinterpret_cast<uint4*>(gA + (size_t)((ar0 + wi / P) * P + wi % P) * DK) + cg) = pack16<T>(acc);
+                }
+            }
+        }
+        for (int wi = warp; cnt > tpl && wi < nwin; wi += NT / 32) {
             const int ay = ar0 + wi / P, ax = wi % P;
             const int y0 = ay * win_h, x0 = ax * win_w;
             float acc[8];
