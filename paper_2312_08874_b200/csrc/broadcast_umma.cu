@@ -12,8 +12,11 @@
 //                         the steps with its own running maximum, sum and accumulator O_g in tensor memory
 //                         (no reduction crosses threads inside the loop).  At the end of a tile the four
 //                         groups of a row exchange (max, sum), every thread combines 16 output channels from
-//                         the four accumulators, adds the depthwise 3x3 term that it computed from V while the
-//                         last product was in flight, rounds once and stores.
+//                         the four accumulators, adds the depthwise 3x3 term, rounds once and stores.
+// The probabilities of a step overwrite, in place, the bias values that the same thread has just read (same
+// rows, same columns of the B2 stage), so P needs no buffer of its own; the room holds the V tokens of the
+// depthwise window instead: three runs of 130 consecutive tokens (the tile's own, and those one grid row above
+// and below, each with one token more on either side), fetched by TMA with the 128-byte swizzle.
 // Every wait is bounded (pipe.cuh).  No TMA multicast, no clusters.
 #include "common.cuh"
 #include "kernels.h"
@@ -38,9 +41,11 @@ constexpr int OFF_W = OFF_ML + 4 * 128 * 8;              // filter taps [9][64] 
 constexpr int OFF_A = 8192;                              // agents [256][128 B]
 constexpr int OFF_VA = OFF_A + 4 * kTile;                // agent features [256][128 B]
 constexpr int OFF_Q = OFF_VA + 4 * kTile;                // 2 x query tile [128][128 B]
-constexpr int OFF_P = OFF_Q + 4 * kTile;                 // probabilities of the step: 2 column atoms x [128][128 B]
-constexpr int OFF_B2 = OFF_P + 4 * kTile;                // 2 stages x (2 column atoms x [128][128 B])
-constexpr int kSmemBytes = OFF_B2 + 2 * 4 * kTile + 1024;
+constexpr int OFF_B2 = OFF_Q + 4 * kTile;                // 2 stages x (2 column atoms x [128][128 B]): bias, then probabilities
+constexpr int kHaloRows = 136;                           // 130 tokens of a run, rounded up to whole swizzle atoms
+constexpr int kHaloSeg = kHaloRows * 128;
+constexpr int OFF_H = OFF_B2 + 2 * 4 * kTile;            // 3 runs of V tokens [136][128 B]
+constexpr int kSmemBytes = OFF_H + 3 * kHaloSeg + 1024;
 static_assert(OFF_W + 9 * 64 * 4 <= OFF_A, "small buffers");
 static_assert(kSmemBytes <= 232448 && kSmemBytes > 116 * 1024, "one block per SM");
 
@@ -50,12 +55,14 @@ constexpr int BAR_PREP = 1;        //          1              MMA issuer      V_
 constexpr int BAR_Q_FULL = 2;      // [2]      tx             MMA issuer
 constexpr int BAR_Q_EMPTY = 4;     // [2]      commit         producer
 constexpr int BAR_B_FULL = 6;      // [2]      tx             row warps
-constexpr int BAR_B_EMPTY = 8;     // [2]      row threads    producer
+constexpr int BAR_B_EMPTY = 8;     // [2]      commit         producer        the product that read the stage is done
 constexpr int BAR_S_FULL = 10;     // [2]      commit         row warps
 constexpr int BAR_S_EMPTY = 12;    // [2]      row threads    MMA issuer
 constexpr int BAR_P_FULL = 14;     //          row threads    MMA issuer
 constexpr int BAR_PV = 15;         //          commit         row warps
-constexpr int kBars = 16;
+constexpr int BAR_H_FULL = 16;     //          tx             row warps       V tokens of the tile's depthwise window
+constexpr int BAR_H_EMPTY = 17;    //          row threads    producer
+constexpr int kBars = 18;
 
 // tensor memory: logits 2 buffers x 128 columns, accumulators 4 groups x 64 columns
 constexpr uint32_t TM_S = 0, TM_O = 256;
@@ -63,7 +70,7 @@ constexpr uint32_t TM_S = 0, TM_O = 256;
 struct UmmaBcArgs {
     AttnArgs a;
     int MB, tps;                       // 128-agent blocks (1 or 2), tiles per split
-    alignas(64) CUtensorMap tm_q, tm_a, tm_va, tm_b;
+    alignas(64) CUtensorMap tm_q, tm_a, tm_va, tm_b, tm_h;     // tm_h: V as [slabs*N][d] with 136-row boxes
 };
 }  // namespace
 
@@ -94,7 +101,7 @@ __global__ void __launch_bounds__(NT, 1) broadcast_umma_kernel(const __grid_cons
     if (tid == 0) {
         s_dead = 0;
         for (int i = 0; i < kBars; ++i) {
-            const bool many = i == BAR_B_EMPTY || i == BAR_B_EMPTY + 1 || i == BAR_S_EMPTY || i == BAR_S_EMPTY + 1 || i == BAR_P_FULL;
+            const bool many = i == BAR_S_EMPTY || i == BAR_S_EMPTY + 1 || i == BAR_P_FULL || i == BAR_H_EMPTY;
             mbar_init(pp.bars + 8 * i, many ? (uint32_t)NROW : 1u);
         }
         mbar_fence_init();
@@ -106,7 +113,7 @@ __global__ void __launch_bounds__(NT, 1) broadcast_umma_kernel(const __grid_cons
     pp.tmem = s_tmem;
 
     const uint32_t sA = smem_u32(smem + OFF_A), sVA = smem_u32(smem + OFF_VA), sQ = smem_u32(smem + OFF_Q);
-    const uint32_t sP = smem_u32(smem + OFF_P), sB2 = smem_u32(smem + OFF_B2);
+    const uint32_t sB2 = smem_u32(smem + OFF_B2), sH = smem_u32(smem + OFF_H);
 
     if (warp == 16) {
         // ------------------------------------------------------------------ producer
@@ -121,6 +128,14 @@ __global__ void __launch_bounds__(NT, 1) broadcast_umma_kernel(const __grid_cons
                 if (i >= 2) pipe_wait_one(pp, BAR_Q_EMPTY + (i & 1), kTimeoutRole);
                 mbar_arrive_expect_tx(pipe_bar(pp, BAR_Q_FULL + (i & 1)), 2 * kTile);
                 tma_load_2d(sQ + (i & 1) * 2 * kTile, &g.tm_q, 0, slab * N + tok0, pipe_bar(pp, BAR_Q_FULL + (i & 1)));
+                if (has_dwc) {
+                    // runs of tokens one grid row above, around and below the tile, each from one token before
+                    // it (rows outside the tensor are zero-filled; tokens of other slabs are masked by the readers)
+                    if (i >= 1) pipe_wait_one(pp, BAR_H_EMPTY, kTimeoutRole);
+                    mbar_arrive_expect_tx(pipe_bar(pp, BAR_H_FULL), 3 * kHaloSeg);
+                    for (int u = 0; u < 3; ++u)
+                        tma_load_2d(sH + u * kHaloSeg, &g.tm_h, 0, slab * N + tok0 + (u - 1) * p.W - 1, pipe_bar(pp, BAR_H_FULL));
+                }
                 if (has_b2)
                     for (int a = 0; a < MB; ++a) {
                         const int j = i * MB + a, b = j & 1;
@@ -134,6 +149,7 @@ __global__ void __launch_bounds__(NT, 1) broadcast_umma_kernel(const __grid_cons
             for (int i = max(0, tiles - 2); i < tiles; ++i) pipe_wait_one(pp, BAR_Q_EMPTY + (i & 1), kTimeoutRole);
             if (has_b2)
                 for (int j = max(0, steps - 2); j < steps; ++j) pipe_wait_one(pp, BAR_B_EMPTY + (j & 1), kTimeoutRole);
+            if (has_dwc) pipe_wait_one(pp, BAR_H_EMPTY, kTimeoutRole);
         }
         __syncwarp();
     } else if (warp == 17) {
@@ -165,7 +181,7 @@ __global__ void __launch_bounds__(NT, 1) broadcast_umma_kernel(const __grid_cons
         // ------------------------------------------------------------------ MMA issuer: products P V_A
         if (lane == 0) {
             const uint32_t idMN = umma_idesc(fmt, 128, 64, 1);
-            const uint64_t dVA = umma_desc_sw128(sVA), dP = umma_desc_sw128(sP);
+            const uint64_t dVA = umma_desc_sw128(sVA), dP0 = umma_desc_sw128(sB2);
             // + 128 per K-step of an MN-major operand (16 rows of 128 bytes)
             pipe_wait_one(pp, BAR_PREP, kTimeoutLoads);
             unsigned started = 0u;
@@ -174,6 +190,7 @@ __global__ void __launch_bounds__(NT, 1) broadcast_umma_kernel(const __grid_cons
                 if (a == 0) started = 0u;
                 pipe_wait_one(pp, BAR_P_FULL, kTimeoutRole);
                 tc_fence_after_sync();
+                const uint64_t dP = dP0 + 2048 * (j & 1);             // the step's stage: 32 KB = 2048 units
                 for (int gq = 0; gq < 4; ++gq) {
                     if (128 * a + 32 * gq >= n) break;
                     const uint32_t dd = pp.tmem + TM_O + 64 * gq;
@@ -182,6 +199,7 @@ __global__ void __launch_bounds__(NT, 1) broadcast_umma_kernel(const __grid_cons
                     umma_f16_c<1>(dd, da + 2, db + 128, idMN);
                     started |= 1u << gq;
                 }
+                if (has_b2) umma_commit(pipe_bar(pp, BAR_B_EMPTY + (j & 1)));     // the stage may take the bias of step j + 2
                 umma_commit(pipe_bar(pp, BAR_PV));
             }
         }
@@ -212,7 +230,6 @@ __global__ void __launch_bounds__(NT, 1) broadcast_umma_kernel(const __grid_cons
         asm volatile("bar.sync 1, %0;\n" ::"n"(NROW) : "memory");
         if (tid == 0) pipe_arrive(pp, BAR_PREP);
 
-        const T* gV = static_cast<const T*>(p.dwc_v) + (size_t)slab * N * d;
         T* gO = static_cast<T*>(p.out) + (size_t)slab * N * d;
         for (int i = 0; i < tiles; ++i) {
             const int tok = (i0 + i) * QT + row;
@@ -242,7 +259,6 @@ __global__ void __launch_bounds__(NT, 1) broadcast_umma_kernel(const __grid_cons
 #pragma unroll
                             for (int k = 0; k < 8; ++k) sv[8 * jj + k] = fmaf(__uint_as_float(ra[8 * jj + k]), p.scale, f[k]);
                         }
-                        pipe_arrive(pp, BAR_B_EMPTY + b);
                     } else {
 #pragma unroll
                         for (int k = 0; k < 32; ++k) sv[k] = __uint_as_float(ra[k]) * p.scale;
@@ -301,7 +317,7 @@ __global__ void __launch_bounds__(NT, 1) broadcast_umma_kernel(const __grid_cons
                 if (tv) {
 #pragma unroll
                     for (int jj = 0; jj < 4; ++jj)
-                        *reinterpret_cast<uint4*>(smem + OFF_P + (gq >> 1) * 2 * kTile + row * 128 + (((4 * (gq & 1) + jj) ^ (row & 7)) << 4)) =
+                        *reinterpret_cast<uint4*>(smem + OFF_B2 + b * 4 * kTile + (gq >> 1) * 2 * kTile + row * 128 + (((4 * (gq & 1) + jj) ^ (row & 7)) << 4)) =
                             make_uint4(pk[4 * jj], pk[4 * jj + 1], pk[4 * jj + 2], pk[4 * jj + 3]);
                 }
                 fence_proxy_async();
@@ -313,8 +329,9 @@ __global__ void __launch_bounds__(NT, 1) broadcast_umma_kernel(const __grid_cons
 #pragma unroll
             for (int k = 0; k < 8; ++k) dw[k] = make_float2(0.f, 0.f);
             if (has_dwc) {
-                // all taps of a grid row are fetched before they are used (loads outside the grid or past the
-                // head dim become zeros, from a clamped address), so the L2 latency is paid once per row
+                // tap (u, v) of this thread's token sits at row (row + v) of run u; taps outside the grid
+                // (or in another slab, or past the head dim) contribute nothing
+                pipe_wait(pp, BAR_H_FULL, kTimeoutLoads);
                 const int tk = min(tok, N - 1);
                 const int y = tk / W, x = tk - y * W;
                 const bool live = tok < N && nch > 0;
@@ -322,29 +339,26 @@ __global__ void __launch_bounds__(NT, 1) broadcast_umma_kernel(const __grid_cons
                 for (int u = 0; u < 3; ++u) {
                     const int yy = y + u - 1;
                     const bool rowok = live && yy >= 0 && yy < H;
-                    uint4 raw[3][2];
 #pragma unroll
                     for (int v = 0; v < 3; ++v) {
                         const int xx = x + v - 1;
                         const bool ok = rowok && xx >= 0 && xx < W;
-                        const uint4* src = reinterpret_cast<const uint4*>(gV + (ok ? (yy * W + xx) * d + c0 : 0));
-                        raw[v][0] = ok ? __ldg(src) : make_uint4(0u, 0u, 0u, 0u);
-                        raw[v][1] = (ok && nch > 8) ? __ldg(src + 1) : make_uint4(0u, 0u, 0u, 0u);
-                    }
-#pragma unroll
-                    for (int v = 0; v < 3; ++v) {
+                        const int r = row + v;
+                        const unsigned char* src = smem + OFF_H + u * kHaloSeg + r * 128;
                         const float4* wt = reinterpret_cast<const float4*>(sW + (u * 3 + v) * 64 + c0);
 #pragma unroll
                         for (int hh = 0; hh < 2; ++hh) {
+                            uint4 rr = *reinterpret_cast<const uint4*>(src + ((((c0 >> 3) + hh) ^ (r & 7)) << 4));
+                            if (!ok || (hh == 1 && nch <= 8)) rr = make_uint4(0u, 0u, 0u, 0u);
                             const float4 w0 = wt[2 * hh], w1 = wt[2 * hh + 1];
-                            const uint4 r = raw[v][hh];
-                            dw[4 * hh + 0] = ffma2(make_float2(w0.x, w0.y), unpack2<T>(r.x), dw[4 * hh + 0]);
-                            dw[4 * hh + 1] = ffma2(make_float2(w0.z, w0.w), unpack2<T>(r.y), dw[4 * hh + 1]);
-                            dw[4 * hh + 2] = ffma2(make_float2(w1.x, w1.y), unpack2<T>(r.z), dw[4 * hh + 2]);
-                            dw[4 * hh + 3] = ffma2(make_float2(w1.z, w1.w), unpack2<T>(r.w), dw[4 * hh + 3]);
+                            dw[4 * hh + 0] = ffma2(make_float2(w0.x, w0.y), unpack2<T>(rr.x), dw[4 * hh + 0]);
+                            dw[4 * hh + 1] = ffma2(make_float2(w0.z, w0.w), unpack2<T>(rr.y), dw[4 * hh + 1]);
+                            dw[4 * hh + 2] = ffma2(make_float2(w1.x, w1.y), unpack2<T>(rr.z), dw[4 * hh + 2]);
+                            dw[4 * hh + 3] = ffma2(make_float2(w1.z, w1.w), unpack2<T>(rr.w), dw[4 * hh + 3]);
                         }
                     }
                 }
+                pipe_arrive(pp, BAR_H_EMPTY);
             }
             sML[gq * 128 + row] = make_float2(started ? m_ref : -INFINITY, started ? l : 0.f);
             pipe_wait(pp, BAR_PV, kTimeoutTile);
@@ -429,6 +443,7 @@ cudaError_t launch_broadcast_umma(int dtype, const AttnArgs& p, int sm_count, cu
     if (!make_map_2d_u16(&g.tm_a, p.km, S * n, p.d, 128, 64)) return cudaErrorNotSupported;
     if (!make_map_2d_u16(&g.tm_va, p.vm, S * n, p.d, 128, 64)) return cudaErrorNotSupported;
     if (p.bias && !make_map_2d_u16(&g.tm_b, p.bias, (uint64_t)p.heads * N, n, 128, 64)) return cudaErrorNotSupported;
+    if (p.dwc_w && !make_map_2d_u16(&g.tm_h, p.dwc_v, S * N, p.d, kHaloRows, 64)) return cudaErrorNotSupported;
     if (dtype == kBF16) return launch_bc_umma_t<__nv_bfloat16>(g, splits, st);
     if (dtype == kF16) return launch_bc_umma_t<__half>(g, splits, st);
     return cudaErrorInvalidValue;
