@@ -3,7 +3,7 @@
 //
 // Grid: (splits, slabs), one block of 19 warps per SM.  A block keeps the slab's agents resident (up to
 // two 128-row operand blocks) and streams its share of the slab's 64-token tiles (K, V and the matching
-// B1 columns) through a three-stage TMA ring.
+// B1 columns) through a four-stage TMA ring.
 //   warp 16 "producer":  one lane issues every TMA copy, ahead of the others through full/empty mbarriers.
 //   warp 17 "MMA issuer": one lane issues S = A K^T (tcgen05.mma, accumulator in tensor memory) one tile
 //                        ahead; warp 18 issues the products P V once the probabilities of a tile are written
@@ -11,7 +11,9 @@
 //   warps 0-15 "row warps": thread (agent row, token half): reads its 32 logits of the tile from tensor
 //                        memory, adds scale and bias, keeps its own running maximum / sum (no reduction
 //                        crosses threads: each token half has its own accumulator in tensor memory),
-//                        writes the probabilities back to shared memory as the A operand of P V.
+//                        writes the probabilities back to shared memory as the A operand of P V, in place
+//                        of the bias values it has just read (so P needs no buffer and the ring has a
+//                        fourth stage).
 //                        A row's reference maximum moves only when exceeded by a margin; then the thread
 //                        rescales its accumulator row in tensor memory.
 // At the end the two token halves of a row meet in shared memory and the block writes one partial state;
@@ -31,7 +33,7 @@ namespace {
 constexpr int KT = 64;                 // tokens per tile
 constexpr int NROW = 512;              // row-warp threads
 constexpr int NT = NROW + 96;          // + producer warp + two MMA issuer warps (logits, products)
-constexpr int STAGES = 3;
+constexpr int STAGES = 4;
 constexpr int kTile = 64 * 128;        // swizzled [64][64] tile of 16-bit elements
 constexpr float kTau = 5.5f;           // margin (natural units) before a row's reference maximum moves
 constexpr int kTimeoutTile = 3, kTimeoutLoads = 4, kTimeoutRole = 6;
@@ -39,21 +41,20 @@ constexpr int kTimeoutTile = 3, kTimeoutLoads = 4, kTimeoutRole = 6;
 // shared memory (bytes from a 1024-aligned base)
 constexpr int OFF_BAR = 0;                               // mbarriers
 constexpr int OFF_A = 1024;                              // agents [256][128 B]
-constexpr int OFF_P = OFF_A + 4 * kTile;                 // probabilities of the tile [256][128 B]
-constexpr int OFF_RING = OFF_P + 4 * kTile;              // STAGES x (K | V | B1 [256][128 B])
+constexpr int OFF_RING = OFF_A + 4 * kTile;              // STAGES x (K | V | B1 [256][128 B], later the probabilities)
 constexpr int kStage = 2 * kTile + 4 * kTile;
 constexpr int kSmemBytes = OFF_RING + STAGES * kStage + 1024;
 static_assert(kSmemBytes <= 232448 && kSmemBytes > 116 * 1024, "one block per SM");
 
 // mbarriers                                    count            waiter
-constexpr int BAR_FULL = 0;       // [STAGES]   tx               MMA issuer (and, for the bias, nobody else: see P_FULL)
-constexpr int BAR_EMPTY = 3;      // [STAGES]   commit           producer
-constexpr int BAR_S_FULL = 6;     // [2]        commit           row warps
-constexpr int BAR_S_EMPTY = 8;    // [2]        row threads      MMA issuer
-constexpr int BAR_P_FULL = 10;    //            row threads      MMA issuer
-constexpr int BAR_PV = 11;        //            commit           row warps
-constexpr int BAR_AG = 12;        //            tx               MMA issuer
-constexpr int kBars = 13;
+constexpr int BAR_FULL = 0;       // [STAGES]   tx               both MMA issuers
+constexpr int BAR_EMPTY = 4;      // [STAGES]   commit           producer
+constexpr int BAR_S_FULL = 8;     // [2]        commit           row warps
+constexpr int BAR_S_EMPTY = 10;   // [2]        row threads      MMA issuer (logits)
+constexpr int BAR_P_FULL = 12;    //            row threads      MMA issuer (products)
+constexpr int BAR_PV = 13;        //            commit           row warps
+constexpr int BAR_AG = 14;        //            tx               MMA issuer (logits)
+constexpr int kBars = 15;
 
 // tensor memory: logits 2 buffers x (2 agent blocks x 64), accumulators (agent block, token half) x 64
 constexpr uint32_t TM_S = 0, TM_O = 256;
@@ -101,7 +102,7 @@ __global__ void __launch_bounds__(NT, 1) aggregate_umma_kernel(const __grid_cons
     tc_fence_after_sync();
     pp.tmem = s_tmem;
 
-    const uint32_t sA = smem_u32(smem + OFF_A), sP = smem_u32(smem + OFF_P), ring = smem_u32(smem + OFF_RING);
+    const uint32_t sA = smem_u32(smem + OFF_A), ring = smem_u32(smem + OFF_RING);
     const size_t pf = partial_floats(g.rows_pad, 64);
     float* slab_parts = p.partials + (size_t)slab * gridDim.x * pf;
 
@@ -155,7 +156,7 @@ __global__ void __launch_bounds__(NT, 1) aggregate_umma_kernel(const __grid_cons
         // ------------------------------------------------------------------ MMA issuer: products P V
         if (lane == 0) {
             const uint32_t idMN = umma_idesc(fmt, 128, 64, 1);
-            const uint64_t dP = umma_desc_sw128(sP), dRing = umma_desc_sw128(ring);
+            const uint64_t dRing = umma_desc_sw128(ring);
             // + 128 per K-step of an MN-major operand (16 rows of 128 bytes)
             for (int t = 0; t < tiles; ++t) {
                 const int s = t % STAGES;
@@ -164,6 +165,7 @@ __global__ void __launch_bounds__(NT, 1) aggregate_umma_kernel(const __grid_cons
                 tc_fence_after_sync();
                 const int ntok = min(KT, N - (t0 + t) * KT);
                 const uint64_t dV = dRing + (uint64_t)(s * (kStage >> 4)) + (uint64_t)(kTile >> 4);
+                const uint64_t dP = dV + (uint64_t)(kTile >> 4);      // the probabilities replaced the stage's bias tile
                 for (int mb = 0; mb < MB; ++mb)
                     for (int c = 0; c < 2; ++c) {
                         if (32 * c >= ntok) break;
@@ -270,7 +272,7 @@ __global__ void __launch_bounds__(NT, 1) aggregate_umma_kernel(const __grid_cons
             if (tv) {
 #pragma unroll
                 for (int j = 0; j < 4; ++j)
-                    *reinterpret_cast<uint4*>(smem + OFF_P + row * 128 + (((4 * c + j) ^ (row & 7)) << 4)) =
+                    *reinterpret_cast<uint4*>(smem + OFF_RING + s * kStage + 2 * kTile + row * 128 + (((4 * c + j) ^ (row & 7)) << 4)) =
                         make_uint4(pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);
             }
             fence_proxy_async();
