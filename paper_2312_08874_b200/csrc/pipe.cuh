@@ -9,19 +9,6 @@ namespace aa {
 constexpr unsigned kPipeBarLimit = 1u << 20;      // mbarrier try_wait attempts before a wait gives up
 constexpr unsigned kPipeSuspendNs = 2000;         // a try_wait may keep its thread suspended this long
 
-// try_wait with a suspend-time hint: the hardware parks the thread until the phase completes or the
-// time is up, so a waiting warp issues next to nothing (a spinning one would take issue slots away
-// from the working warps).
-__device__ __forceinline__ bool mbar_try_wait_hint(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}\n"
-        : "=r"(ok) : "r"(bar), "r"(parity), "r"(kPipeSuspendNs) : "memory");
-    return ok != 0;
-}
-
 // Per-thread view of a block's mbarriers.  Every wait is bounded: on expiry the thread sets the
 // block-wide `dead` flag (every later wait of the block then returns at once) and records `code` in the
 // device status word, so a logic error ends as a status code instead of a hang.
@@ -42,7 +29,7 @@ __device__ __forceinline__ void pipe_wait_one(Pipe& pp, int i, int code) {
     if (pipe_dead(pp)) return;
     const uint32_t bar = pipe_bar(pp, i);
     for (unsigned tries = 0; tries < kPipeBarLimit; ++tries) {
-        if (mbar_try_wait_hint(bar, parity)) return;
+        if (mbar_try_wait_suspend(bar, parity, kPipeSuspendNs)) return;
         if ((tries & 15u) == 15u && pipe_dead(pp)) return;
     }
     *reinterpret_cast<volatile int*>(pp.dead) = 1;
