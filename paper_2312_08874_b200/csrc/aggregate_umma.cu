@@ -88,7 +88,7 @@ __global__ void __launch_bounds__(NT, 1) aggregate_umma_kernel(const __grid_cons
     pp.status = p.status;
     pp.dead = &s_dead;
     pp.bars = smem_u32(smem + OFF_BAR);
-    pp.ph = 0ull;
+    pp.ph = 0u;
     const uint32_t row_threads = 256u * (uint32_t)MB;
     if (tid == 0) {
         s_dead = 0;

@@ -97,7 +97,7 @@ __global__ void __launch_bounds__(NT, 1) broadcast_umma_kernel(const __grid_cons
     pp.status = p.status;
     pp.dead = &s_dead;
     pp.bars = smem_u32(smem + OFF_BAR);
-    pp.ph = 0ull;
+    pp.ph = 0u;
     if (tid == 0) {
         s_dead = 0;
         for (int i = 0; i < kBars; ++i) {

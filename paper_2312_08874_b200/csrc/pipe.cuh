@@ -16,21 +16,22 @@ struct Pipe {
     int* status;          // device status word (global)
     int* dead;            // shared flag
     uint32_t bars;        // shared address of mbarrier 0
-    uint64_t ph;          // parity to wait for next, one bit per mbarrier this thread waits on
+    uint32_t ph;          // parity to wait for next, one bit per mbarrier this thread waits on (at most 32 barriers)
     uint32_t tmem;        // base of the block's tensor-memory columns
 };
 __device__ __forceinline__ uint32_t pipe_bar(const Pipe& pp, int i) { return pp.bars + 8u * (uint32_t)i; }
 __device__ __forceinline__ int pipe_dead(const Pipe& pp) { return *reinterpret_cast<const volatile int*>(pp.dead); }
 
-// One thread waits for the next phase of mbarrier i (its parity bit flips either way).
+// One thread waits for the next phase of mbarrier i (its parity bit flips either way).  The first
+// attempt is the fast path; the bounded loop and the look at the block's flag come only after it fails.
 __device__ __forceinline__ void pipe_wait_one(Pipe& pp, int i, int code) {
-    const uint32_t parity = (uint32_t)(pp.ph >> i) & 1u;
-    pp.ph ^= 1ull << i;
-    if (pipe_dead(pp)) return;
+    const uint32_t parity = (pp.ph >> i) & 1u;
+    pp.ph ^= 1u << i;
     const uint32_t bar = pipe_bar(pp, i);
+    if (mbar_try_wait_suspend(bar, parity, kPipeSuspendNs)) return;
     for (unsigned tries = 0; tries < kPipeBarLimit; ++tries) {
+        if (pipe_dead(pp)) return;
         if (mbar_try_wait_suspend(bar, parity, kPipeSuspendNs)) return;
-        if ((tries & 15u) == 15u && pipe_dead(pp)) return;
     }
     *reinterpret_cast<volatile int*>(pp.dead) = 1;
     if (pp.status) atomicCAS(pp.status, 0, code);
