@@ -254,10 +254,13 @@ __global__ void __launch_bounds__(NT, 1) broadcast_umma_kernel(const __grid_cons
 #pragma unroll
                         for (int jj = 0; jj < 4; ++jj) {
                             const uint4 raw = *reinterpret_cast<const uint4*>(sB + (((4 * (gq & 1) + jj) ^ (row & 7)) << 4));
-                            float f[8];
-                            unpack16<T>(raw, f);
+                            const uint32_t w4[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
-                            for (int k = 0; k < 8; ++k) sv[8 * jj + k] = fmaf(__uint_as_float(ra[8 * jj + k]), p.scale, f[k]);
+                            for (int k = 0; k < 4; ++k) {        // packed pairs: one instruction per two logits
+                                const float2 r2 = ffma2(make_float2(__uint_as_float(ra[8 * jj + 2 * k]), __uint_as_float(ra[8 * jj + 2 * k + 1])),
+                                                        make_float2(p.scale, p.scale), unpack2<T>(w4[k]));
+                                sv[8 * jj + 2 * k] = r2.x; sv[8 * jj + 2 * k + 1] = r2.y;
+                            }
                         }
                     } else {
 #pragma unroll
@@ -286,18 +289,19 @@ __global__ void __launch_bounds__(NT, 1) broadcast_umma_kernel(const __grid_cons
                         l *= corr;
                     }
                     const float nb = -m_ref * kLog2e;
-                    float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
+                    float2 s01 = make_float2(0.f, 0.f), s23 = make_float2(0.f, 0.f);
+                    const float2 l2e = make_float2(kLog2e, kLog2e), nb2 = make_float2(nb, nb);
 #pragma unroll
                     for (int k = 0; k < 16; k += 2) {
-                        const float p0 = fast_exp2(fmaf(sv[2 * k], kLog2e, nb));      // exp2(-inf) = 0 past the last agent
-                        const float p1 = fast_exp2(fmaf(sv[2 * k + 1], kLog2e, nb));
-                        const float p2 = fast_exp2(fmaf(sv[2 * k + 2], kLog2e, nb));
-                        const float p3 = fast_exp2(fmaf(sv[2 * k + 3], kLog2e, nb));
-                        pk[k] = pack2<T>(p0, p1);
-                        pk[k + 1] = pack2<T>(p2, p3);
-                        sum0 += p0; sum1 += p1; sum2 += p2; sum3 += p3;
+                        const float2 a0 = ffma2(make_float2(sv[2 * k], sv[2 * k + 1]), l2e, nb2);
+                        const float2 a1 = ffma2(make_float2(sv[2 * k + 2], sv[2 * k + 3]), l2e, nb2);
+                        const float2 p01 = make_float2(fast_exp2(a0.x), fast_exp2(a0.y));     // exp2(-inf) = 0 past the last agent
+                        const float2 p23 = make_float2(fast_exp2(a1.x), fast_exp2(a1.y));
+                        s01 = fadd2(s01, p01); s23 = fadd2(s23, p23);
+                        pk[k] = pack2<T>(p01.x, p01.y);
+                        pk[k + 1] = pack2<T>(p23.x, p23.y);
                     }
-                    l += (sum0 + sum1) + (sum2 + sum3);
+                    l += (s01.x + s01.y) + (s23.x + s23.y);
                     started = true;
                 }
                 // the previous step's product is done: P may be overwritten, this thread's accumulator is at rest
