@@ -6,7 +6,6 @@
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
-#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <new>
@@ -316,14 +315,6 @@ int agent_attn_forward(agent_attn_handle* h, const void* Q, const void* K, const
     cudaStream_t st = (cudaStream_t)stream;
     char* ws = static_cast<char*>(workspace);
     if (!A && h->cfg.path == AA_PATH_AUTO && h->cfg.dtype != AA_F32) {
-        // small token counts: one kernel with the slab resident in shared memory
-        if (slab_eligible(h->cfg.dtype, grid_h, grid_w, h->cfg.head_dim, n_agents) && !getenv("AGENT_ATTN_NO_SLAB")) {
-            cudaError_t e = launch_slab(h->cfg.dtype, Q, K, V, b1, b2, dwc_weight, out, h->d_status, h->cfg.batch * h->cfg.heads,
-                                        h->cfg.heads, grid_h, grid_w, n_agents, p, h->scale1, h->scale2, h->sm_count, st);
-            if (e != cudaSuccess) return fail(h, AA_ERR_CUDA, "slab kernel launch failed: %s", cudaGetErrorString(e));
-            h->launches = 1;
-            return AA_OK;
-        }
         // one persistent kernel for the whole module where the shape allows it
         if (h->fused_key[0] != grid_h || h->fused_key[1] != grid_w || h->fused_key[2] != n_agents) {
             h->fused_plan = plan_fused(h->cfg.dtype, h->cfg.batch * h->cfg.heads, grid_h, grid_w, h->cfg.head_dim,

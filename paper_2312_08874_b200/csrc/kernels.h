@@ -74,11 +74,6 @@ cudaError_t launch_broadcast_mma(int dtype, const AttnArgs& p, cudaStream_t st);
 bool aggregate_umma_eligible(int dtype, int n_agents, int n_tokens, int d, bool has_bias);
 AggPlan plan_aggregate_umma(int slabs, int n_agents, int n_tokens, int d, int sm_count);
 cudaError_t launch_aggregate_umma(int dtype, const AttnArgs& p, const AggPlan& plan, cudaStream_t st);
-// whole module with the slab resident in shared memory, for small token counts (slab_kernel.cu)
-bool slab_eligible(int dtype, int H, int W, int d, int n_agents);
-cudaError_t launch_slab(int dtype, const void* q, const void* k, const void* v, const void* b1, const void* b2,
-                        const void* dwc_w, void* out, int* status, int slabs, int heads, int H, int W, int n_agents,
-                        int pool, float scale1, float scale2, int sm_count, cudaStream_t st);
 bool broadcast_umma_eligible(int dtype, int n_agents, int n_tokens, int d);
 cudaError_t launch_broadcast_umma(int dtype, const AttnArgs& p, int sm_count, cudaStream_t st);
 
