@@ -5,9 +5,11 @@
 // two 128-row operand blocks) and streams its share of the slab's 64-token tiles (K, V and the matching
 // B1 columns) through a four-stage TMA ring.
 //   warp 16 "producer":  one lane issues every TMA copy, ahead of the others through full/empty mbarriers.
-//   warp 17 "MMA issuer": one lane issues S = A K^T (tcgen05.mma, accumulator in tensor memory) one tile
-//                        ahead; warp 18 issues the products P V once the probabilities of a tile are written
-//                        (two issuing threads, so that neither instruction stream delays the other).
+//   warps 17, 18 "MMA issuers": one lane each, one per agent block ("chain"): S = A_block K^T (tcgen05.mma,
+//                        accumulator in tensor memory) one tile ahead, and the products P V once the chain's
+//                        probabilities of a tile are written.  The two chains (agents 0-127, agents 128-255)
+//                        share the ring but have their own barriers, so that one computes while the other
+//                        waits for its products.
 //   warps 0-15 "row warps": thread (agent row, token half): reads its 32 logits of the tile from tensor
 //                        memory, adds scale and bias, keeps its own running maximum / sum (no reduction
 //                        crosses threads: each token half has its own accumulator in tensor memory),
@@ -47,14 +49,14 @@ constexpr int kSmemBytes = OFF_RING + STAGES * kStage + 1024;
 static_assert(kSmemBytes <= 232448 && kSmemBytes > 116 * 1024, "one block per SM");
 
 // mbarriers                                    count            waiter
-constexpr int BAR_FULL = 0;       // [STAGES]   tx               both MMA issuers
-constexpr int BAR_EMPTY = 4;      // [STAGES]   commit           producer
-constexpr int BAR_S_FULL = 8;     // [2]        commit           row warps
-constexpr int BAR_S_EMPTY = 10;   // [2]        row threads      MMA issuer (logits)
-constexpr int BAR_P_FULL = 12;    //            row threads      MMA issuer (products)
-constexpr int BAR_PV = 13;        //            commit           row warps
-constexpr int BAR_AG = 14;        //            tx               MMA issuer (logits)
-constexpr int kBars = 15;
+constexpr int BAR_FULL = 0;       // [STAGES]        tx             each chain's MMA issuer
+constexpr int BAR_EMPTY = 4;      // [STAGES]        one commit per chain     producer
+constexpr int BAR_S_FULL = 8;     // [chain][2]      commit         the chain's row warps
+constexpr int BAR_S_EMPTY = 12;   // [chain][2]      256 threads    the chain's MMA issuer
+constexpr int BAR_P_FULL = 16;    // [chain]         256 threads    the chain's MMA issuer
+constexpr int BAR_PV = 18;        // [chain]         commit         the chain's row warps
+constexpr int BAR_AG = 20;        //                 tx             both MMA issuers
+constexpr int kBars = 21;
 
 // tensor memory: logits 2 buffers x (2 agent blocks x 64), accumulators (agent block, token half) x 64
 constexpr uint32_t TM_S = 0, TM_O = 256;
@@ -89,11 +91,10 @@ __global__ void __launch_bounds__(NT, 1) aggregate_umma_kernel(const __grid_cons
     pp.dead = &s_dead;
     pp.bars = smem_u32(smem + OFF_BAR);
     pp.ph = 0u;
-    const uint32_t row_threads = 256u * (uint32_t)MB;
     if (tid == 0) {
         s_dead = 0;
         for (int i = 0; i < kBars; ++i)
-            mbar_init(pp.bars + 8 * i, (i >= BAR_S_EMPTY && i <= BAR_P_FULL) ? row_threads : 1u);
+            mbar_init(pp.bars + 8 * i, (i >= BAR_S_EMPTY && i < BAR_PV) ? 256u : (i >= BAR_EMPTY && i < BAR_S_FULL) ? (uint32_t)MB : 1u);
         mbar_fence_init();
     }
     if (warp == 0) tmem_alloc<512>(smem_u32(&s_tmem));
@@ -125,58 +126,48 @@ __global__ void __launch_bounds__(NT, 1) aggregate_umma_kernel(const __grid_cons
             for (int t = max(0, tiles - STAGES); t < tiles; ++t) pipe_wait_one(pp, BAR_EMPTY + t % STAGES, kTimeoutRole);
         }
         __syncwarp();
-    } else if (warp == 17) {
-        // ------------------------------------------------------------------ MMA issuer: logits, one tile ahead
-        if (lane == 0) {
-            const uint32_t idK = umma_idesc(fmt, 128, 64, 0);
-            const uint64_t dA = umma_desc_sw128(sA), dRing = umma_desc_sw128(ring);
+    } else if (warp == 17 || warp == 18) {
+        // ------------------------------------------------------------------ MMA issuer of chain m = agent block m
+        const int m = warp - 17;
+        if (lane == 0 && m < MB) {
+            const uint32_t idK = umma_idesc(fmt, 128, 64, 0), idMN = umma_idesc(fmt, 128, 64, 1);
+            const uint64_t dA = umma_desc_sw128(sA) + 1024 * m, dRing = umma_desc_sw128(ring);
             // descriptor start addresses count 16-byte units: + 2 per K-step of a K-major operand (32 bytes),
-            // + 1024 per 128-row block
-            pipe_wait_one(pp, BAR_AG, kTimeoutLoads);
-            for (int t = 0; t < tiles; ++t) {
+            // + 128 per K-step of an MN-major operand (16 rows of 128 bytes), + 1024 per 128-row block
+            auto issue_S = [&](int t) {
                 const int b = t & 1, s = t % STAGES;
-                if (t >= 2) pipe_wait_one(pp, BAR_S_EMPTY + b, kTimeoutRole);
+                if (t >= 2) pipe_wait_one(pp, BAR_S_EMPTY + 2 * m + b, kTimeoutRole);
                 pipe_wait_one(pp, BAR_FULL + s, kTimeoutTile);
                 tc_fence_after_sync();
                 const uint64_t dK = dRing + (uint64_t)(s * (kStage >> 4));
-                for (int mb = 0; mb < MB; ++mb) {
-                    const uint32_t dd = pp.tmem + TM_S + 128 * b + 64 * mb;
-                    const uint64_t da = dA + 1024 * mb;
-                    umma_f16_c<0>(dd, da, dK, idK);
-                    umma_f16_c<1>(dd, da + 2, dK + 2, idK);
-                    umma_f16_c<1>(dd, da + 4, dK + 4, idK);
-                    umma_f16_c<1>(dd, da + 6, dK + 6, idK);
-                }
-                umma_commit(pipe_bar(pp, BAR_S_FULL + b));
-            }
-            for (int t = max(0, tiles - 2); t < tiles; ++t) pipe_wait_one(pp, BAR_S_EMPTY + (t & 1), kTimeoutRole);
-        }
-        __syncwarp();
-    } else if (warp == 18) {
-        // ------------------------------------------------------------------ MMA issuer: products P V
-        if (lane == 0) {
-            const uint32_t idMN = umma_idesc(fmt, 128, 64, 1);
-            const uint64_t dRing = umma_desc_sw128(ring);
-            // + 128 per K-step of an MN-major operand (16 rows of 128 bytes)
+                const uint32_t dd = pp.tmem + TM_S + 128 * b + 64 * m;
+                umma_f16_c<0>(dd, dA, dK, idK);
+                umma_f16_c<1>(dd, dA + 2, dK + 2, idK);
+                umma_f16_c<1>(dd, dA + 4, dK + 4, idK);
+                umma_f16_c<1>(dd, dA + 6, dK + 6, idK);
+                umma_commit(pipe_bar(pp, BAR_S_FULL + 2 * m + b));
+            };
+            pipe_wait_one(pp, BAR_AG, kTimeoutLoads);
+            issue_S(0);
             for (int t = 0; t < tiles; ++t) {
+                if (t + 1 < tiles) issue_S(t + 1);
                 const int s = t % STAGES;
-                pipe_wait_one(pp, BAR_FULL + s, kTimeoutTile);          // long done: the logits of the tile used this stage
-                pipe_wait_one(pp, BAR_P_FULL, kTimeoutRole);
+                pipe_wait_one(pp, BAR_P_FULL + m, kTimeoutRole);
                 tc_fence_after_sync();
                 const int ntok = min(KT, N - (t0 + t) * KT);
                 const uint64_t dV = dRing + (uint64_t)(s * (kStage >> 4)) + (uint64_t)(kTile >> 4);
-                const uint64_t dP = dV + (uint64_t)(kTile >> 4);      // the probabilities replaced the stage's bias tile
-                for (int mb = 0; mb < MB; ++mb)
-                    for (int c = 0; c < 2; ++c) {
-                        if (32 * c >= ntok) break;
-                        const uint32_t dd = pp.tmem + TM_O + 64 * (2 * mb + c);
-                        const uint64_t da = dP + 1024 * mb + 4 * c, db = dV + 256 * c;
-                        if (t > 0) umma_f16_c<1>(dd, da, db, idMN); else umma_f16_c<0>(dd, da, db, idMN);
-                        umma_f16_c<1>(dd, da + 2, db + 128, idMN);
-                    }
+                const uint64_t dP = dV + (uint64_t)(kTile >> 4) + 1024 * m;      // the probabilities replaced the stage's bias tile
+                for (int c = 0; c < 2; ++c) {
+                    if (32 * c >= ntok) break;
+                    const uint32_t dd = pp.tmem + TM_O + 64 * (2 * m + c);
+                    const uint64_t da = dP + 4 * c, db = dV + 256 * c;
+                    if (t > 0) umma_f16_c<1>(dd, da, db, idMN); else umma_f16_c<0>(dd, da, db, idMN);
+                    umma_f16_c<1>(dd, da + 2, db + 128, idMN);
+                }
                 umma_commit(pipe_bar(pp, BAR_EMPTY + s));
-                umma_commit(pipe_bar(pp, BAR_PV));
+                umma_commit(pipe_bar(pp, BAR_PV + m));
             }
+            for (int t = max(0, tiles - 2); t < tiles; ++t) pipe_wait_one(pp, BAR_S_EMPTY + 2 * m + (t & 1), kTimeoutRole);
         }
         __syncwarp();
     } else if ((warp >> 2 & 1) < MB) {
@@ -190,7 +181,7 @@ __global__ void __launch_bounds__(NT, 1) aggregate_umma_kernel(const __grid_cons
         for (int t = 0; t < tiles; ++t) {
             const int b = t & 1, s = t % STAGES;
             const int valid = min(32, N - ((t0 + t) * KT + 32 * c));      // tokens of this thread's half
-            pipe_wait(pp, BAR_S_FULL + b, kTimeoutTile);
+            pipe_wait(pp, BAR_S_FULL + 2 * mb + b, kTimeoutTile);
             tc_fence_after_sync();
             float sv[32];
             {
@@ -198,7 +189,7 @@ __global__ void __launch_bounds__(NT, 1) aggregate_umma_kernel(const __grid_cons
                 tmem_ld32(pp.tmem + TM_S + 128 * b + 64 * mb + 32 * c + lane_base, ra);
                 tmem_ld_wait();
                 tc_fence_before_sync();
-                pipe_arrive(pp, BAR_S_EMPTY + b);
+                pipe_arrive(pp, BAR_S_EMPTY + 2 * mb + b);
                 if (has_bias) {                              // logits in natural units: scale1 * a.k + b1
                     const unsigned char* sB = smem + OFF_RING + s * kStage + 2 * kTile + row * 128;
 #pragma unroll
@@ -256,7 +247,7 @@ __global__ void __launch_bounds__(NT, 1) aggregate_umma_kernel(const __grid_cons
                 started = true;
             }
             // P of the previous tile has been consumed (and every product into this thread's accumulator is done)
-            if (t > 0) { pipe_wait(pp, BAR_PV, kTimeoutTile); tc_fence_after_sync(); }
+            if (t > 0) { pipe_wait(pp, BAR_PV + mb, kTimeoutTile); tc_fence_after_sync(); }
             if (__any_sync(0xffffffffu, resc)) {               // rare: the reference maximum of some row moved
                 uint32_t ra[32];
 #pragma unroll
@@ -277,9 +268,9 @@ __global__ void __launch_bounds__(NT, 1) aggregate_umma_kernel(const __grid_cons
             }
             fence_proxy_async();
             tc_fence_before_sync();
-            pipe_arrive(pp, BAR_P_FULL);
+            pipe_arrive(pp, BAR_P_FULL + mb);
         }
-        pipe_wait(pp, BAR_PV, kTimeoutTile);
+        pipe_wait(pp, BAR_PV + mb, kTimeoutTile);
         tc_fence_after_sync();
         // the two token halves of a row meet in shared memory (the ring is drained: every product is done)
         float o[64];
@@ -301,7 +292,7 @@ __global__ void __launch_bounds__(NT, 1) aggregate_umma_kernel(const __grid_cons
             for (int k = 0; k < 16; ++k) *reinterpret_cast<float4*>(sX + 4 * k) = make_float4(o[4 * k], o[4 * k + 1], o[4 * k + 2], o[4 * k + 3]);
             sX[64] = m_ref; sX[65] = started ? l : 0.f;
         }
-        asm volatile("bar.sync 1, %0;\n" ::"r"(row_threads) : "memory");
+        asm volatile("bar.sync %0, 256;\n" ::"r"(1 + mb) : "memory");      // the chain's own barrier
         if (c == 0) {
             const float om = sX[64], ol = sX[65];
             const float mm = fmaxf(m_ref, om);
