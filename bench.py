@@ -276,19 +276,29 @@ def main():
         for _ in range(2):
             mod.forward_host(pin["q"], pin["k"], pin["v"], w.grid_h, w.grid_w, w.agents, b1=pin["b1"],
                              b2=pin["b2"], dwc_weight=pin["dwc"], out=out_h, stream=stream)
+        # two calls in flight on two streams, each with its own staging and result buffer: the copy back of one
+        # step overlaps the copy in of the next (the copies of a step itself stay in order on its stream)
+        need = mod.staging_bytes(w.grid_h, w.grid_w, w.agents)
+        lanes = [(torch.cuda.Stream(device=dev), torch.empty(need, dtype=torch.uint8, device=dev),
+                  torch.empty_like(pin["q"]).pin_memory()) for _ in range(2)]
         pdist.barrier()
         torch.cuda.synchronize()
         e0.record(stream)
-        for _ in range(args.e2e_steps):
+        for st, _, _ in lanes:
+            st.wait_stream(stream)
+        for i in range(args.e2e_steps):
+            st, stg, oh = lanes[i & 1]
             mod.forward_host(pin["q"], pin["k"], pin["v"], w.grid_h, w.grid_w, w.agents, b1=pin["b1"],
-                             b2=pin["b2"], dwc_weight=pin["dwc"], out=out_h, stream=stream, synchronize=False)
+                             b2=pin["b2"], dwc_weight=pin["dwc"], out=oh, stream=st, synchronize=False, staging=stg)
+        for st, _, _ in lanes:
+            stream.wait_stream(st)
         e1.record(stream)
         torch.cuda.synchronize()
         ms_e2e = pdist.max_over_ranks(e0.elapsed_time(e1)) / args.e2e_steps
         h2d = sum(v.numel() * v.element_size() for v in pin.values() if v is not None)
         e2e = {"value": tokens_per_step / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": out_h.numel() * out_h.element_size(), "ms_per_step": ms_e2e,
-               "steps": args.e2e_steps}
+               "steps": args.e2e_steps, "streams": 2}
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

@@ -267,8 +267,13 @@ class AgentAttention:
         return out
 
     def forward_host(self, q, k, v, grid_h: int, grid_w: int, n_agents: int, agents=None, b1=None, b2=None,
-                     dwc_weight=None, out=None, stream=None, synchronize: bool = True) -> torch.Tensor:
-        """Eq. 6 on host (ideally pinned) tensors: copies in, runs, copies the result back."""
+                     dwc_weight=None, out=None, stream=None, synchronize: bool = True, staging=None) -> torch.Tensor:
+        """Eq. 6 on host (ideally pinned) tensors: copies in, runs, copies the result back.
+
+        Everything is queued on `stream`.  `staging` is the device scratch of the call (uint8, at least
+        `staging_bytes(...)`); calls that are in flight at the same time on different streams (to overlap one
+        step's copies with the next) need a staging buffer each.  By default the module keeps one of its own.
+        """
         B, h, d, N = self.batch, self.heads, self.head_dim, grid_h * grid_w
         for t, nm in ((q, "q"), (k, "k"), (v, "v")):
             self._chk_tensor(t, (B, h, N, d), nm, cuda=False)
@@ -282,14 +287,19 @@ class AgentAttention:
         need = self.staging_bytes(grid_h, grid_w, n_agents)
         if need == 0:
             raise ValueError("shape not supported by this handle")
-        if self._staging is None or self._staging.numel() < need:
-            self._staging = torch.empty(need, dtype=torch.uint8, device=self.device)
+        if staging is not None:
+            if staging.dtype != torch.uint8 or not staging.is_cuda or staging.numel() < need:
+                raise ValueError(f"staging must be a CUDA uint8 tensor of at least {need} bytes")
+        else:
+            if self._staging is None or self._staging.numel() < need:
+                self._staging = torch.empty(need, dtype=torch.uint8, device=self.device)
+            staging = self._staging
         bias = AgentAttnBias(_ptr(b1), _ptr(b2)) if (b1 is not None or b2 is not None) else None
         s = torch.cuda.current_stream() if stream is None else stream
         self._check(self.lib.agent_attn_forward_host(
             self._h, _ptr(q), _ptr(k), _ptr(v), _ptr(agents), grid_h, grid_w, n_agents,
             ctypes.byref(bias) if bias is not None else None, _ptr(dwc_weight), _ptr(out),
-            _ptr(self._staging), self._staging.numel(), ctypes.c_void_p(s.cuda_stream)))
+            _ptr(staging), staging.numel(), ctypes.c_void_p(s.cuda_stream)))
         if synchronize:
             s.synchronize()
         return out
