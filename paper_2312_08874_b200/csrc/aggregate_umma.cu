@@ -64,6 +64,7 @@ constexpr uint32_t TM_S = 0, TM_O = 256;
 struct UmmaAggArgs {
     AttnArgs a;
     int rows_pad, tps;                 // padded agent rows (128 or 256), tiles per split
+    int hf_k, hf_v;                    // dimension order of the K and V maps (tma_load_tok)
     alignas(64) CUtensorMap tm_a, tm_k, tm_v, tm_b;
 };
 }  // namespace
@@ -118,8 +119,8 @@ __global__ void __launch_bounds__(NT, 1) aggregate_umma_kernel(const __grid_cons
                 if (t >= STAGES) pipe_wait_one(pp, BAR_EMPTY + s, kTimeoutRole);
                 const uint32_t bar = pipe_bar(pp, BAR_FULL + s), dst = ring + s * kStage;
                 mbar_arrive_expect_tx(bar, tx);
-                tma_load_2d(dst, &g.tm_k, 0, slab * N + c0, bar);
-                tma_load_2d(dst + kTile, &g.tm_v, 0, slab * N + c0, bar);
+                tma_load_tok(dst, &g.tm_k, g.hf_k, c0, head, slab / p.heads, bar);
+                tma_load_tok(dst + kTile, &g.tm_v, g.hf_v, c0, head, slab / p.heads, bar);
                 if (has_bias)
                     for (int mb = 0; mb < MB; ++mb) tma_load_2d(dst + 2 * kTile + mb * 2 * kTile, &g.tm_b, c0, head * n + 128 * mb, bar);
             }
@@ -402,8 +403,9 @@ cudaError_t launch_aggregate_umma(int dtype, const AttnArgs& p, const AggPlan& p
     g.tps = (tiles + plan.splits - 1) / plan.splits;
     const uint64_t S = p.slabs, N = p.cols, n = p.rows;
     if (!make_map_2d_u16(&g.tm_a, p.qm, S * n, p.d, 128, 64)) return cudaErrorNotSupported;
-    if (!make_map_2d_u16(&g.tm_k, p.km, S * N, p.d, 64, 64)) return cudaErrorNotSupported;
-    if (!make_map_2d_u16(&g.tm_v, p.vm, S * N, p.d, 64, 64)) return cudaErrorNotSupported;
+    const int batch = p.slabs / p.heads;
+    if (!make_map_tok_u16(&g.tm_k, &g.hf_k, p.km, p.lin, batch, p.heads, (long long)N, p.d, 64, true)) return cudaErrorNotSupported;
+    if (!make_map_tok_u16(&g.tm_v, &g.hf_v, p.vm, p.lin, batch, p.heads, (long long)N, p.d, 64, true)) return cudaErrorNotSupported;
     if (p.bias && !make_map_2d_u16(&g.tm_b, p.bias, (uint64_t)p.heads * n, N, 128, 64)) return cudaErrorNotSupported;
     if (dtype == kBF16) return launch_umma_t<__nv_bfloat16>(g, st);
     if (dtype == kF16) return launch_umma_t<__half>(g, st);

@@ -99,11 +99,26 @@ int isqrt_exact(int n) {
     return (p * p == n) ? p : -1;
 }
 
-int do_pool(agent_attn_handle* h, const void* Q, int gh, int gw, int ph, int pw, void* A, cudaStream_t st) {
+// Layouts of the token-major tensors of a call: Q, K and V share `in`, O has `out`.
+struct CallLayout {
+    TokLayout in, out;
+    bool strided;
+};
+CallLayout dense_call(const agent_attn_handle* h, int n_tokens) {
+    CallLayout l;
+    l.in = l.out = dense_layout(h->cfg.heads, n_tokens, h->cfg.head_dim);
+    l.strided = false;
+    return l;
+}
+
+int do_pool(agent_attn_handle* h, const void* Q, int gh, int gw, int ph, int pw, void* A, cudaStream_t st,
+            const CallLayout* cl = nullptr) {
     PoolArgs pa;
     pa.q = Q; pa.a = A;
     pa.slabs = h->cfg.batch * h->cfg.heads;
     pa.H = gh; pa.W = gw; pa.d = h->cfg.head_dim; pa.ph = ph; pa.pw = pw;
+    pa.heads = h->cfg.heads;
+    pa.lq = cl ? cl->in : dense_layout(h->cfg.heads, (long long)gh * gw, h->cfg.head_dim);
     cudaError_t e = launch_pool(h->cfg.dtype, pa, st);
     if (e != cudaSuccess) return fail(h, AA_ERR_CUDA, "pool launch failed: %s", cudaGetErrorString(e));
     h->launches++;
@@ -111,7 +126,10 @@ int do_pool(agent_attn_handle* h, const void* Q, int gh, int gw, int ph, int pw,
 }
 
 int do_aggregate(agent_attn_handle* h, const void* A, const void* K, const void* V, const void* b1,
-                 int N, int n, void* VA, float* partials, unsigned* tickets, cudaStream_t st) {
+                 int N, int n, void* VA, float* partials, unsigned* tickets, cudaStream_t st,
+                 const CallLayout* cl = nullptr) {
+    if (cl && cl->strided && !use_umma(h, N, n))
+        return fail(h, AA_ERR_UNSUPPORTED, "strided K and V need the fused or the tensor-memory kernels (16-bit, d <= 64, n <= 256)");
     const AggPlan pl = plan_for(h, N, n);
     cudaError_t e = cudaMemsetAsync(tickets, 0, (size_t)h->cfg.batch * h->cfg.heads * sizeof(unsigned), st);
     if (e != cudaSuccess) return fail(h, AA_ERR_CUDA, "ticket reset failed: %s", cudaGetErrorString(e));
@@ -123,6 +141,9 @@ int do_aggregate(agent_attn_handle* h, const void* A, const void* K, const void*
     a.rows = n; a.cols = N; a.d = h->cfg.head_dim;
     a.scale = h->scale1; a.splits = pl.splits;
     a.status = h->d_status;
+    a.lin = cl ? cl->in : dense_layout(h->cfg.heads, N, h->cfg.head_dim);
+    a.lout = a.lin;
+    a.strided = cl && cl->strided;
     e = use_umma(h, N, n) ? launch_aggregate_umma(h->cfg.dtype, a, pl, st)
         : use_simt(h)     ? launch_aggregate_simt(h->cfg.dtype, a, pl, st)
                           : launch_aggregate_mma(h->cfg.dtype, a, pl, st);
@@ -132,7 +153,8 @@ int do_aggregate(agent_attn_handle* h, const void* A, const void* K, const void*
 }
 
 int do_broadcast(agent_attn_handle* h, const void* Q, const void* A, const void* VA, const void* V,
-                 const void* b2, const void* wd, int gh, int gw, int n, void* out, cudaStream_t st) {
+                 const void* b2, const void* wd, int gh, int gw, int n, void* out, cudaStream_t st,
+                 const CallLayout* cl = nullptr) {
     AttnArgs a;
     memset(&a, 0, sizeof(a));
     a.qm = Q; a.km = A; a.vm = VA; a.bias = b2; a.out = out;
@@ -141,8 +163,13 @@ int do_broadcast(agent_attn_handle* h, const void* Q, const void* A, const void*
     a.scale = h->scale2; a.splits = 1;
     a.dwc_v = wd ? V : nullptr; a.dwc_w = wd; a.H = gh; a.W = gw;
     a.status = h->d_status;
+    a.lin = cl ? cl->in : dense_layout(h->cfg.heads, (long long)gh * gw, h->cfg.head_dim);
+    a.lout = cl ? cl->out : a.lin;
+    a.strided = cl && cl->strided;
     const bool umma = !use_simt(h) && h->cfg.path == AA_PATH_AUTO &&
                       broadcast_umma_eligible(h->cfg.dtype, n, gh * gw, h->cfg.head_dim);
+    if (a.strided && !umma)
+        return fail(h, AA_ERR_UNSUPPORTED, "strided Q, V and out need the fused or the tensor-memory kernels (16-bit, d <= 64, n a multiple of 8 up to 256)");
     cudaError_t e = umma          ? launch_broadcast_umma(h->cfg.dtype, a, h->sm_count, st)
                     : use_simt(h) ? launch_broadcast_simt(h->cfg.dtype, a, st)
                                   : launch_broadcast_mma(h->cfg.dtype, a, st);
@@ -281,9 +308,11 @@ int agent_attn_broadcast(agent_attn_handle* h, const void* Q, const void* A, con
     return do_broadcast(h, Q, A, VA, V, b2, dwc_weight, grid_h, grid_w, n_agents, out, (cudaStream_t)stream);
 }
 
-int agent_attn_forward(agent_attn_handle* h, const void* Q, const void* K, const void* V, const void* A,
-                       int grid_h, int grid_w, int n_agents, const agent_attn_bias* bias, const void* dwc_weight,
-                       void* out, void* workspace, size_t workspace_bytes, void* stream) {
+static bool fused_layout_ok(const CallLayout& cl) { return !cl.strided; }
+
+static int forward_impl(agent_attn_handle* h, const void* Q, const void* K, const void* V, const void* A,
+                        int grid_h, int grid_w, int n_agents, const agent_attn_bias* bias, const void* dwc_weight,
+                        void* out, void* workspace, size_t workspace_bytes, void* stream, const CallLayout* clp) {
     if (!h) return AA_ERR_INVALID_ARG;
     h->err[0] = 0;
     if (!Q || !K || !V || !out || !workspace) return fail(h, AA_ERR_INVALID_ARG, "null pointer");
@@ -314,6 +343,7 @@ int agent_attn_forward(agent_attn_handle* h, const void* Q, const void* K, const
     h->launches = 0;
     cudaStream_t st = (cudaStream_t)stream;
     char* ws = static_cast<char*>(workspace);
+    const CallLayout cl = clp ? *clp : dense_call(h, N);
     if (!A && h->cfg.path == AA_PATH_AUTO && h->cfg.dtype != AA_F32) {
         // one persistent kernel for the whole module where the shape allows it
         if (h->fused_key[0] != grid_h || h->fused_key[1] != grid_w || h->fused_key[2] != n_agents) {
@@ -321,7 +351,7 @@ int agent_attn_forward(agent_attn_handle* h, const void* Q, const void* K, const
                                        n_agents, h->sm_count);
             h->fused_key[0] = grid_h; h->fused_key[1] = grid_w; h->fused_key[2] = n_agents;
         }
-        if (h->fused_plan.ok) {
+        if (h->fused_plan.ok && fused_layout_ok(cl)) {
             const int slabs = h->cfg.batch * h->cfg.heads;
             unsigned* counters = reinterpret_cast<unsigned*>(ws + w.ticket_off);
             cudaError_t e = cudaMemsetAsync(counters, 0, fused_counter_words(slabs) * sizeof(unsigned), st);
@@ -334,6 +364,7 @@ int agent_attn_forward(agent_attn_handle* h, const void* Q, const void* K, const
             fa.counters = counters; fa.status = h->d_status;
             fa.slabs = slabs; fa.heads = h->cfg.heads; fa.H = grid_h; fa.W = grid_w; fa.d = h->cfg.head_dim;
             fa.n = n_agents; fa.p = p; fa.scale1 = h->scale1; fa.scale2 = h->scale2; fa.plan = h->fused_plan;
+            fa.lin = cl.in; fa.lout = cl.out;
             if (!fused_make_maps(&fa)) return fail(h, AA_ERR_CUDA, "tensor map encoding failed");
             e = launch_fused(h->cfg.dtype, fa, st);
             if (e != cudaSuccess) return fail(h, AA_ERR_CUDA, "fused launch failed: %s", cudaGetErrorString(e));
@@ -343,14 +374,46 @@ int agent_attn_forward(agent_attn_handle* h, const void* Q, const void* K, const
     }
     const void* agents = A;
     if (!A) {
-        if (int rc = do_pool(h, Q, grid_h, grid_w, p, p, ws + w.a_off, st)) return rc;
+        if (int rc = do_pool(h, Q, grid_h, grid_w, p, p, ws + w.a_off, st, &cl)) return rc;
         agents = ws + w.a_off;
     }
     void* va = ws + w.va_off;
     if (int rc = do_aggregate(h, agents, K, V, b1, N, n_agents, va, reinterpret_cast<float*>(ws + w.part_off),
-                              reinterpret_cast<unsigned*>(ws + w.ticket_off), st))
+                              reinterpret_cast<unsigned*>(ws + w.ticket_off), st, &cl))
         return rc;
-    return do_broadcast(h, Q, agents, va, V, b2, dwc_weight, grid_h, grid_w, n_agents, out, st);
+    return do_broadcast(h, Q, agents, va, V, b2, dwc_weight, grid_h, grid_w, n_agents, out, st, &cl);
+}
+
+int agent_attn_forward(agent_attn_handle* h, const void* Q, const void* K, const void* V, const void* A,
+                       int grid_h, int grid_w, int n_agents, const agent_attn_bias* bias, const void* dwc_weight,
+                       void* out, void* workspace, size_t workspace_bytes, void* stream) {
+    return forward_impl(h, Q, K, V, A, grid_h, grid_w, n_agents, bias, dwc_weight, out, workspace, workspace_bytes,
+                        stream, nullptr);
+}
+
+int agent_attn_forward_strided(agent_attn_handle* h, const void* Q, const void* K, const void* V, const void* A,
+                               const long long in_strides[3], int grid_h, int grid_w, int n_agents,
+                               const agent_attn_bias* bias, const void* dwc_weight, void* out,
+                               const long long out_strides[3], void* workspace, size_t workspace_bytes, void* stream) {
+    if (!h) return AA_ERR_INVALID_ARG;
+    h->err[0] = 0;
+    if (!in_strides || !out_strides) return fail(h, AA_ERR_INVALID_ARG, "null stride array");
+    if (grid_h <= 0 || grid_w <= 0) return fail(h, AA_ERR_INVALID_ARG, "grid must be positive");
+    const long long N = (long long)grid_h * grid_w, d = h->cfg.head_dim;
+    CallLayout cl;
+    cl.in.sb = in_strides[0]; cl.in.sh = in_strides[1]; cl.in.st = in_strides[2];
+    cl.out.sb = out_strides[0]; cl.out.sh = out_strides[1]; cl.out.st = out_strides[2];
+    for (const TokLayout* l : {&cl.in, &cl.out}) {
+        if (l->sb <= 0 || l->sh <= 0 || l->st < d)
+            return fail(h, AA_ERR_INVALID_ARG, "strides must be positive and the token stride at least head_dim");
+        if ((l->sb * h->elem_bytes) % 16 || (l->sh * h->elem_bytes) % 16 || (l->st * h->elem_bytes) % 16)
+            return fail(h, AA_ERR_INVALID_ARG, "strides must be multiples of 16 bytes");
+    }
+    const TokLayout dl = dense_layout(h->cfg.heads, N, (int)d);
+    auto same = [](const TokLayout& a, const TokLayout& b) { return a.sb == b.sb && a.sh == b.sh && a.st == b.st; };
+    cl.strided = !(same(cl.in, dl) && same(cl.out, dl));
+    return forward_impl(h, Q, K, V, A, grid_h, grid_w, n_agents, bias, dwc_weight, out, workspace, workspace_bytes,
+                        stream, &cl);
 }
 
 int agent_attn_compose_bias(agent_attn_handle* h, const void* col, const void* row, const void* blk, int block_h,

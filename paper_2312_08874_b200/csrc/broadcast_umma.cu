@@ -70,7 +70,8 @@ constexpr uint32_t TM_S = 0, TM_O = 256;
 struct UmmaBcArgs {
     AttnArgs a;
     int MB, tps;                       // 128-agent blocks (1 or 2), tiles per split
-    alignas(64) CUtensorMap tm_q, tm_a, tm_va, tm_b, tm_h;     // tm_h: V as [slabs*N][d] with 136-row boxes
+    int hf_q, hf_h;                    // dimension order of the Q and V maps (tma_load_tok)
+    alignas(64) CUtensorMap tm_q, tm_a, tm_va, tm_b, tm_h;     // tm_h: V with 136-token boxes
 };
 }  // namespace
 
@@ -127,14 +128,14 @@ __global__ void __launch_bounds__(NT, 1) broadcast_umma_kernel(const __grid_cons
                 const int tok0 = (i0 + i) * QT;
                 if (i >= 2) pipe_wait_one(pp, BAR_Q_EMPTY + (i & 1), kTimeoutRole);
                 mbar_arrive_expect_tx(pipe_bar(pp, BAR_Q_FULL + (i & 1)), 2 * kTile);
-                tma_load_2d(sQ + (i & 1) * 2 * kTile, &g.tm_q, 0, slab * N + tok0, pipe_bar(pp, BAR_Q_FULL + (i & 1)));
+                tma_load_tok(sQ + (i & 1) * 2 * kTile, &g.tm_q, g.hf_q, tok0, head, slab / p.heads, pipe_bar(pp, BAR_Q_FULL + (i & 1)));
                 if (has_dwc) {
                     // runs of tokens one grid row above, around and below the tile, each from one token before
-                    // it (rows outside the tensor are zero-filled; tokens of other slabs are masked by the readers)
+                    // it (tokens outside the slab are zero-filled)
                     if (i >= 1) pipe_wait_one(pp, BAR_H_EMPTY, kTimeoutRole);
                     mbar_arrive_expect_tx(pipe_bar(pp, BAR_H_FULL), 3 * kHaloSeg);
                     for (int u = 0; u < 3; ++u)
-                        tma_load_2d(sH + u * kHaloSeg, &g.tm_h, 0, slab * N + tok0 + (u - 1) * p.W - 1, pipe_bar(pp, BAR_H_FULL));
+                        tma_load_tok(sH + u * kHaloSeg, &g.tm_h, g.hf_h, tok0 + (u - 1) * p.W - 1, head, slab / p.heads, pipe_bar(pp, BAR_H_FULL));
                 }
                 if (has_b2)
                     for (int a = 0; a < MB; ++a) {
@@ -230,7 +231,8 @@ __global__ void __launch_bounds__(NT, 1) broadcast_umma_kernel(const __grid_cons
         asm volatile("bar.sync 1, %0;\n" ::"n"(NROW) : "memory");
         if (tid == 0) pipe_arrive(pp, BAR_PREP);
 
-        T* gO = static_cast<T*>(p.out) + (size_t)slab * N * d;
+        T* gO = static_cast<T*>(p.out) + tok_offset(p.lout, slab, p.heads, 0);
+        const size_t so = (size_t)p.lout.st;
         for (int i = 0; i < tiles; ++i) {
             const int tok = (i0 + i) * QT + row;
             float m_ref = -INFINITY, l = 0.f;
@@ -398,11 +400,11 @@ __global__ void __launch_bounds__(NT, 1) broadcast_umma_kernel(const __grid_cons
                     float o8[8];
 #pragma unroll
                     for (int k = 0; k < 8; ++k) o8[k] = fmaf(acc[k], inv, (k & 1) ? dw[k >> 1].y : dw[k >> 1].x);
-                    *reinterpret_cast<uint4*>(gO + (size_t)tok * d + c0) = pack16<T>(o8);
+                    *reinterpret_cast<uint4*>(gO + (size_t)tok * so + c0) = pack16<T>(o8);
                     if (nch > 8) {
 #pragma unroll
                         for (int k = 0; k < 8; ++k) o8[k] = fmaf(acc[8 + k], inv, (k & 1) ? dw[4 + (k >> 1)].y : dw[4 + (k >> 1)].x);
-                        *(reinterpret_cast<uint4*>(gO + (size_t)tok * d + c0) + 1) = pack16<T>(o8);
+                        *(reinterpret_cast<uint4*>(gO + (size_t)tok * so + c0) + 1) = pack16<T>(o8);
                     }
                 }
             }
@@ -443,11 +445,12 @@ cudaError_t launch_broadcast_umma(int dtype, const AttnArgs& p, int sm_count, cu
     g.tps = (tiles + splits - 1) / splits;
     splits = (tiles + g.tps - 1) / g.tps;
     const uint64_t S = p.slabs, N = p.rows, n = p.cols;
-    if (!make_map_2d_u16(&g.tm_q, p.qm, S * N, p.d, 128, 64)) return cudaErrorNotSupported;
+    const int batch = p.slabs / p.heads;
+    if (!make_map_tok_u16(&g.tm_q, &g.hf_q, p.qm, p.lin, batch, p.heads, (long long)N, p.d, 128, true)) return cudaErrorNotSupported;
     if (!make_map_2d_u16(&g.tm_a, p.km, S * n, p.d, 128, 64)) return cudaErrorNotSupported;
     if (!make_map_2d_u16(&g.tm_va, p.vm, S * n, p.d, 128, 64)) return cudaErrorNotSupported;
     if (p.bias && !make_map_2d_u16(&g.tm_b, p.bias, (uint64_t)p.heads * N, n, 128, 64)) return cudaErrorNotSupported;
-    if (p.dwc_w && !make_map_2d_u16(&g.tm_h, p.dwc_v, S * N, p.d, kHaloRows, 64)) return cudaErrorNotSupported;
+    if (p.dwc_w && !make_map_tok_u16(&g.tm_h, &g.hf_h, p.dwc_v, p.lin, batch, p.heads, (long long)N, p.d, kHaloRows, true)) return cudaErrorNotSupported;
     if (dtype == kBF16) return launch_bc_umma_t<__nv_bfloat16>(g, splits, st);
     if (dtype == kF16) return launch_bc_umma_t<__half>(g, splits, st);
     return cudaErrorInvalidValue;

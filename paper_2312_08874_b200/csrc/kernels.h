@@ -10,6 +10,21 @@ namespace aa {
 
 enum DType { kF32 = 0, kBF16 = 1, kF16 = 2 };
 
+// Strides of a [batch, head, token, d] tensor in elements (d contiguous).  Dense [B, h, N, d] is
+// {h N d, N d, d}; the output of a fused projection kept as [B, N, h, d] is {N h d, d, h d}.
+struct TokLayout {
+    long long sb, sh, st;
+};
+inline TokLayout dense_layout(int heads, long long n_tokens, int d) {
+    TokLayout l;
+    l.sb = (long long)heads * n_tokens * d; l.sh = n_tokens * d; l.st = d;
+    return l;
+}
+__host__ __device__ inline long long tok_offset(const TokLayout& l, int slab, int heads, long long tok) {
+    return (long long)(slab / heads) * l.sb + (long long)(slab % heads) * l.sh + tok * l.st;
+}
+
+
 // Split-partial layout.  One partial per (slab, part): m[rows_pad], l[rows_pad],
 // acc[rows_pad][dpad], all fp32, with m and the logits in log2 units (logit * log2(e)), so the
 // merge weights are exp2(m_j - m).
@@ -22,6 +37,8 @@ struct PoolArgs {
     const void* q;      // [slabs][H*W][d]
     void* a;            // [slabs][ph*pw][d]
     int slabs, H, W, d, ph, pw;
+    int heads;          // slab = batch item * heads + head
+    TokLayout lq;       // strides of q
 };
 cudaError_t launch_pool(int dtype, const PoolArgs& p, cudaStream_t st);
 
@@ -52,6 +69,10 @@ struct AttnArgs {
     const void* dwc_w;    // broadcast only: [heads][d][3][3] or nullptr
     int H, W;             // broadcast only: token grid
     int* status;          // device status word for bounded waits (tensor-memory kernels), may be null
+    // token-major tensors of the call ([batch, head, token, d] with strides): aggregation K and V; broadcast Q,
+    // the V of the depthwise term, and out.  The agent-side tensors (A, V_A) are dense [slabs][n][d].
+    TokLayout lin, lout;
+    int strided;          // lin or lout is not the dense layout (only the kernels that read strides may run)
 };
 
 // Plan of the aggregation launch for a problem shape (used for workspace sizing too).
@@ -104,6 +125,7 @@ struct FusedArgs {
     int* status;          // device status word: set when a bounded wait gives up
     int slabs, heads, H, W, d, n, p;
     float scale1, scale2;
+    TokLayout lin, lout;  // strides of Q, K, V and of out
     FusedPlan plan;
     // TMA descriptors (128-byte swizzle, 64-column boxes): K and V as [slabs*N][d] with 64-row boxes,
     // B1 as [heads*n][N] with 64x64 boxes, A and V_A workspaces as [slabs*n][d] with 64-row boxes

@@ -25,7 +25,7 @@ __global__ void __launch_bounds__(256) pool_kernel(PoolArgs p) {
     const int cpt = p.d / VEC;                    // 16-byte chunks per token
     const int tpl = 32 / cpt;                     // tokens covered by one warp-wide load
     const int cg = lane % cpt, tsub = lane / cpt;
-    const T* q = static_cast<const T*>(p.q) + (size_t)slab * p.H * p.W * p.d;
+    const T* q = static_cast<const T*>(p.q) + tok_offset(p.lq, slab, p.heads, 0);
 
     float acc[VEC];
 #pragma unroll
@@ -35,7 +35,7 @@ __global__ void __launch_bounds__(256) pool_kernel(PoolArgs p) {
         for (int i = tsub; i < cnt; i += tpl) {
             const int wy = i / ww, wx = i - wy * ww;
             const size_t tok = (size_t)(y0 + wy) * p.W + (x0 + wx);
-            const uint4 raw = __ldg(reinterpret_cast<const uint4*>(q + tok * p.d) + cg);
+            const uint4 raw = __ldg(reinterpret_cast<const uint4*>(q + tok * (size_t)p.lq.st) + cg);
             float f[VEC];
             unpack16<T>(raw, f);
 #pragma unroll
