@@ -273,6 +273,8 @@ __global__ void __launch_bounds__(NT, 1) aggregate_umma_kernel(const __grid_cons
         }
         pipe_wait(pp, BAR_PV + mb, kTimeoutTile);
         tc_fence_after_sync();
+        // both chains are through with the ring before its memory is reused for the exchange below
+        asm volatile("bar.sync 3, %0;\n" ::"r"(256 * MB) : "memory");
         // the two token halves of a row meet in shared memory (the ring is drained: every product is done)
         float o[64];
         {
