@@ -155,6 +155,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
     ap.add_argument("--e2e-steps", type=int, default=10)
+    ap.add_argument("--layout", choices=["dense", "bnhd", "qkv"], default="dense",
+                    help="storage of Q, K, V and out: dense [B,h,N,d]; bnhd = [B,N,h,d] (forward_strided); "
+                         "qkv = Q, K, V interleaved as [B,N,3,h,d], out [B,N,h,d] (forward_strided)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--min-warmup-seconds", type=float, default=0.2)
     args = ap.parse_args()
@@ -186,6 +189,15 @@ def main():
             for k in ("q", "k", "v"):
                 d[k] = torch.roll(d[k], roll, dims=2).contiguous()
         d["out"] = torch.empty_like(d["q"])
+        if args.layout != "dense":      # the same values behind token-major storage; views keep the [B,h,N,d] shape
+            if args.layout == "qkv":
+                packed = torch.stack([d[k].permute(0, 2, 1, 3) for k in ("q", "k", "v")], dim=2).contiguous()
+                for j, k in enumerate(("q", "k", "v")):
+                    d[k] = packed[:, :, j].permute(0, 2, 1, 3)
+            else:
+                for k in ("q", "k", "v"):
+                    d[k] = d[k].permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+            d["out"] = torch.empty((w.batch, w.tokens, w.heads, w.head_dim), dtype=dt, device=dev).permute(0, 2, 1, 3)
         sets.append(d)
     mod = AgentAttention(w.batch, w.heads, w.head_dim, w.tokens, w.agents, dt, device=local_rank)
     ws = mod.workspace(w.grid_h, w.grid_w, w.agents)
@@ -193,8 +205,9 @@ def main():
 
     def step(i):
         d = sets[i % n_sets]
-        mod.forward(d["q"], d["k"], d["v"], w.grid_h, w.grid_w, w.agents, b1=d["b1"], b2=d["b2"],
-                    dwc_weight=d["dwc"], out=d["out"], workspace=ws, stream=stream)
+        fwd = mod.forward if args.layout == "dense" else mod.forward_strided
+        fwd(d["q"], d["k"], d["v"], w.grid_h, w.grid_w, w.agents, b1=d["b1"], b2=d["b2"],
+            dwc_weight=d["dwc"], out=d["out"], workspace=ws, stream=stream)
 
     # warm-up: W steps, and at least 0.2 s so that clocks have ramped
     t_w = time.perf_counter()
@@ -228,7 +241,12 @@ def main():
     unit = w.slabs * w.tokens * w.head_dim * s                       # one [B,h,N,d] tensor
     bias_b = w.heads * w.agents * w.tokens * s if w.bias else 0
     peak, peak_src = measured_peaks()
-    if launches_per_step == 1:
+    if launches_per_step != 1 and args.layout != "dense":
+        # the step-level entry points take dense tensors only: report the whole path as one unit
+        dominant = "forward_path"
+        kern_ms = {dominant: ms_step}
+        kern_bytes = {dominant: set_bytes}
+    elif launches_per_step == 1:
         # the whole path is one persistent kernel: its launch duration is the step time (the only other
         # node on the stream is a few-hundred-byte memset), its algorithmic bytes are the path's
         dominant = "fused_kernel"
@@ -322,7 +340,7 @@ def main():
             "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
             "config": {"workload": w.name, "batch_per_gpu": w.batch, "heads": w.heads, "tokens": w.tokens,
                        "grid": [w.grid_h, w.grid_w], "head_dim": w.head_dim, "agents": w.agents,
-                       "bias": w.bias, "dwc": w.dwc,
+                       "bias": w.bias, "dwc": w.dwc, "layout": args.layout,
                        "l2": f"{n_sets} rotating buffer sets of {set_bytes / 1e6:.1f} MB (> 4x the 126 MB L2)",
                        "parallelism": f"batch-sharded x{world}, no collective"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,

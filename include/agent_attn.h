@@ -114,6 +114,29 @@ int agent_attn_forward(agent_attn_handle* h,
                        const agent_attn_bias* bias, const void* dwc_weight,
                        void* out, void* workspace, size_t workspace_bytes, void* stream);
 
+/* The whole module, Eq. 6, on token-major tensors with explicit strides (Eq. 1 computes Q, K and V with one
+ * projection per token: its output, kept as [B][N][heads][d] or interleaved as [B][N][3][heads][d], is read
+ * in place, and O can be written as [B][N][heads][d] for the projection that follows).
+ *   Q, K, V      device; element (b, head, token, c) of each at
+ *                base + b * in_strides[0] + head * in_strides[1] + token * in_strides[2] + c
+ *   in_strides   host, 3 values in ELEMENTS: batch, head, token stride shared by Q, K and V (the d channels of
+ *                a token are contiguous); each a multiple of 16 bytes, token stride >= head_dim
+ *   out          device; element (b, head, token, c) at base + b * out_strides[0] + head * out_strides[1]
+ *                + token * out_strides[2] + c
+ *   everything else as in agent_attn_forward (A, biases and the filter are dense).
+ * Dense strides {heads*N*d, N*d, d} make this call identical to agent_attn_forward.  Other strides run on the
+ * fused and the tensor-memory kernels only: AA_ERR_UNSUPPORTED for fp32, head_dim > 64 (or != 64 with
+ * n_agents <= 64), caller-supplied A with n_agents <= 64, n_agents > 64 not a multiple of 8, N not a multiple
+ * of 8 with a bias, and handles created with a path other than AA_PATH_AUTO.  Other errors as in
+ * agent_attn_forward.  No host synchronisation, no allocation. */
+int agent_attn_forward_strided(agent_attn_handle* h,
+                               const void* Q, const void* K, const void* V, const void* A,
+                               const long long in_strides[3],
+                               int grid_h, int grid_w, int n_agents,
+                               const agent_attn_bias* bias, const void* dwc_weight,
+                               void* out, const long long out_strides[3],
+                               void* workspace, size_t workspace_bytes, void* stream);
+
 /* Step 1 alone: agent tokens by pooling (text under Eq. 6).  Q device [B][heads][N][d] ->
  * A_out device [B][heads][n][d], n = pool_h * pool_w, windows as described above. */
 int agent_attn_pool(agent_attn_handle* h, const void* Q, int grid_h, int grid_w,

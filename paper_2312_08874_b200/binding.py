@@ -25,7 +25,7 @@ EXPORTS = [
     "agent_attn_forward", "agent_attn_pool", "agent_attn_aggregate", "agent_attn_broadcast",
     "agent_attn_staging_bytes", "agent_attn_forward_host", "agent_attn_query_status",
     "agent_attn_last_launch_count", "agent_attn_aggregate_static", "agent_attn_static_scratch_bytes",
-    "agent_attn_compose_bias",
+    "agent_attn_compose_bias", "agent_attn_forward_strided",
 ]
 
 
@@ -75,6 +75,10 @@ def load_library(build_if_missing: bool = True) -> ctypes.CDLL:
     lib.agent_attn_forward.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ctypes.POINTER(AgentAttnBias), vp,
                                        vp, vp, sz, vp]
     lib.agent_attn_forward.restype = ci
+    ll3 = ctypes.POINTER(ctypes.c_longlong)
+    lib.agent_attn_forward_strided.argtypes = [vp, vp, vp, vp, vp, ll3, ci, ci, ci, ctypes.POINTER(AgentAttnBias), vp,
+                                               vp, ll3, vp, ctypes.c_size_t, vp]
+    lib.agent_attn_forward_strided.restype = ci
     lib.agent_attn_pool.argtypes = [vp, vp, ci, ci, ci, ci, vp, vp]
     lib.agent_attn_pool.restype = ci
     lib.agent_attn_aggregate.argtypes = [vp, vp, vp, vp, vp, ci, ci, vp, vp, sz, vp]
@@ -186,6 +190,38 @@ class AgentAttention:
         self._check(self.lib.agent_attn_forward(
             self._h, _ptr(q), _ptr(k), _ptr(v), _ptr(agents), grid_h, grid_w, n_agents,
             ctypes.byref(bias) if bias is not None else None, _ptr(dwc_weight), _ptr(out), _ptr(ws),
+            ws.numel(), _stream_ptr(stream)))
+        return out
+
+    def forward_strided(self, q, k, v, grid_h: int, grid_w: int, n_agents: int, agents=None, b1=None, b2=None,
+                        dwc_weight=None, out=None, workspace=None, stream=None) -> torch.Tensor:
+        """Eq. 6 on VIEWS of shape [B, heads, N, d] with any batch / head / token strides (last dim contiguous).
+
+        Typical use: `qkv` of shape [B, N, 3, heads, d] straight from a projection, passed as
+        `qkv[:, :, i].permute(0, 2, 1, 3)`; `out` may be such a view of a [B, N, heads, d] tensor (that is
+        what is allocated when `out` is None).  Q, K and V must share their strides.
+        """
+        B, h, d, N = self.batch, self.heads, self.head_dim, grid_h * grid_w
+        for t, nm in ((q, "q"), (k, "k"), (v, "v"), (out, "out")):
+            if t is None:
+                continue
+            if tuple(t.shape) != (B, h, N, d) or t.dtype != self.dtype or not t.is_cuda or t.stride(3) != 1:
+                raise ValueError(f"{nm}: expected a cuda {self.dtype} view of shape {(B, h, N, d)} with contiguous channels")
+        if q.stride() != k.stride() or q.stride() != v.stride():
+            raise ValueError("q, k and v must have the same strides")
+        self._chk_tensor(agents, (B, h, n_agents, d), "agents")
+        self._chk_tensor(b1, (h, n_agents, N), "b1")
+        self._chk_tensor(b2, (h, N, n_agents), "b2")
+        self._chk_tensor(dwc_weight, (h, d, 3, 3), "dwc_weight")
+        if out is None:
+            out = torch.empty((B, N, h, d), dtype=self.dtype, device=self.device).permute(0, 2, 1, 3)
+        ws = self.workspace(grid_h, grid_w, n_agents) if workspace is None else workspace
+        bias = AgentAttnBias(_ptr(b1), _ptr(b2)) if (b1 is not None or b2 is not None) else None
+        sin = (ctypes.c_longlong * 3)(q.stride(0), q.stride(1), q.stride(2))
+        sout = (ctypes.c_longlong * 3)(out.stride(0), out.stride(1), out.stride(2))
+        self._check(self.lib.agent_attn_forward_strided(
+            self._h, _ptr(q), _ptr(k), _ptr(v), _ptr(agents), sin, grid_h, grid_w, n_agents,
+            ctypes.byref(bias) if bias is not None else None, _ptr(dwc_weight), _ptr(out), sout, _ptr(ws),
             ws.numel(), _stream_ptr(stream)))
         return out
 

@@ -308,7 +308,7 @@ int agent_attn_broadcast(agent_attn_handle* h, const void* Q, const void* A, con
     return do_broadcast(h, Q, A, VA, V, b2, dwc_weight, grid_h, grid_w, n_agents, out, (cudaStream_t)stream);
 }
 
-static bool fused_layout_ok(const CallLayout& cl) { return !cl.strided; }
+static bool fused_layout_ok(const CallLayout&) { return true; }
 
 static int forward_impl(agent_attn_handle* h, const void* Q, const void* K, const void* V, const void* A,
                         int grid_h, int grid_w, int n_agents, const agent_attn_bias* bias, const void* dwc_weight,

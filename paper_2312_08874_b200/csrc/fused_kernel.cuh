@@ -109,6 +109,14 @@ __device__ __forceinline__ int swz(int row, int col) {
     return row * 128 + ((((col >> 3) ^ row) & 7) << 4) + (col & 7) * 2;
 }
 
+// Tile of `box` tokens from token `tok` of slab (b, head): a 2-D map over [slabs * N][d] when the tensor is
+// dense (rows past the slab then belong to the next slab: the readers mask them), else the 4-D strided map.
+__device__ __forceinline__ void load_tokens(uint32_t dst, const CUtensorMap* map, int dense, int head_first, int tok,
+                                            int head, int b, int row0, uint32_t bar) {
+    if (dense) tma_load_2d(dst, map, 0, row0 + tok, bar);
+    else tma_load_tok(dst, map, head_first, tok, head, b, bar);
+}
+
 // Optional per-task phase timestamps (debug builds only): define AA_FUSED_TRACE and hand a device
 // buffer to aa_fused_trace_buffer; record i of a block goes to slot (blockIdx, i).
 #ifdef AA_FUSED_TRACE
@@ -177,7 +185,9 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
     unsigned char* sA = smem + OFF_A;
     unsigned char* ring = smem + OFF_UNION;
     const uint32_t ring_u32 = smem_u32(ring);
-    const T* gQ = static_cast<const T*>(p.q) + (size_t)slab * N * DK;
+    // the shape-specialised kernels serve dense tensors only: their strides are compile-time constants
+    const T* gQ = static_cast<const T*>(p.q) + (SH::kFixed ? (long long)slab * N * DK : tok_offset(p.lin, slab, p.heads, 0));
+    const size_t sq = SH::kFixed ? (size_t)DK : (size_t)p.lin.st;     // token stride of Q, K and V
     const T* gB = has_bias ? static_cast<const T*>(p.b1) + (size_t)head * n * N : nullptr;
     T* gA = static_cast<T*>(p.a_ws) + (size_t)slab * n * DK;
     const uint32_t tile_tx = 2 * kTileBytes + (bias_tma ? kTileBytes : 0);
@@ -188,8 +198,8 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
         if (tid == 0) {
             const uint32_t bar = bar_full(st, s), dst = ring_u32 + s * kStageBytes;
             mbar_arrive_expect_tx(bar, tile_tx);
-            tma_load_2d(dst, &p.tm_k, 0, slab * N + c0, bar);
-            tma_load_2d(dst + kTileBytes, &p.tm_v, 0, slab * N + c0, bar);
+            load_tokens(dst, &p.tm_k, SH::kFixed ? 1 : p.dense_in, p.hf_k, c0, head, slab / p.heads, slab * N, bar);
+            load_tokens(dst + kTileBytes, &p.tm_v, SH::kFixed ? 1 : p.dense_in, p.hf_v, c0, head, slab / p.heads, slab * N, bar);
             if (bias_tma) tma_load_2d(dst + 2 * kTileBytes, &p.tm_b1, c0, head * n, bar);
         }
         if (has_bias && !bias_tma) {       // B1 rows not 16-byte aligned: plain loads into the same layout
@@ -227,7 +237,7 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
                     const int ay = ar0 + wi / P, ax = wi % P;
                     const int wy = tsub / win_w, wx = tsub - wy * win_w;
                     const size_t tok = (size_t)(ay * win_h + wy) * W + (ax * win_w + wx);
-                    raw[u] = __ldg(reinterpret_cast<const uint4*>(gQ + tok * DK) + cg);
+                    raw[u] = __ldg(reinterpret_cast<const uint4*>(gQ + tok * sq) + cg);
                 }
             }
 #pragma unroll
@@ -263,7 +273,7 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
                     if (i < cnt) {
                         const int wy = i / win_w, wx = i - wy * win_w;
                         const size_t tok = (size_t)(y0 + wy) * W + (x0 + wx);
-                        raw[u] = __ldg(reinterpret_cast<const uint4*>(gQ + tok * DK) + cg);
+                        raw[u] = __ldg(reinterpret_cast<const uint4*>(gQ + tok * sq) + cg);
                     }
                 }
 #pragma unroll
@@ -527,8 +537,6 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
     T* sH = reinterpret_cast<T*>(smem + OFF_HALO);                   // [(rows+2)][W+2][DK]
     T* sB2 = reinterpret_cast<T*>(smem + OFF_B2);                    // [TQ][n] flat
 
-    const T* gQ = static_cast<const T*>(p.q) + ((size_t)slab * N + q0) * DK;
-    const T* gV = static_cast<const T*>(p.v) + (size_t)slab * N * DK;
     const unsigned* va_flag = p.counters + 2 * p.slabs + slab;
 
     TRACE(slot, 0);
@@ -552,12 +560,19 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
         const uint32_t bar = bar_bin(st);
         mbar_arrive_expect_tx(bar, bin_bytes);
         // Q tile: 128 rows from the tile's first token (rows past the tile feed rows that are never stored)
-        tma_load_2d(smem_u32(smem + OFF_PATCH), &p.tm_q, 0, slab * N + q0, bar);
+        load_tokens(smem_u32(smem + OFF_PATCH), &p.tm_q, SH::kFixed ? 1 : p.dense_in, p.hf_q, q0, head, slab / p.heads, slab * N, bar);
         if (has_dwc) {
             for (int hr = 0; hr < rows + 2; ++hr) {
                 const int y = y0 - 1 + hr;
                 if (y >= 0 && y < H)
-                    bulk_load_1d(smem_u32(sH + ((size_t)hr * HP + 1) * DK), gV + (size_t)y * W * DK, W * DK * 2, bar);
+                    if (SH::kFixed)              // dense: one copy of W * 128 contiguous bytes
+                        bulk_load_1d(smem_u32(sH + ((size_t)hr * HP + 1) * DK),
+                                     static_cast<const T*>(p.v) + ((size_t)slab * N + (size_t)y * W) * DK, W * DK * 2, bar);
+                    else if (p.v_rows_contiguous)
+                        bulk_load_1d(smem_u32(sH + ((size_t)hr * HP + 1) * DK),
+                                     static_cast<const T*>(p.v) + tok_offset(p.lin, slab, p.heads, (long long)y * W), W * DK * 2, bar);
+                    else
+                        tma_load_tok(smem_u32(sH + ((size_t)hr * HP + 1) * DK), &p.tm_vrow, p.hf_vrow, y * W, head, slab / p.heads, bar);
             }
         }
         if (b2_bulk) bulk_load_1d(smem_u32(sB2), b2src, b2bytes, bar);
@@ -713,14 +728,15 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
         if (nseg < 1) nseg = 1;
         if (nseg > W) nseg = W;
         const int seg_len = (W + nseg - 1) / nseg;
-        T* gO = static_cast<T*>(p.out) + ((size_t)slab * N + q0) * DK;
+        T* gO = static_cast<T*>(p.out) + (SH::kFixed ? ((long long)slab * N + q0) * DK : tok_offset(p.lout, slab, p.heads, q0));
+        const size_t so = SH::kFixed ? (size_t)DK : (size_t)p.lout.st;    // token stride of out
         for (int item = tid; item < npairs * nseg; item += NT) {
             const int pair = item % npairs, seg = item / npairs;
             const int r = pair / NCQ, cq = pair - r * NCQ;
             const int x0 = seg * seg_len, x1 = min(W, x0 + seg_len);
             if (x0 >= x1) continue;
             const float* pp = sPatchAll + (r * W) * PO + cq * 4;
-            T* op = gO + (size_t)(r * W) * DK + cq * 4;
+            T* op = gO + (size_t)(r * W) * so + cq * 4;
             if (has_dwc) {
                 float2 w[9][2];                 // taps x two channel pairs
 #pragma unroll
@@ -752,7 +768,7 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
                     uint2 outw;
                     outw.x = pack2<T>(o0.x, o0.y);
                     outw.y = pack2<T>(o1.x, o1.y);
-                    *reinterpret_cast<uint2*>(op + x * DK) = outw;
+                    *reinterpret_cast<uint2*>(op + x * so) = outw;
                 };
                 load_col(x0, ca);          // grid column x0 - 1
                 load_col(x0 + 1, cb);      // grid column x0
@@ -768,7 +784,7 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
                     uint2 outw;
                     outw.x = pack2<T>(a4.x, a4.y);
                     outw.y = pack2<T>(a4.z, a4.w);
-                    *reinterpret_cast<uint2*>(op + x * DK) = outw;
+                    *reinterpret_cast<uint2*>(op + x * so) = outw;
                 }
             }
         }

@@ -112,9 +112,22 @@ FusedPlan plan_fused(int dtype, int slabs, int H, int W, int d, int n_agents, in
 // Fills the tensor maps of `a` from its pointers and shape; false if one cannot be encoded.
 bool fused_make_maps(FusedArgs* a) {
     const uint64_t N = (uint64_t)a->H * a->W, S = a->slabs;
-    if (!make_map_2d_u16(&a->tm_k, a->k, S * N, DK, KT, DK)) return false;
-    if (!make_map_2d_u16(&a->tm_v, a->v, S * N, DK, KT, DK)) return false;
-    if (!make_map_2d_u16(&a->tm_q, a->q, S * N, DK, QT, DK)) return false;
+    const int batch = a->slabs / a->heads;
+    const TokLayout dl = dense_layout(a->heads, (long long)N, DK);
+    a->dense_in = (a->lin.sb == dl.sb && a->lin.sh == dl.sh && a->lin.st == dl.st) ? 1 : 0;
+    if (a->dense_in) {
+        if (!make_map_2d_u16(&a->tm_k, a->k, S * N, DK, KT, DK)) return false;
+        if (!make_map_2d_u16(&a->tm_v, a->v, S * N, DK, KT, DK)) return false;
+        if (!make_map_2d_u16(&a->tm_q, a->q, S * N, DK, QT, DK)) return false;
+    } else {
+        if (!make_map_tok_u16(&a->tm_k, &a->hf_k, a->k, a->lin, batch, a->heads, (long long)N, DK, KT, true)) return false;
+        if (!make_map_tok_u16(&a->tm_v, &a->hf_v, a->v, a->lin, batch, a->heads, (long long)N, DK, KT, true)) return false;
+        if (!make_map_tok_u16(&a->tm_q, &a->hf_q, a->q, a->lin, batch, a->heads, (long long)N, DK, QT, true)) return false;
+    }
+    a->v_rows_contiguous = (a->lin.st == DK) ? 1 : 0;
+    if (a->dwc_w && !a->v_rows_contiguous &&
+        !make_map_tok_u16(&a->tm_vrow, &a->hf_vrow, a->v, a->lin, batch, a->heads, (long long)N, DK, (uint32_t)a->W, false))
+        return false;
     if (!make_map_2d_u16(&a->tm_a, a->a_ws, S * a->n, DK, RP, DK)) return false;
     if (!make_map_2d_u16(&a->tm_va, a->va_ws, S * a->n, DK, RP, DK)) return false;
     a->b1_tma = 0;
@@ -125,7 +138,10 @@ bool fused_make_maps(FusedArgs* a) {
 
 cudaError_t launch_fused(int dtype, const FusedArgs& a, cudaStream_t st) {
     // the shape-specialised kernels assume both biases and the depthwise filter are present
-    const bool full = a.b1 && a.b2 && a.dwc_w;
+    // ... and dense layouts
+    const TokLayout dl = dense_layout(a.heads, (long long)a.H * a.W, DK);
+    const bool dense = a.dense_in && a.lout.sb == dl.sb && a.lout.sh == dl.sh && a.lout.st == dl.st;
+    const bool full = a.b1 && a.b2 && a.dwc_w && dense;
     if (full && a.plan.spec == 1) return launch_fused_s56(dtype, a, st);
     if (full && a.plan.spec == 2) return launch_fused_s14(dtype, a, st);
     return fused_launch_dt<ShapeAny>(dtype, a, st);

@@ -127,11 +127,15 @@ struct FusedArgs {
     float scale1, scale2;
     TokLayout lin, lout;  // strides of Q, K, V and of out
     FusedPlan plan;
-    // TMA descriptors (128-byte swizzle, 64-column boxes): K and V as [slabs*N][d] with 64-row boxes,
+    // TMA descriptors (128-byte swizzle, 64-column boxes): K and V with 64-token boxes (any batch / head / token strides),
     // B1 as [heads*n][N] with 64x64 boxes, A and V_A workspaces as [slabs*n][d] with 64-row boxes
     int b1_tma;           // B1 tiles come through TMA (needs N % 8 == 0 and 8-aligned task ranges)
     alignas(64) CUtensorMap tm_k, tm_v, tm_b1, tm_a, tm_va;
-    alignas(64) CUtensorMap tm_q;     // Q as [slabs*N][d] with 128-row boxes (A operand of the broadcast MMA)
+    alignas(64) CUtensorMap tm_q;     // Q with 128-token boxes (A operand of the broadcast MMA)
+    alignas(64) CUtensorMap tm_vrow;  // V with boxes of one grid row (W tokens), no swizzle: rows of the depthwise window
+    int hf_k, hf_v, hf_q, hf_vrow;    // dimension order of the token-major maps (tma_load_tok)
+    int v_rows_contiguous;            // token stride of V == d: a grid row of V is one contiguous run
+    int dense_in;                     // Q, K, V are dense [B][heads][N][d]: their maps are 2-D over [slabs * N][d]
 };
 FusedPlan plan_fused(int dtype, int slabs, int H, int W, int d, int n_agents, int sm_count);
 bool fused_make_maps(FusedArgs* a);     // encode the tensor maps from a's pointers and shape

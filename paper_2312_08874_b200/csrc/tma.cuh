@@ -123,7 +123,9 @@ inline bool make_map_tok_u16(CUtensorMap* out, int* head_first, const void* base
     const int hf = (heads > 1 && l.sh < l.st) ? 1 : 0;
     *head_first = hf;
     const cuuint64_t n1 = hf ? (cuuint64_t)heads : (cuuint64_t)n_tokens, n2 = hf ? (cuuint64_t)n_tokens : (cuuint64_t)heads;
-    const cuuint64_t s1 = (cuuint64_t)(hf ? l.sh : l.st) * 2, s2 = (cuuint64_t)(hf ? l.st : l.sh) * 2;
+    const cuuint64_t s1 = (cuuint64_t)(hf ? l.sh : l.st) * 2;
+    cuuint64_t s2 = (cuuint64_t)(hf ? l.st : l.sh) * 2;
+    if (heads == 1 && s2 < s1 * n1) s2 = s1 * n1;          // a single head: its stride is never used
     cuuint64_t s3 = (cuuint64_t)l.sb * 2;
     if (batch == 1 && s3 < s2 * n2) s3 = s2 * n2;          // a single batch item: its stride is never used
     const cuuint64_t dims[4] = {(cuuint64_t)d, n1, n2, (cuuint64_t)batch};

@@ -246,3 +246,58 @@ def test_invalid_arguments_are_rejected_without_launching():
     with pytest.raises(AgentAttnError):
         AgentAttention(1, 1, 64, 64, 257, torch.bfloat16)
     torch.cuda.synchronize()
+
+
+# ------------------------------------------------------------- token-major layouts with strides
+STRIDED = [
+    # batch heads H  W   d   pool dtype   bias  dwc     kernel that takes it
+    (2, 3, 28, 28, 64, 7, "bf16", True, True),       # fused persistent kernel
+    (3, 2, 14, 14, 64, 7, "f16", True, True),        # fused, one G task per slab, unaligned bias rows
+    (2, 2, 32, 32, 64, 16, "bf16", True, True),      # tensor-memory kernels, n = 256
+    (1, 4, 36, 36, 40, 12, "f16", True, True),       # tensor-memory kernels, n = 144, d = 40
+    (2, 1, 24, 24, 64, 12, "bf16", False, False),    # one head, no bias, no DWC
+]
+
+
+@pytest.mark.parametrize("packed", [False, True], ids=["bnhd", "qkv_interleaved"])
+@pytest.mark.parametrize("case", STRIDED, ids=[f"B{c[0]}h{c[1]}_{c[2]}x{c[3]}_d{c[4]}_p{c[5]}_{c[6]}" for c in STRIDED])
+def test_strided_token_major_layouts(case, packed):
+    """Q, K, V read in place from [B, N, heads, d] (or interleaved [B, N, 3, heads, d]) and O written as
+    [B, N, heads, d]: same result as the dense call on transposed copies, and within tolerance of the oracle."""
+    B, heads, H, W, d, pool, dtype, bias, dwc = case
+    w = Workload("strided", B, heads, H, W, d, pool, dtype, bias, dwc, 1.0, seed=300 + H * W + d)
+    inp = make_inputs(w, bias_std=0.5, dwc_std=0.2)
+    mod = make_module(w)
+    dense = gpu_forward(mod, w, inp)
+    q, k, v = (to_dev(inp[x]) for x in ("q", "k", "v"))                 # [B, heads, N, d]
+    if packed:
+        qkv = torch.stack([t.permute(0, 2, 1, 3) for t in (q, k, v)], dim=2).contiguous()    # [B, N, 3, heads, d]
+        views = [qkv[:, :, i].permute(0, 2, 1, 3) for i in range(3)]
+    else:
+        views = [t.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3) for t in (q, k, v)]  # [B, N, heads, d] storage
+    assert not views[0].is_contiguous() or heads == 1
+    out = mod.forward_strided(views[0], views[1], views[2], H, W, w.agents, b1=to_dev(inp["b1"]), b2=to_dev(inp["b2"]),
+                              dwc_weight=to_dev(inp["dwc"]))
+    torch.cuda.synchronize()
+    assert mod.query_status() == 0
+    assert out.permute(0, 2, 1, 3).is_contiguous()                       # stored as [B, N, heads, d]
+    assert torch.equal(out, dense), "the strided call must match the dense call bit for bit"
+    assert_close(out.contiguous(), oracle_forward(w, inp), dtype, f"strided {case}")
+
+
+def test_strided_call_with_dense_strides_is_the_dense_call_and_fp32_is_refused():
+    w = WORKLOADS["cfg3_pvt_bf16"].scaled(batch=2)
+    inp = make_inputs(w)
+    mod = make_module(w)
+    dense = gpu_forward(mod, w, inp)
+    out = torch.empty_like(dense)
+    mod.forward_strided(to_dev(inp["q"]), to_dev(inp["k"]), to_dev(inp["v"]), w.grid_h, w.grid_w, w.agents,
+                        b1=to_dev(inp["b1"]), b2=to_dev(inp["b2"]), dwc_weight=to_dev(inp["dwc"]), out=out)
+    torch.cuda.synchronize()
+    assert torch.equal(out, dense)
+    w32 = Workload("strided32", 1, 2, 8, 8, 32, 2, "f32", False, False, 1.0, seed=9)
+    i32 = make_inputs(w32)
+    m32 = make_module(w32)
+    qv = to_dev(i32["q"]).permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    with pytest.raises(RuntimeError, match="AA_ERR_UNSUPPORTED"):
+        m32.forward_strided(qv, qv, qv, 8, 8, 4)
