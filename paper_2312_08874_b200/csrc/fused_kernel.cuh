@@ -158,11 +158,12 @@ __device__ __forceinline__ void sync_rows() { asm volatile("bar.sync 1, 128;\n" 
 // Compile-time shape: a kernel instantiated for one token grid and agent grid (with biases and the
 // depthwise term present) folds its index arithmetic and loop bounds; 0 means "read it from the
 // arguments".  The generic kernel uses ShapeAny.
-template <int H_, int W_, int P_> struct FusedShape {
+template <int H_, int W_, int P_, bool DENSE_ = true> struct FusedShape {
     static constexpr int kH = H_, kW = W_, kP = P_;
     static constexpr bool kFixed = (H_ > 0);
+    static constexpr bool kDense = kFixed && DENSE_;     // dense [B][heads][N][d] tensors: constant strides, 2-D maps
 };
-using ShapeAny = FusedShape<0, 0, 0>;
+using ShapeAny = FusedShape<0, 0, 0, false>;
 
 // ---------------------------------------------------------------------------------- G task
 template <typename T, typename SH>
@@ -186,8 +187,8 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
     unsigned char* ring = smem + OFF_UNION;
     const uint32_t ring_u32 = smem_u32(ring);
     // the shape-specialised kernels serve dense tensors only: their strides are compile-time constants
-    const T* gQ = static_cast<const T*>(p.q) + (SH::kFixed ? (long long)slab * N * DK : tok_offset(p.lin, slab, p.heads, 0));
-    const size_t sq = SH::kFixed ? (size_t)DK : (size_t)p.lin.st;     // token stride of Q, K and V
+    const T* gQ = static_cast<const T*>(p.q) + (SH::kDense ? (long long)slab * N * DK : tok_offset(p.lin, slab, p.heads, 0));
+    const size_t sq = SH::kDense ? (size_t)DK : (size_t)p.lin.st;     // token stride of Q, K and V
     const T* gB = has_bias ? static_cast<const T*>(p.b1) + (size_t)head * n * N : nullptr;
     T* gA = static_cast<T*>(p.a_ws) + (size_t)slab * n * DK;
     const uint32_t tile_tx = 2 * kTileBytes + (bias_tma ? kTileBytes : 0);
@@ -198,8 +199,8 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
         if (tid == 0) {
             const uint32_t bar = bar_full(st, s), dst = ring_u32 + s * kStageBytes;
             mbar_arrive_expect_tx(bar, tile_tx);
-            load_tokens(dst, &p.tm_k, SH::kFixed ? 1 : p.dense_in, p.hf_k, c0, head, slab / p.heads, slab * N, bar);
-            load_tokens(dst + kTileBytes, &p.tm_v, SH::kFixed ? 1 : p.dense_in, p.hf_v, c0, head, slab / p.heads, slab * N, bar);
+            load_tokens(dst, &p.tm_k, SH::kDense ? 1 : p.dense_in, p.hf_k, c0, head, slab / p.heads, slab * N, bar);
+            load_tokens(dst + kTileBytes, &p.tm_v, SH::kDense ? 1 : p.dense_in, p.hf_v, c0, head, slab / p.heads, slab * N, bar);
             if (bias_tma) tma_load_2d(dst + 2 * kTileBytes, &p.tm_b1, c0, head * n, bar);
         }
         if (has_bias && !bias_tma) {       // B1 rows not 16-byte aligned: plain loads into the same layout
@@ -560,12 +561,12 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
         const uint32_t bar = bar_bin(st);
         mbar_arrive_expect_tx(bar, bin_bytes);
         // Q tile: 128 rows from the tile's first token (rows past the tile feed rows that are never stored)
-        load_tokens(smem_u32(smem + OFF_PATCH), &p.tm_q, SH::kFixed ? 1 : p.dense_in, p.hf_q, q0, head, slab / p.heads, slab * N, bar);
+        load_tokens(smem_u32(smem + OFF_PATCH), &p.tm_q, SH::kDense ? 1 : p.dense_in, p.hf_q, q0, head, slab / p.heads, slab * N, bar);
         if (has_dwc) {
             for (int hr = 0; hr < rows + 2; ++hr) {
                 const int y = y0 - 1 + hr;
                 if (y >= 0 && y < H)
-                    if (SH::kFixed)              // dense: one copy of W * 128 contiguous bytes
+                    if (SH::kDense)              // dense: one copy of W * 128 contiguous bytes
                         bulk_load_1d(smem_u32(sH + ((size_t)hr * HP + 1) * DK),
                                      static_cast<const T*>(p.v) + ((size_t)slab * N + (size_t)y * W) * DK, W * DK * 2, bar);
                     else if (p.v_rows_contiguous)
@@ -728,8 +729,8 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
         if (nseg < 1) nseg = 1;
         if (nseg > W) nseg = W;
         const int seg_len = (W + nseg - 1) / nseg;
-        T* gO = static_cast<T*>(p.out) + (SH::kFixed ? ((long long)slab * N + q0) * DK : tok_offset(p.lout, slab, p.heads, q0));
-        const size_t so = SH::kFixed ? (size_t)DK : (size_t)p.lout.st;    // token stride of out
+        T* gO = static_cast<T*>(p.out) + (SH::kDense ? ((long long)slab * N + q0) * DK : tok_offset(p.lout, slab, p.heads, q0));
+        const size_t so = SH::kDense ? (size_t)DK : (size_t)p.lout.st;    // token stride of out
         for (int item = tid; item < npairs * nseg; item += NT) {
             const int pair = item % npairs, seg = item / npairs;
             const int r = pair / NCQ, cq = pair - r * NCQ;

@@ -15,6 +15,10 @@ int fused_occupancy_s56(int dtype);
 int fused_occupancy_s14(int dtype);
 cudaError_t launch_fused_s56(int dtype, const FusedArgs& a, cudaStream_t st);
 cudaError_t launch_fused_s14(int dtype, const FusedArgs& a, cudaStream_t st);
+int fused_occupancy_s56s(int dtype);
+int fused_occupancy_s14s(int dtype);
+cudaError_t launch_fused_s56s(int dtype, const FusedArgs& a, cudaStream_t st);
+cudaError_t launch_fused_s14s(int dtype, const FusedArgs& a, cudaStream_t st);
 
 static int fused_spec_of(int H, int W, int n_agents) {
 #ifdef AA_FUSED_TRACE
@@ -65,8 +69,8 @@ FusedPlan plan_fused(int dtype, int slabs, int H, int W, int d, int n_agents, in
     // (each query also raises that kernel's dynamic shared-memory limit; the generic kernel serves a
     // specialised shape whenever a bias or the depthwise filter is absent)
     int occ = fused_occupancy_dt<ShapeAny>(dtype);
-    if (pl.spec == 1) occ = std::min(occ, fused_occupancy_s56(dtype));
-    if (pl.spec == 2) occ = std::min(occ, fused_occupancy_s14(dtype));
+    if (pl.spec == 1) occ = std::min(occ, std::min(fused_occupancy_s56(dtype), fused_occupancy_s56s(dtype)));
+    if (pl.spec == 2) occ = std::min(occ, std::min(fused_occupancy_s14(dtype), fused_occupancy_s14s(dtype)));
     if (occ < 1) return pl;
     // The occupancy query counts a block that allocates tensor memory as taking all of it.  Two blocks
     // of 128 columns each fit the 512 columns of an SM, so where registers and shared memory allow a
@@ -137,13 +141,13 @@ bool fused_make_maps(FusedArgs* a) {
 }
 
 cudaError_t launch_fused(int dtype, const FusedArgs& a, cudaStream_t st) {
-    // the shape-specialised kernels assume both biases and the depthwise filter are present
-    // ... and dense layouts
+    // the shape-specialised kernels assume both biases and the depthwise filter are present; each shape has
+    // an instantiation for dense tensors and one for tensors with strides
     const TokLayout dl = dense_layout(a.heads, (long long)a.H * a.W, DK);
     const bool dense = a.dense_in && a.lout.sb == dl.sb && a.lout.sh == dl.sh && a.lout.st == dl.st;
-    const bool full = a.b1 && a.b2 && a.dwc_w && dense;
-    if (full && a.plan.spec == 1) return launch_fused_s56(dtype, a, st);
-    if (full && a.plan.spec == 2) return launch_fused_s14(dtype, a, st);
+    const bool full = a.b1 && a.b2 && a.dwc_w;
+    if (full && a.plan.spec == 1) return dense ? launch_fused_s56(dtype, a, st) : launch_fused_s56s(dtype, a, st);
+    if (full && a.plan.spec == 2) return dense ? launch_fused_s14(dtype, a, st) : launch_fused_s14s(dtype, a, st);
     return fused_launch_dt<ShapeAny>(dtype, a, st);
 }
 

@@ -7,4 +7,9 @@ int fused_occupancy_s14(int dtype) { return fused_occupancy_dt<FusedShape<14, 14
 cudaError_t launch_fused_s14(int dtype, const FusedArgs& a, cudaStream_t st) {
     return fused_launch_dt<FusedShape<14, 14, 7>>(dtype, a, st);
 }
+// the same shape on tensors with strides (token-major or interleaved storage)
+int fused_occupancy_s14s(int dtype) { return fused_occupancy_dt<FusedShape<14, 14, 7, false>>(dtype); }
+cudaError_t launch_fused_s14s(int dtype, const FusedArgs& a, cudaStream_t st) {
+    return fused_launch_dt<FusedShape<14, 14, 7, false>>(dtype, a, st);
+}
 }  // namespace aa

@@ -256,6 +256,7 @@ STRIDED = [
     (2, 2, 32, 32, 64, 16, "bf16", True, True),      # tensor-memory kernels, n = 256
     (1, 4, 36, 36, 40, 12, "f16", True, True),       # tensor-memory kernels, n = 144, d = 40
     (2, 1, 24, 24, 64, 12, "bf16", False, False),    # one head, no bias, no DWC
+    (1, 2, 56, 56, 64, 7, "bf16", True, True),       # fused, the 56x56 shape-specialised instantiation for strides
 ]
 
 
