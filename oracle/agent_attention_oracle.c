@@ -246,6 +246,145 @@ void aa_oracle_compose_bias(const double* col, const double* row, const double* 
 }
 
 /* ---------------------------------------------------------------------------------
+ * Gradients of Eq. 6 (pooled agents).  The paper prints no backward formulas; these are the
+ * chain rule applied to the steps of aa_oracle_forward, written out densely per slab:
+ *   with P2 = s(scale2 Q A^T + B2), P1 = s(scale1 A K^T + B1), V_A = P1 V, O = P2 V_A + DWC(V)
+ *   dV_A = P2^T dO            dP2 = dO V_A^T      dS2 = P2 o (dP2 - rowsum(P2 o dP2))
+ *   dQ  = scale2 dS2 A        dA  = scale2 dS2^T Q + scale1 dS1 K
+ *   dP1 = dV_A V^T            dS1 = P1 o (dP1 - rowsum(P1 o dP1))
+ *   dK  = scale1 dS1^T A      dV  = P1^T dV_A + DWC^T(dO)
+ *   dB1 = sum over batch dS1  dB2 = sum over batch dS2   dWd[c][u][v] = sum dO[y,x,c] V[y+u-1,x+v-1,c]
+ *   dQ += Pooling^T(dA): every token of agent a's window receives dA[a] / (window size).
+ * dO, dQ, dK, dV [B][heads][N][d]; dB1 [heads][n][N], dB2 [heads][N][n], dWd [heads][d][3][3]
+ * (each may be NULL when the forward had no such input; they are overwritten, not accumulated into).
+ * Serial over slabs (the bias and filter gradients sum over the batch).  Returns 0, or -1 on bad arguments.
+ * ------------------------------------------------------------------------------- */
+int aa_oracle_backward(const double* Q, const double* K, const double* V, const double* dO,
+                       int B, int heads, int H, int W, int d, int n, int ph, int pw,
+                       const double* b1, const double* b2, const double* wd,
+                       double scale1, double scale2,
+                       double* dQ, double* dK, double* dV, double* dB1, double* dB2, double* dWd)
+{
+    if (!Q || !K || !V || !dO || !dQ || !dK || !dV || B <= 0 || heads <= 0 || H <= 0 || W <= 0 || d <= 0)
+        return -1;
+    if (ph <= 0 || pw <= 0 || ph * pw != n || ph > H || pw > W) return -1;
+    const int N = H * W;
+    const size_t nN = (size_t)n * N, nd = (size_t)n * d, Nd = (size_t)N * d;
+    if (dB1) memset(dB1, 0, sizeof(double) * heads * nN);
+    if (dB2) memset(dB2, 0, sizeof(double) * heads * nN);
+    if (dWd) memset(dWd, 0, sizeof(double) * (size_t)heads * d * 9);
+    double* a = (double*)malloc(sizeof(double) * nd);
+    double* va = (double*)malloc(sizeof(double) * nd);
+    double* dva = (double*)malloc(sizeof(double) * nd);
+    double* da = (double*)malloc(sizeof(double) * nd);
+    double* p1 = (double*)malloc(sizeof(double) * nN);      /* [n][N] */
+    double* p2 = (double*)malloc(sizeof(double) * nN);      /* [N][n] */
+    double* ds = (double*)malloc(sizeof(double) * nN);
+    double* oat = (double*)malloc(sizeof(double) * Nd);
+    for (int s = 0; s < B * heads; ++s) {
+        const int head = s % heads;
+        const double *q = Q + s * Nd, *k = K + s * Nd, *v = V + s * Nd, *go = dO + s * Nd;
+        double *gq = dQ + s * Nd, *gk = dK + s * Nd, *gv = dV + s * Nd;
+        aa_oracle_pool(q, H, W, d, ph, pw, a);
+        aa_oracle_softmax_attention(a, k, v, b1 ? b1 + head * nN : NULL, n, N, d, d, scale1, va, p1);
+        aa_oracle_softmax_attention(q, a, va, b2 ? b2 + head * nN : NULL, N, n, d, d, scale2, oat, p2);
+        /* broadcast stage */
+        for (int r = 0; r < n; ++r)
+            for (int c = 0; c < d; ++c) {
+                double acc = 0.0;
+                for (int i = 0; i < N; ++i) acc += p2[(size_t)i * n + r] * go[(size_t)i * d + c];
+                dva[(size_t)r * d + c] = acc;
+            }
+        for (int i = 0; i < N; ++i) {
+            double dot = 0.0;
+            for (int r = 0; r < n; ++r) {
+                double dp = 0.0;
+                for (int c = 0; c < d; ++c) dp += go[(size_t)i * d + c] * va[(size_t)r * d + c];
+                ds[(size_t)i * n + r] = dp;
+                dot += p2[(size_t)i * n + r] * dp;
+            }
+            for (int r = 0; r < n; ++r) {
+                const double g = p2[(size_t)i * n + r] * (ds[(size_t)i * n + r] - dot);
+                ds[(size_t)i * n + r] = g;
+                if (dB2) dB2[head * nN + (size_t)i * n + r] += g;
+            }
+        }
+        for (int i = 0; i < N; ++i)
+            for (int c = 0; c < d; ++c) {
+                double acc = 0.0;
+                for (int r = 0; r < n; ++r) acc += ds[(size_t)i * n + r] * a[(size_t)r * d + c];
+                gq[(size_t)i * d + c] = scale2 * acc;
+            }
+        for (int r = 0; r < n; ++r)
+            for (int c = 0; c < d; ++c) {
+                double acc = 0.0;
+                for (int i = 0; i < N; ++i) acc += ds[(size_t)i * n + r] * q[(size_t)i * d + c];
+                da[(size_t)r * d + c] = scale2 * acc;
+            }
+        /* aggregation stage */
+        for (int r = 0; r < n; ++r) {
+            double dot = 0.0;
+            for (int j = 0; j < N; ++j) {
+                double dp = 0.0;
+                for (int c = 0; c < d; ++c) dp += dva[(size_t)r * d + c] * v[(size_t)j * d + c];
+                ds[(size_t)r * N + j] = dp;
+                dot += p1[(size_t)r * N + j] * dp;
+            }
+            for (int j = 0; j < N; ++j) {
+                const double g = p1[(size_t)r * N + j] * (ds[(size_t)r * N + j] - dot);
+                ds[(size_t)r * N + j] = g;
+                if (dB1) dB1[head * nN + (size_t)r * N + j] += g;
+            }
+        }
+        for (int j = 0; j < N; ++j)
+            for (int c = 0; c < d; ++c) {
+                double gk_acc = 0.0, gv_acc = 0.0;
+                for (int r = 0; r < n; ++r) {
+                    gk_acc += ds[(size_t)r * N + j] * a[(size_t)r * d + c];
+                    gv_acc += p1[(size_t)r * N + j] * dva[(size_t)r * d + c];
+                }
+                gk[(size_t)j * d + c] = scale1 * gk_acc;
+                gv[(size_t)j * d + c] = gv_acc;
+            }
+        for (int r = 0; r < n; ++r)
+            for (int c = 0; c < d; ++c) {
+                double acc = 0.0;
+                for (int j = 0; j < N; ++j) acc += ds[(size_t)r * N + j] * k[(size_t)j * d + c];
+                da[(size_t)r * d + c] += scale1 * acc;
+            }
+        /* depthwise term */
+        if (wd) {
+            const double* w = wd + (size_t)head * d * 9;
+            for (int y = 0; y < H; ++y)
+                for (int x = 0; x < W; ++x)
+                    for (int u = 0; u < 3; ++u)
+                        for (int t = 0; t < 3; ++t) {
+                            const int yy = y + u - 1, xx = x + t - 1;
+                            if (yy < 0 || yy >= H || xx < 0 || xx >= W) continue;
+                            for (int c = 0; c < d; ++c) {
+                                const double g = go[((size_t)y * W + x) * d + c];
+                                gv[((size_t)yy * W + xx) * d + c] += w[(size_t)c * 9 + u * 3 + t] * g;
+                                if (dWd) dWd[((size_t)head * d + c) * 9 + u * 3 + t] += g * v[((size_t)yy * W + xx) * d + c];
+                            }
+                        }
+        }
+        /* pooling: the window of agent (ay, ax) as in aa_oracle_pool */
+        for (int ay = 0; ay < ph; ++ay)
+            for (int ax = 0; ax < pw; ++ax) {
+                const int y0 = (ay * H) / ph, y1 = ((ay + 1) * H + ph - 1) / ph;
+                const int x0 = (ax * W) / pw, x1 = ((ax + 1) * W + pw - 1) / pw;
+                const double inv = 1.0 / (double)((y1 - y0) * (x1 - x0));
+                for (int y = y0; y < y1; ++y)
+                    for (int x = x0; x < x1; ++x)
+                        for (int c = 0; c < d; ++c)
+                            gq[((size_t)y * W + x) * d + c] += da[(size_t)(ay * pw + ax) * d + c] * inv;
+            }
+    }
+    free(a); free(va); free(dva); free(da); free(p1); free(p2); free(ds); free(oat);
+    return 0;
+}
+
+/* ---------------------------------------------------------------------------------
  * Module complexity, Eq. 7, in multiply-accumulates for N tokens, C channels (all heads),
  * n agents, DWC kernel size k:
  *   parts = { 4NC^2 (projections), NC (agents), 2nNC (aggregation: logits and weighted

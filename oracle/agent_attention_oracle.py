@@ -53,6 +53,8 @@ def _load() -> ctypes.CDLL:
         lib.aa_oracle_macs.restype = ctypes.c_longlong
         lib.aa_oracle_compose_bias.argtypes = [_DP] * 3 + [ctypes.c_int] * 6 + [_DP]
         lib.aa_oracle_compose_bias.restype = None
+        lib.aa_oracle_backward.argtypes = ([_DP] * 4 + [ctypes.c_int] * 8 + [_DP] * 3 + [ctypes.c_double] * 2 + [_DP] * 6)
+        lib.aa_oracle_backward.restype = ctypes.c_int
         lib.aa_oracle_max_threads.argtypes = []
         lib.aa_oracle_max_threads.restype = ctypes.c_int
         _lib = lib
@@ -151,6 +153,38 @@ def forward(q, k, v, grid_h: int, grid_w: int, *, pool_hw: Optional[Tuple[int, i
 
 
 forward.last_threads = 1
+
+
+def backward(q, k, v, d_out, grid_h: int, grid_w: int, pool_hw: Tuple[int, int], b1=None, b2=None,
+             dwc_weight=None, scale1: Optional[float] = None, scale2: Optional[float] = None):
+    """Gradients of Eq. 6 with pooled agents for an upstream gradient d_out [B, heads, N, d].
+
+    Returns a dict with dq, dk, dv [B, heads, N, d] and, for the inputs that were given, db1 [heads, n, N],
+    db2 [heads, N, n], dwd [heads, d, 3, 3] (fp64).
+    """
+    q, k, v, g = _c(q), _c(k), _c(v), _c(d_out)
+    B, heads, N, d = q.shape
+    assert N == grid_h * grid_w and k.shape == q.shape and v.shape == q.shape and g.shape == q.shape
+    ph, pw = pool_hw
+    n = ph * pw
+    b1 = None if b1 is None else _c(b1)
+    b2 = None if b2 is None else _c(b2)
+    wd = None if dwc_weight is None else _c(dwc_weight)
+    assert b1 is None or b1.shape == (heads, n, N)
+    assert b2 is None or b2.shape == (heads, N, n)
+    assert wd is None or wd.shape == (heads, d, 3, 3)
+    s1 = d ** -0.5 if scale1 is None else float(scale1)
+    s2 = d ** -0.5 if scale2 is None else float(scale2)
+    out = {"dq": np.empty_like(q), "dk": np.empty_like(q), "dv": np.empty_like(q)}
+    if b1 is not None: out["db1"] = np.empty((heads, n, N), dtype=np.float64)
+    if b2 is not None: out["db2"] = np.empty((heads, N, n), dtype=np.float64)
+    if wd is not None: out["dwd"] = np.empty((heads, d, 3, 3), dtype=np.float64)
+    rc = _load().aa_oracle_backward(_p(q), _p(k), _p(v), _p(g), B, heads, grid_h, grid_w, d, n, ph, pw,
+                                    _p(b1), _p(b2), _p(wd), s1, s2, _p(out["dq"]), _p(out["dk"]), _p(out["dv"]),
+                                    _p(out.get("db1")), _p(out.get("db2")), _p(out.get("dwd")))
+    if rc != 0:
+        raise ValueError("aa_oracle_backward rejected its arguments")
+    return out
 
 
 def explicit(q, a, k, v, b1=None, b2=None, scale1: Optional[float] = None,
