@@ -274,7 +274,7 @@ int aa_oracle_backward(const double* Q, const double* K, const double* V, const 
     if (dB2) memset(dB2, 0, sizeof(double) * heads * nN);
     if (dWd) memset(dWd, 0, sizeof(double) * (size_t)heads * d * 9);
     double* a = (double*)malloc(sizeof(double) * nd);
-    double* va = (double*)malloc(sizeof(double) * nd);
+    double* v_a = (double*)malloc(sizeof(double) * nd);
     double* dva = (double*)malloc(sizeof(double) * nd);
     double* da = (double*)malloc(sizeof(double) * nd);
     double* p1 = (double*)malloc(sizeof(double) * nN);      /* [n][N] */
@@ -286,8 +286,8 @@ int aa_oracle_backward(const double* Q, const double* K, const double* V, const 
         const double *q = Q + s * Nd, *k = K + s * Nd, *v = V + s * Nd, *go = dO + s * Nd;
         double *gq = dQ + s * Nd, *gk = dK + s * Nd, *gv = dV + s * Nd;
         aa_oracle_pool(q, H, W, d, ph, pw, a);
-        aa_oracle_softmax_attention(a, k, v, b1 ? b1 + head * nN : NULL, n, N, d, d, scale1, va, p1);
-        aa_oracle_softmax_attention(q, a, va, b2 ? b2 + head * nN : NULL, N, n, d, d, scale2, oat, p2);
+        aa_oracle_softmax_attention(a, k, v, b1 ? b1 + head * nN : NULL, n, N, d, d, scale1, v_a, p1);
+        aa_oracle_softmax_attention(q, a, v_a, b2 ? b2 + head * nN : NULL, N, n, d, d, scale2, oat, p2);
         /* broadcast stage */
         for (int r = 0; r < n; ++r)
             for (int c = 0; c < d; ++c) {
@@ -299,7 +299,7 @@ int aa_oracle_backward(const double* Q, const double* K, const double* V, const 
             double dot = 0.0;
             for (int r = 0; r < n; ++r) {
                 double dp = 0.0;
-                for (int c = 0; c < d; ++c) dp += go[(size_t)i * d + c] * va[(size_t)r * d + c];
+                for (int c = 0; c < d; ++c) dp += go[(size_t)i * d + c] * v_a[(size_t)r * d + c];
                 ds[(size_t)i * n + r] = dp;
                 dot += p2[(size_t)i * n + r] * dp;
             }
@@ -354,7 +354,7 @@ int aa_oracle_backward(const double* Q, const double* K, const double* V, const 
             }
         /* depthwise term */
         if (wd) {
-            const double* w = wd + (size_t)head * d * 9;
+            const double* w = wd + (size_t)9 * d * head;          /* this head's [d][3][3] filter */
             for (int y = 0; y < H; ++y)
                 for (int x = 0; x < W; ++x)
                     for (int u = 0; u < 3; ++u)
@@ -380,7 +380,7 @@ int aa_oracle_backward(const double* Q, const double* K, const double* V, const 
                             gq[((size_t)y * W + x) * d + c] += da[(size_t)(ay * pw + ax) * d + c] * inv;
             }
     }
-    free(a); free(va); free(dva); free(da); free(p1); free(p2); free(ds); free(oat);
+    free(a); free(v_a); free(dva); free(da); free(p1); free(p2); free(ds); free(oat);
     return 0;
 }
 
