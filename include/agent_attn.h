@@ -137,6 +137,44 @@ int agent_attn_forward_strided(agent_attn_handle* h,
                                void* out, const long long out_strides[3],
                                void* workspace, size_t workspace_bytes, void* stream);
 
+/* Gradient buffers of agent_attn_backward, all fp32 device memory owned by the caller and overwritten
+ * by the call (no accumulation into their previous contents). */
+typedef struct {
+    void* dq;                 /* [B][heads][N][d], required                                  */
+    void* dk;                 /* [B][heads][N][d], required                                  */
+    void* dv;                 /* [B][heads][N][d], required                                  */
+    void* db1;                /* [heads][n][N], or NULL: gradient of bias b1, summed over B  */
+    void* db2;                /* [heads][N][n], or NULL: gradient of bias b2, summed over B  */
+    void* dwd;                /* [heads][d][3][3], or NULL: gradient of the depthwise filter */
+} agent_attn_grads;
+
+/* Bytes of device workspace agent_attn_backward needs (fp32 copies of A, V_A, dV_A, dA, the row
+ * statistics of the aggregation softmax and its per-block partial states).  0 on invalid arguments
+ * or an unsupported shape. */
+size_t agent_attn_backward_workspace_bytes(const agent_attn_handle* h, int grid_h, int grid_w, int n_agents);
+
+/* Gradients of Eq. 6 with pooled agents (A = Pooling(Q), so dQ includes the path through the agents):
+ * given d_out = dL/dO, writes dL/dQ, dL/dK, dL/dV and, where requested, dL/dB1, dL/dB2 (Eq. 5) and the
+ * gradient of the depthwise filter.  The forward quantities are recomputed from Q, K and V; nothing
+ * has to be saved by the forward call.
+ *   Q, K, V, d_out   device [B][heads][N][d] in the handle's element type
+ *   bias, dwc_weight as in agent_attn_forward (the same values the forward pass used)
+ *   grads            host struct of fp32 device buffers (see agent_attn_grads)
+ *   workspace        device, >= agent_attn_backward_workspace_bytes(...)
+ * n_agents must be a perfect square p*p with p <= min(grid_h, grid_w), and n_agents * head_dim <= 16384.
+ * All arithmetic is fp32 on CUDA cores for every element type and path setting.  Sums over tokens
+ * and over the batch are accumulated with floating-point atomics, so the low-order bits of the results
+ * may differ from run to run (the one exception to the reproducibility rule above).
+ * Errors: AA_ERR_INVALID_ARG (null, misaligned or aliasing buffers, n not a square, dwd without a
+ * filter), AA_ERR_UNSUPPORTED (shape limits), AA_ERR_WORKSPACE, AA_ERR_CUDA.  No host synchronisation,
+ * no allocation. */
+int agent_attn_backward(agent_attn_handle* h,
+                        const void* Q, const void* K, const void* V, const void* d_out,
+                        int grid_h, int grid_w, int n_agents,
+                        const agent_attn_bias* bias, const void* dwc_weight,
+                        const agent_attn_grads* grads,
+                        void* workspace, size_t workspace_bytes, void* stream);
+
 /* Step 1 alone: agent tokens by pooling (text under Eq. 6).  Q device [B][heads][N][d] ->
  * A_out device [B][heads][n][d], n = pool_h * pool_w, windows as described above. */
 int agent_attn_pool(agent_attn_handle* h, const void* Q, int grid_h, int grid_w,

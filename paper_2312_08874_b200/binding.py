@@ -26,6 +26,7 @@ EXPORTS = [
     "agent_attn_staging_bytes", "agent_attn_forward_host", "agent_attn_query_status",
     "agent_attn_last_launch_count", "agent_attn_aggregate_static", "agent_attn_static_scratch_bytes",
     "agent_attn_compose_bias", "agent_attn_forward_strided",
+    "agent_attn_backward_workspace_bytes", "agent_attn_backward",
 ]
 
 
@@ -38,6 +39,11 @@ class AgentAttnConfig(ctypes.Structure):
 
 class AgentAttnBias(ctypes.Structure):
     _fields_ = [("b1", ctypes.c_void_p), ("b2", ctypes.c_void_p)]
+
+
+class AgentAttnGrads(ctypes.Structure):
+    _fields_ = [("dq", ctypes.c_void_p), ("dk", ctypes.c_void_p), ("dv", ctypes.c_void_p),
+                ("db1", ctypes.c_void_p), ("db2", ctypes.c_void_p), ("dwd", ctypes.c_void_p)]
 
 
 class AgentAttnError(RuntimeError):
@@ -98,6 +104,11 @@ def load_library(build_if_missing: bool = True) -> ctypes.CDLL:
     lib.agent_attn_aggregate_static.restype = ci
     lib.agent_attn_compose_bias.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, vp, vp]
     lib.agent_attn_compose_bias.restype = ci
+    lib.agent_attn_backward_workspace_bytes.argtypes = [vp, ci, ci, ci]
+    lib.agent_attn_backward_workspace_bytes.restype = sz
+    lib.agent_attn_backward.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ctypes.POINTER(AgentAttnBias), vp,
+                                        ctypes.POINTER(AgentAttnGrads), vp, sz, vp]
+    lib.agent_attn_backward.restype = ci
     lib.agent_attn_static_scratch_bytes.argtypes = []
     lib.agent_attn_static_scratch_bytes.restype = sz
     _lib = lib
@@ -224,6 +235,47 @@ class AgentAttention:
             ctypes.byref(bias) if bias is not None else None, _ptr(dwc_weight), _ptr(out), sout, _ptr(ws),
             ws.numel(), _stream_ptr(stream)))
         return out
+
+    def backward_workspace(self, grid_h: int, grid_w: int, n_agents: int) -> torch.Tensor:
+        nbytes = self.lib.agent_attn_backward_workspace_bytes(self._h, grid_h, grid_w, n_agents)
+        if nbytes == 0:
+            raise AgentAttnError(2, f"backward does not support grid {grid_h}x{grid_w} with {n_agents} agents")
+        return torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+
+    def backward(self, q, k, v, d_out, grid_h: int, grid_w: int, n_agents: int, b1=None, b2=None,
+                 dwc_weight=None, need_bias_grads: bool = True, need_filter_grad: bool = True,
+                 workspace=None, stream=None) -> dict:
+        """`agent_attn_backward`: fp32 gradients of Eq. 6 (pooled agents) for the upstream gradient `d_out`.
+
+        Returns a dict with `dq`, `dk`, `dv` ([B, heads, N, d]) and, for the inputs that were given and asked
+        for, `db1` ([heads, n, N]), `db2` ([heads, N, n]) and `dwd` ([heads, d, 3, 3]).
+        """
+        B, h, d, N = self.batch, self.heads, self.head_dim, grid_h * grid_w
+        for t, nm in ((q, "q"), (k, "k"), (v, "v"), (d_out, "d_out")):
+            if t is None:
+                raise ValueError(f"{nm} is required")
+            self._chk_tensor(t, (B, h, N, d), nm)
+        self._chk_tensor(b1, (h, n_agents, N), "b1")
+        self._chk_tensor(b2, (h, N, n_agents), "b2")
+        self._chk_tensor(dwc_weight, (h, d, 3, 3), "dwc_weight")
+        f32 = dict(dtype=torch.float32, device=self.device)
+        g = {"dq": torch.empty((B, h, N, d), **f32), "dk": torch.empty((B, h, N, d), **f32),
+             "dv": torch.empty((B, h, N, d), **f32)}
+        if b1 is not None and need_bias_grads:
+            g["db1"] = torch.empty((h, n_agents, N), **f32)
+        if b2 is not None and need_bias_grads:
+            g["db2"] = torch.empty((h, N, n_agents), **f32)
+        if dwc_weight is not None and need_filter_grad:
+            g["dwd"] = torch.empty((h, d, 3, 3), **f32)
+        ws = self.backward_workspace(grid_h, grid_w, n_agents) if workspace is None else workspace
+        bias = AgentAttnBias(_ptr(b1), _ptr(b2)) if (b1 is not None or b2 is not None) else None
+        grads = AgentAttnGrads(_ptr(g["dq"]), _ptr(g["dk"]), _ptr(g["dv"]), _ptr(g.get("db1")), _ptr(g.get("db2")),
+                               _ptr(g.get("dwd")))
+        self._check(self.lib.agent_attn_backward(
+            self._h, _ptr(q), _ptr(k), _ptr(v), _ptr(d_out), grid_h, grid_w, n_agents,
+            ctypes.byref(bias) if bias is not None else None, _ptr(dwc_weight), ctypes.byref(grads), _ptr(ws),
+            ws.numel(), _stream_ptr(stream)))
+        return g
 
     def pool(self, q, grid_h: int, grid_w: int, pool_h: int, pool_w: int, out=None, stream=None):
         B, h, d = self.batch, self.heads, self.head_dim

@@ -23,7 +23,7 @@ NVCC_FLAGS = [
 ]
 # --use_fast_math is wanted only in the tensor-core kernels' exponent path, which uses explicit
 # ex2.approx anyway; the fp32 path must keep IEEE division and exp2f, so it is compiled without it.
-PRECISE_FILES = {"attn_simt.cu", "pool.cu", "api.cu"}
+PRECISE_FILES = {"attn_simt.cu", "pool.cu", "api.cu", "backward.cu"}
 
 
 def _nvcc() -> str:

@@ -511,6 +511,92 @@ int agent_attn_query_status(agent_attn_handle* h, void* stream) {
     return AA_OK;
 }
 
+// Workspace of the backward pass: [A | V_A | dV_A | dA | lse | dot | partial (max, sum)], fp32, each
+// region 256-byte aligned (V_A, dV_A and dA are cleared with one memset, so their regions have one size).
+namespace {
+struct BwdLayout {
+    size_t a, va, dva, da, lse, dot, part, total;
+};
+bool bwd_layout(const agent_attn_handle* h, int N, int n, BwdPlan* pl, BwdLayout* w) {
+    const int slabs = h->cfg.batch * h->cfg.heads;
+    if (!plan_backward(slabs, n, N, h->cfg.head_dim, h->sm_count, pl)) return false;
+    const size_t snd = align_up((size_t)slabs * n * h->cfg.head_dim * sizeof(float), 256);
+    const size_t sn = align_up((size_t)slabs * n * sizeof(float), 256);
+    w->a = 0; w->va = snd; w->dva = 2 * snd; w->da = 3 * snd;
+    w->lse = 4 * snd; w->dot = w->lse + sn; w->part = w->dot + sn;
+    w->total = w->part + align_up((size_t)slabs * pl->chunks * n * 2 * sizeof(float), 256);
+    return true;
+}
+}  // namespace
+
+size_t agent_attn_backward_workspace_bytes(const agent_attn_handle* h, int grid_h, int grid_w, int n_agents) {
+    if (!h || grid_h <= 0 || grid_w <= 0 || n_agents <= 0) return 0;
+    if ((long long)grid_h * grid_w > h->cfg.max_tokens || n_agents > h->cfg.max_agents) return 0;
+    BwdPlan pl;
+    BwdLayout w;
+    return bwd_layout(h, grid_h * grid_w, n_agents, &pl, &w) ? w.total : 0;
+}
+
+int agent_attn_backward(agent_attn_handle* h, const void* Q, const void* K, const void* V, const void* d_out,
+                        int grid_h, int grid_w, int n_agents, const agent_attn_bias* bias, const void* dwc_weight,
+                        const agent_attn_grads* grads, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!h) return AA_ERR_INVALID_ARG;
+    h->err[0] = 0;
+    if (!Q || !K || !V || !d_out || !grads || !workspace) return fail(h, AA_ERR_INVALID_ARG, "null pointer");
+    if (!grads->dq || !grads->dk || !grads->dv) return fail(h, AA_ERR_INVALID_ARG, "dq, dk and dv are required");
+    if (grads->dwd && !dwc_weight) return fail(h, AA_ERR_INVALID_ARG, "dwd requested without a depthwise filter");
+    if (grid_h <= 0 || grid_w <= 0) return fail(h, AA_ERR_INVALID_ARG, "grid must be positive");
+    if ((long long)grid_h * grid_w > 0x7fffffffLL) return fail(h, AA_ERR_INVALID_ARG, "grid too large");
+    const int N = grid_h * grid_w;
+    if (int rc = check_shape(h, N, n_agents)) return rc;
+    const int p = isqrt_exact(n_agents);
+    if (p < 0 || p > grid_h || p > grid_w)
+        return fail(h, AA_ERR_INVALID_ARG, "pooled agents need n = p*p with p <= min(grid_h, grid_w); got n=%d on %dx%d",
+                    n_agents, grid_h, grid_w);
+    const void* b1 = bias ? bias->b1 : nullptr;
+    const void* b2 = bias ? bias->b2 : nullptr;
+    const void* ptrs[] = {Q, K, V, d_out, workspace, grads->dq, grads->dk, grads->dv, grads->db1, grads->db2,
+                          grads->dwd, b1, b2, dwc_weight};
+    for (const void* q : ptrs)
+        if (q && misaligned(q)) return fail(h, AA_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
+    const void* outs[] = {grads->dq, grads->dk, grads->dv, grads->db1, grads->db2, grads->dwd};
+    const void* ins[] = {Q, K, V, d_out, b1, b2, dwc_weight};
+    for (size_t i = 0; i < 6; ++i) {
+        if (!outs[i]) continue;
+        for (const void* q : ins)
+            if (outs[i] == q) return fail(h, AA_ERR_INVALID_ARG, "a gradient buffer aliases an input");
+        for (size_t j = 0; j < i; ++j)
+            if (outs[i] == outs[j]) return fail(h, AA_ERR_INVALID_ARG, "two gradient buffers alias");
+    }
+    BwdCall c;
+    memset(&c, 0, sizeof(c));
+    BwdLayout w;
+    if (!bwd_layout(h, N, n_agents, &c.plan, &w))
+        return fail(h, AA_ERR_UNSUPPORTED, "backward needs n * head_dim <= 16384 (n=%d, d=%d)", n_agents, h->cfg.head_dim);
+    if (workspace_bytes < w.total)
+        return fail(h, AA_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", workspace_bytes, w.total);
+    DeviceGuard guard(h->cfg.device);
+    if (!guard.ok) return fail(h, AA_ERR_CUDA, "cannot select device %d", h->cfg.device);
+    h->launches = 0;
+    char* ws = static_cast<char*>(workspace);
+    c.q = Q; c.k = K; c.v = V; c.d_out = d_out; c.b1 = b1; c.b2 = b2; c.wd = dwc_weight;
+    c.dq = static_cast<float*>(grads->dq); c.dk = static_cast<float*>(grads->dk); c.dv = static_cast<float*>(grads->dv);
+    c.db1 = static_cast<float*>(grads->db1); c.db2 = static_cast<float*>(grads->db2);
+    c.dwd = static_cast<float*>(grads->dwd);
+    c.ws_a = reinterpret_cast<float*>(ws + w.a); c.ws_va = reinterpret_cast<float*>(ws + w.va);
+    c.ws_dva = reinterpret_cast<float*>(ws + w.dva); c.ws_da = reinterpret_cast<float*>(ws + w.da);
+    c.ws_lse = reinterpret_cast<float*>(ws + w.lse); c.ws_dot = reinterpret_cast<float*>(ws + w.dot);
+    c.ws_part = reinterpret_cast<float*>(ws + w.part);
+    c.clear_bytes = w.lse - w.va;
+    c.slabs = h->cfg.batch * h->cfg.heads; c.heads = h->cfg.heads; c.H = grid_h; c.W = grid_w;
+    c.d = h->cfg.head_dim; c.n = n_agents; c.p = p; c.sm_count = h->sm_count;
+    c.scale1 = h->scale1; c.scale2 = h->scale2;
+    cudaError_t e = launch_backward(h->cfg.dtype, c, (cudaStream_t)stream);
+    if (e != cudaSuccess) return fail(h, AA_ERR_CUDA, "backward launch failed: %s", cudaGetErrorString(e));
+    h->launches = backward_launch_count(c.dwd != nullptr);
+    return AA_OK;
+}
+
 }  // extern "C"
 
 // --------------------------------------------------------------------------------------------

@@ -143,4 +143,40 @@ cudaError_t launch_fused(int dtype, const FusedArgs& a, cudaStream_t st);
 int fused_parts_per_slab(int dtype, int H, int W, int d, int n_agents);   // 0 if the shape is not eligible
 inline size_t fused_counter_words(int slabs) { return 3 * (size_t)slabs + 4; }
 
+// ------------------------------------------------------------------------------ backward pass
+// Tiling of the backward kernels: tiles of `tile` tokens, `chunks` blocks per slab, each block
+// walking `tiles_per_chunk` consecutive tiles; np = agents padded to a multiple of 32, plus 1.
+struct BwdPlan {
+    int tile, np, tiles, chunks, tiles_per_chunk;
+};
+// Arguments of one backward kernel (set per launch by launch_backward).
+struct BwdArgs {
+    const void *x, *y;        // token rows [slabs][N][d]: operand of the logits, second operand
+    const void* bias;         // B1 [heads][n][N] or B2 [heads][N][n], or null
+    const float *m0, *m1;     // fp32 [slabs][n][d]: A; V_A or dV_A
+    const float *lse, *dot;   // fp32 [slabs][n]: log-sum-exp of the aggregation rows; dV_A . V_A
+    float* part;              // fp32 [slabs][chunks][n][2]: per-block (max, sum) of the aggregation logits
+    float *outer0, *outer1;   // fp32 [slabs][n][d]: sums over tokens (atomics)
+    float *row0, *row1;       // fp32 [slabs][N][d]: per-token results
+    float* dbias;             // fp32 in the layout of `bias` (atomics), or null
+    int slabs, heads, N, H, W, d, n, ph, pw;
+    int np, tile, tiles, chunks, tiles_per_chunk;
+    float scale;
+};
+// One backward call: inputs in the handle's element type, gradients and workspace in fp32.
+struct BwdCall {
+    const void *q, *k, *v, *d_out, *b1, *b2, *wd;
+    float *dq, *dk, *dv, *db1, *db2, *dwd;
+    float *ws_a, *ws_va, *ws_dva, *ws_da;     // [slabs][n][d] each; V_A, dV_A, dA contiguous in this order
+    float *ws_lse, *ws_dot;                   // [slabs][n]
+    float* ws_part;                           // [slabs][chunks][n][2]
+    size_t clear_bytes;                       // bytes from ws_va to the end of ws_da
+    int slabs, heads, H, W, d, n, p, sm_count;
+    float scale1, scale2;
+    BwdPlan plan;
+};
+bool plan_backward(int slabs, int n, int N, int d, int sm_count, BwdPlan* out);   // false: shape not supported
+int backward_launch_count(bool with_dwd);
+cudaError_t launch_backward(int dtype, const BwdCall& c, cudaStream_t st);
+
 }  // namespace aa

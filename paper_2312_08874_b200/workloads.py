@@ -112,6 +112,15 @@ def make_inputs(w: Workload, seed: Optional[int] = None,
     return out
 
 
+def make_upstream_grad(w: Workload, seed: Optional[int] = None) -> torch.Tensor:
+    """Upstream gradient dL/dO [B, heads, N, d] for the backward pass: fp32 standard normals from a
+    generator of its own (seed + 1000003), cast to the storage dtype."""
+    g = torch.Generator(device="cpu")
+    g.manual_seed((w.seed if seed is None else seed) + 1000003)
+    t = torch.randn((w.batch, w.heads, w.tokens, w.head_dim), generator=g, dtype=torch.float32)
+    return t.to(TORCH_DTYPE[w.dtype]).contiguous()
+
+
 def shard_slabs(total_batch: int, world_size: int, rank: int) -> range:
     """Batch entries owned by `rank` when a batch is split over `world_size` processes.
 
