@@ -147,6 +147,75 @@ def run_reference(args, w):
     }))
 
 
+def backward_flops(w) -> int:
+    """Algorithmic flops of the backward pass: eleven n x N x d products per slab (S1, V_A, S2 recomputed;
+    dV_A, dP2, dQ, dA (two terms), dP1, dK, dV), two flops per multiply-add, plus the two depthwise terms."""
+    mm = 11 * 2 * w.slabs * w.agents * w.tokens * w.head_dim
+    dw = 2 * 2 * 9 * w.slabs * w.tokens * w.head_dim if w.dwc else 0
+    return mm + dw
+
+
+def run_backward(args, w, mod, sets, rank, local_rank, world):
+    """Times agent_attn_backward on device-resident inputs (two rotating sets, each larger than the L2)."""
+    from paper_2312_08874_b200 import make_upstream_grad
+    dev = torch.device("cuda", local_rank)
+    go = make_upstream_grad(w, seed=w.seed + 1000 * rank).to(dev)
+    ws = mod.backward_workspace(w.grid_h, w.grid_w, w.agents)
+    stream = torch.cuda.current_stream()
+    steps = min(args.steps, 200)
+
+    def step(i):
+        d = sets[i % len(sets)]
+        return mod.backward(d["q"], d["k"], d["v"], go, w.grid_h, w.grid_w, w.agents, b1=d["b1"], b2=d["b2"],
+                            dwc_weight=d["dwc"], workspace=ws, stream=stream)
+
+    t_w = time.perf_counter()
+    i = 0
+    while i < args.warmup or time.perf_counter() - t_w < args.min_warmup_seconds:
+        g = step(i)
+        i += 1
+        if i % 16 == 0:
+            torch.cuda.synchronize()
+    torch.cuda.synchronize()
+    launches = mod.last_launch_count()
+    sampler = ClockSampler(local_rank)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    pdist.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    e0.record(stream)
+    for i in range(steps):
+        g = step(i)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    pdist.barrier()
+    clocks = sampler.stop()
+    ms_step = pdist.max_over_ranks(e0.elapsed_time(e1)) / steps
+    tokens_per_step = world * w.batch * w.tokens
+    # fp32 multiply-add peak of the CUDA cores: SMs x 128 lanes x 2 flops x the SM clock seen under load
+    props = torch.cuda.get_device_properties(dev)
+    mhz = clocks.get("sm_mhz") or clocks.get("sm_max_mhz") or 1965
+    peak = props.multi_processor_count * 128 * 2 * mhz * 1e6 / 1e12
+    tfl = backward_flops(w) / (ms_step * 1e-3) / 1e12
+    set_bytes = sum(t.numel() * t.element_size() for t in list(sets[0].values()) + list(g.values()) + [go]
+                    if t is not None) - sets[0]["out"].numel() * sets[0]["out"].element_size()
+    if rank == 0:
+        print(json.dumps({
+            "pass": "backward", "metric": "backward tokens/s", "value": tokens_per_step / (ms_step * 1e-3),
+            "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": args.warmup, "ms_per_step": ms_step,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": w.name, "batch_per_gpu": w.batch, "heads": w.heads, "tokens": w.tokens,
+                       "head_dim": w.head_dim, "agents": w.agents, "bias": w.bias, "dwc": w.dwc,
+                       "gradients": sorted(g), "l2": f"2 rotating input sets, {set_bytes / 1e6:.1f} MB touched per step"},
+            "clocks": clocks, "gpu_launches": launches * steps,
+            "roofline": {"bound": "alu", "kernel": "backward_path", "achieved": tfl, "peak": peak, "unit": "TFLOP/s",
+                         "frac": tfl / peak, "traffic": None,
+                         "peak_source": "SMs x 128 fp32 lanes x 2 x sampled SM clock",
+                         "algorithmic_flops": backward_flops(w), "algorithmic_bytes": set_bytes,
+                         "hbm_frac_if_bandwidth_bound": set_bytes / (ms_step * 1e-3) / 1e9 / measured_peaks()[0]},
+        }))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -158,6 +227,9 @@ def main():
     ap.add_argument("--layout", choices=["dense", "bnhd", "qkv"], default="dense",
                     help="storage of Q, K, V and out: dense [B,h,N,d]; bnhd = [B,N,h,d] (forward_strided); "
                          "qkv = Q, K, V interleaved as [B,N,3,h,d], out [B,N,h,d] (forward_strided)")
+    ap.add_argument("--direction", choices=["forward", "backward"], default="forward",
+                    help="backward: time agent_attn_backward (fp32 gradients of Q, K, V, both biases and the filter) "
+                         "instead of the forward pass; prints a line with \"pass\": \"backward\"")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--min-warmup-seconds", type=float, default=0.2)
     args = ap.parse_args()
@@ -202,6 +274,12 @@ def main():
     mod = AgentAttention(w.batch, w.heads, w.head_dim, w.tokens, w.agents, dt, device=local_rank)
     ws = mod.workspace(w.grid_h, w.grid_w, w.agents)
     stream = torch.cuda.current_stream()
+    if args.direction == "backward":
+        if args.layout != "dense":
+            raise SystemExit("the backward pass takes dense tensors")
+        run_backward(args, w, mod, sets[:2], rank, local_rank, world)
+        pdist.shutdown()
+        return
 
     def step(i):
         d = sets[i % n_sets]

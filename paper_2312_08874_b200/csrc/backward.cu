@@ -29,6 +29,13 @@ constexpr int kBwdWarps = kBwdThreads / 32;
 constexpr int kMaxLaneAgents = 8;                 // 256 agents / 32 lanes
 constexpr int kMaxOuter = 16;                     // float4 accumulators per thread: n * d / 4 <= 16 * 256
 
+// 0: n <= 64 and n d <= 4096;  1: n <= 128 and n d <= 8192;  2: n <= 256 and n d <= 16384
+__host__ __device__ inline int backward_variant(int n, int d) {
+    if (n <= 64 && n * d <= 4096) return 0;
+    if (n <= 128 && n * d <= 8192) return 1;
+    return 2;
+}
+
 enum BwdMode {
     kStats1 = 0,   // running (max, sum) of the aggregation logits over the block's tokens
     kVa1 = 1,      // V_A += P1 V
@@ -50,10 +57,15 @@ __device__ __forceinline__ float warp_sum(float v) {
     return v;
 }
 
-template <typename T, int MODE>
-__global__ void __launch_bounds__(kBwdThreads, 1) bwd_tile_kernel(BwdArgs p) {
+__device__ __forceinline__ float f4c(const float4& v, int i) { return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w; }
+
+// NT = agents per lane (n <= 32 NT), KOUT = float4 sums over tokens per thread (n d / 4 <= 256 KOUT),
+// TOK = tokens a warp works on at once (they share every load of the agents' matrices).
+template <typename T, int MODE, int NT, int KOUT, int TOK>
+__global__ void __launch_bounds__(kBwdThreads, KOUT <= 4 ? 2 : 1) bwd_tile_kernel(BwdArgs p) {
     constexpr bool kHasM1 = MODE == kBcast2 || MODE == kAgg1;
     constexpr bool kRowSoftmax = MODE == kBcast2;
+    constexpr int kOut = MODE == kStats1 ? 0 : KOUT;
     extern __shared__ __align__(16) float sm[];
     const int d = p.d, n = p.n, np = p.np, tt = p.tile;
     float* m0t = sm;                                        // [d][np]  A^T
@@ -77,19 +89,19 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_tile_kernel(BwdArgs p) {
         if (kHasM1) m1t[c * np + r] = p.m1[slab * nd + i];
     }
 
-    float lse[kMaxLaneAgents], dot[kMaxLaneAgents];        // per-agent row statistics of the aggregation
-    float run_m[kMaxLaneAgents], run_l[kMaxLaneAgents];
+    float lse[NT], dot[NT];                                // per-agent row statistics of the aggregation
+    float run_m[NT], run_l[NT];
 #pragma unroll
-    for (int t = 0; t < kMaxLaneAgents; ++t) {
+    for (int t = 0; t < NT; ++t) {
         const int r = lane + 32 * t;
         lse[t] = (MODE == kVa1 || MODE == kAgg1) && r < n ? p.lse[(size_t)slab * n + r] : 0.f;
         dot[t] = MODE == kAgg1 && r < n ? p.dot[(size_t)slab * n + r] : 0.f;
         run_m[t] = -INFINITY;
         run_l[t] = 0.f;
     }
-    float4 acc0[kMaxOuter], acc1[kMaxOuter];
+    float4 acc0[KOUT], acc1[KOUT];
 #pragma unroll
-    for (int k = 0; k < kMaxOuter; ++k) acc0[k] = acc1[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int k = 0; k < KOUT; ++k) acc0[k] = acc1[k] = make_float4(0.f, 0.f, 0.f, 0.f);
     const int outer_total = n * (d >> 2);
 
     const T* xg = static_cast<const T*>(p.x) + (size_t)slab * p.N * d;
@@ -108,103 +120,129 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_tile_kernel(BwdArgs p) {
         }
         __syncthreads();
 
-        for (int tl = warp; tl < tt; tl += kBwdWarps) {
-            const int tok = tok0 + tl;
-            const bool valid = tok < p.N;
-            float s[kMaxLaneAgents], dp[kMaxLaneAgents];
+        for (int tb = warp * TOK; tb < tt; tb += kBwdWarps * TOK) {      // tokens tb .. tb + TOK - 1 of the tile
+            float s[TOK][NT], dp[TOK][NT];
 #pragma unroll
-            for (int t = 0; t < kMaxLaneAgents; ++t) s[t] = dp[t] = 0.f;
-            const float* xr = xs + (size_t)tl * d;
-            const float* yr = ys + (size_t)tl * d;
-            for (int c = 0; c < d; ++c) {
-                const float xv = xr[c];
-                const float yv = kHasM1 ? yr[c] : 0.f;
+            for (int k = 0; k < TOK; ++k)
 #pragma unroll
-                for (int t = 0; t < kMaxLaneAgents; ++t)
-                    if (t < nt) {
-                        s[t] = fmaf(xv, m0t[c * np + lane + 32 * t], s[t]);
-                        if (kHasM1) dp[t] = fmaf(yv, m1t[c * np + lane + 32 * t], dp[t]);
-                    }
+                for (int t = 0; t < NT; ++t) s[k][t] = dp[k][t] = 0.f;
+            for (int c = 0; c < d; c += 4) {
+                float4 xv[TOK], yv[TOK];
+#pragma unroll
+                for (int k = 0; k < TOK; ++k) {
+                    xv[k] = *reinterpret_cast<const float4*>(xs + (size_t)(tb + k) * d + c);
+                    if (kHasM1) yv[k] = *reinterpret_cast<const float4*>(ys + (size_t)(tb + k) * d + c);
+                }
+#pragma unroll
+                for (int cc = 0; cc < 4; ++cc)
+#pragma unroll
+                    for (int t = 0; t < NT; ++t)
+                        if (t < nt) {
+                            const float a0 = m0t[(c + cc) * np + lane + 32 * t];
+                            const float a1 = kHasM1 ? m1t[(c + cc) * np + lane + 32 * t] : 0.f;
+#pragma unroll
+                            for (int k = 0; k < TOK; ++k) {
+                                s[k][t] = fmaf(f4c(xv[k], cc), a0, s[k][t]);
+                                if (kHasM1) dp[k][t] = fmaf(f4c(yv[k], cc), a1, dp[k][t]);
+                            }
+                        }
             }
 #pragma unroll
-            for (int t = 0; t < kMaxLaneAgents; ++t) {
-                const int r = lane + 32 * t;
-                if (t < nt && r < n && valid) {
-                    float b = 0.f;
-                    if (bias)
-                        b = kRowSoftmax ? ld_f32(bias, ((size_t)head * p.N + tok) * n + r)
-                                        : ld_f32(bias, ((size_t)head * n + r) * p.N + tok);
-                    s[t] = fmaf(p.scale, s[t], b);
+            for (int k = 0; k < TOK; ++k) {
+                const int tl = tb + k, tok = tok0 + tl;
+                const bool valid = tok < p.N;
+#pragma unroll
+                for (int t = 0; t < NT; ++t) {
+                    const int r = lane + 32 * t;
+                    if (t < nt && r < n && valid) {
+                        float b = 0.f;
+                        if (bias)
+                            b = kRowSoftmax ? ld_f32(bias, ((size_t)head * p.N + tok) * n + r)
+                                            : ld_f32(bias, ((size_t)head * n + r) * p.N + tok);
+                        s[k][t] = fmaf(p.scale, s[k][t], b);
+                    } else {
+                        s[k][t] = -INFINITY;
+                    }
+                }
+                if (MODE == kStats1) {
+#pragma unroll
+                    for (int t = 0; t < NT; ++t)
+                        if (s[k][t] > -INFINITY) {
+                            const float m = fmaxf(run_m[t], s[k][t]);
+                            run_l[t] = run_l[t] * expf(run_m[t] - m) + expf(s[k][t] - m);
+                            run_m[t] = m;
+                        }
                 } else {
-                    s[t] = -INFINITY;
-                }
-            }
-            if (MODE == kStats1) {
+                    float prob[NT], rdot[NT];
+                    if (kRowSoftmax) {
+                        float m = -INFINITY;
 #pragma unroll
-                for (int t = 0; t < kMaxLaneAgents; ++t)
-                    if (s[t] > -INFINITY) {
-                        const float m = fmaxf(run_m[t], s[t]);
-                        run_l[t] = run_l[t] * expf(run_m[t] - m) + expf(s[t] - m);
-                        run_m[t] = m;
+                        for (int t = 0; t < NT; ++t) m = fmaxf(m, s[k][t]);
+                        m = warp_max(m);
+                        float l = 0.f;
+#pragma unroll
+                        for (int t = 0; t < NT; ++t) {
+                            prob[t] = valid && s[k][t] > -INFINITY ? expf(s[k][t] - m) : 0.f;
+                            l += prob[t];
+                        }
+                        l = warp_sum(l);
+                        const float inv = valid ? 1.f / l : 0.f;
+                        float rd = 0.f;
+#pragma unroll
+                        for (int t = 0; t < NT; ++t) {
+                            prob[t] *= inv;
+                            rd = fmaf(prob[t], dp[k][t], rd);
+                        }
+                        rd = warp_sum(rd);
+#pragma unroll
+                        for (int t = 0; t < NT; ++t) rdot[t] = rd;
+                    } else {
+#pragma unroll
+                        for (int t = 0; t < NT; ++t) {
+                            prob[t] = s[k][t] > -INFINITY ? expf(s[k][t] - lse[t]) : 0.f;
+                            rdot[t] = dot[t];
+                        }
                     }
-                continue;
-            }
-            float prob[kMaxLaneAgents];
-            if (kRowSoftmax) {
-                float m = -INFINITY;
 #pragma unroll
-                for (int t = 0; t < kMaxLaneAgents; ++t) m = fmaxf(m, s[t]);
-                m = warp_max(m);
-                float l = 0.f;
-#pragma unroll
-                for (int t = 0; t < kMaxLaneAgents; ++t) {
-                    prob[t] = valid && s[t] > -INFINITY ? expf(s[t] - m) : 0.f;
-                    l += prob[t];
-                }
-                l = warp_sum(l);
-                const float inv = valid ? 1.f / l : 0.f;
-                float rd = 0.f;
-#pragma unroll
-                for (int t = 0; t < kMaxLaneAgents; ++t) {
-                    prob[t] *= inv;
-                    rd = fmaf(prob[t], dp[t], rd);
-                }
-                rd = warp_sum(rd);
-#pragma unroll
-                for (int t = 0; t < kMaxLaneAgents; ++t) dot[t] = rd;
-            } else {
-#pragma unroll
-                for (int t = 0; t < kMaxLaneAgents; ++t) prob[t] = s[t] > -INFINITY ? expf(s[t] - lse[t]) : 0.f;
-            }
-#pragma unroll
-            for (int t = 0; t < kMaxLaneAgents; ++t) {
-                const int r = lane + 32 * t;
-                if (t < nt) {
-                    pt[(size_t)tl * np + r] = prob[t];
-                    if (kHasM1) {
-                        const float g = prob[t] * (dp[t] - dot[t]);
-                        dst[(size_t)tl * np + r] = g;
-                        if (p.dbias && valid && r < n) {
-                            float* o = kRowSoftmax ? p.dbias + ((size_t)head * p.N + tok) * n + r
-                                                   : p.dbias + ((size_t)head * n + r) * p.N + tok;
-                            atomicAdd(o, g);
+                    for (int t = 0; t < NT; ++t) {
+                        const int r = lane + 32 * t;
+                        if (t < nt) {
+                            pt[(size_t)tl * np + r] = prob[t];
+                            if (kHasM1) {
+                                const float g = prob[t] * (dp[k][t] - rdot[t]);
+                                dst[(size_t)tl * np + r] = g;
+                                if (p.dbias && valid && r < n) {
+                                    float* o = kRowSoftmax ? p.dbias + ((size_t)head * p.N + tok) * n + r
+                                                           : p.dbias + ((size_t)head * n + r) * p.N + tok;
+                                    atomicAdd(o, g);
+                                }
+                            }
                         }
                     }
                 }
             }
             if (kHasM1) {
                 __syncwarp();
-                if (valid) {
-                    const float* gr = dst + (size_t)tl * np;
-                    const float* pr = pt + (size_t)tl * np;
-                    for (int c = lane; c < d; c += 32) {
-                        float a0 = 0.f, a1 = 0.f;
-                        for (int r = 0; r < n; ++r) {
-                            a0 = fmaf(gr[r], m0t[c * np + r], a0);
-                            if (MODE == kAgg1) a1 = fmaf(pr[r], m1t[c * np + r], a1);
+                for (int c = lane; c < d; c += 32) {
+                    float a0[TOK], a1[TOK];
+#pragma unroll
+                    for (int k = 0; k < TOK; ++k) a0[k] = a1[k] = 0.f;
+                    for (int r = 0; r < n; ++r) {
+                        const float w0 = m0t[c * np + r];
+                        const float w1 = MODE == kAgg1 ? m1t[c * np + r] : 0.f;
+#pragma unroll
+                        for (int k = 0; k < TOK; ++k) {
+                            a0[k] = fmaf(dst[(size_t)(tb + k) * np + r], w0, a0[k]);
+                            if (MODE == kAgg1) a1[k] = fmaf(pt[(size_t)(tb + k) * np + r], w1, a1[k]);
                         }
-                        p.row0[((size_t)slab * p.N + tok) * d + c] = p.scale * a0;
-                        if (MODE == kAgg1) p.row1[((size_t)slab * p.N + tok) * d + c] = a1;
+                    }
+#pragma unroll
+                    for (int k = 0; k < TOK; ++k) {
+                        const int tok = tok0 + tb + k;
+                        if (tok < p.N) {
+                            p.row0[((size_t)slab * p.N + tok) * d + c] = p.scale * a0[k];
+                            if (MODE == kAgg1) p.row1[((size_t)slab * p.N + tok) * d + c] = a1[k];
+                        }
                     }
                 }
             }
@@ -212,7 +250,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_tile_kernel(BwdArgs p) {
         if (MODE != kStats1) __syncthreads();
         // sums over the tile's tokens of (per-agent weight) x (token row): thread owns (r, 4 channels)
 #pragma unroll
-        for (int k = 0; k < (MODE == kStats1 ? 0 : kMaxOuter); ++k) {
+        for (int k = 0; k < kOut; ++k) {
             const int o = tid + kBwdThreads * k;
             if (o < outer_total) {
                 const int c4 = o / n, r = o - c4 * n;
@@ -239,7 +277,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_tile_kernel(BwdArgs p) {
         __syncthreads();
         float* red = pt;                                   // [warps][np][2]
 #pragma unroll
-        for (int t = 0; t < kMaxLaneAgents; ++t)
+        for (int t = 0; t < NT; ++t)
             if (t < nt) {
                 red[((size_t)warp * np + lane + 32 * t) * 2] = run_m[t];
                 red[((size_t)warp * np + lane + 32 * t) * 2 + 1] = run_l[t];
@@ -260,7 +298,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_tile_kernel(BwdArgs p) {
         }
     }
 #pragma unroll
-    for (int k = 0; k < (MODE == kStats1 ? 0 : kMaxOuter); ++k) {
+    for (int k = 0; k < kOut; ++k) {
         const int o = tid + kBwdThreads * k;
         if (o < outer_total) {
             const int c4 = o / n, r = o - c4 * n;
@@ -322,52 +360,83 @@ __global__ void bwd_dot_kernel(BwdArgs p, const float* va, const float* dva, flo
     dot[i] = acc;
 }
 
+// Four consecutive elements of a token row as fp32.
+template <typename T> __device__ __forceinline__ float4 ld4_f32(const T* p);
+template <> __device__ __forceinline__ float4 ld4_f32<float>(const float* p) { return *reinterpret_cast<const float4*>(p); }
+template <> __device__ __forceinline__ float4 ld4_f32<__nv_bfloat16>(const __nv_bfloat16* p) {
+    const uint2 w = *reinterpret_cast<const uint2*>(p);
+    const float2 a = unpack2<__nv_bfloat16>(w.x), b = unpack2<__nv_bfloat16>(w.y);
+    return make_float4(a.x, a.y, b.x, b.y);
+}
+template <> __device__ __forceinline__ float4 ld4_f32<__half>(const __half* p) {
+    const uint2 w = *reinterpret_cast<const uint2*>(p);
+    const float2 a = unpack2<__half>(w.x), b = unpack2<__half>(w.y);
+    return make_float4(a.x, a.y, b.x, b.y);
+}
+
 // Token-wise tail: dQ += Pooling^T(dA) (each window spreads its agent's gradient evenly over its
 // tokens) and dV += DWC^T(dO) (tap (u, v) of output token (y, x) read V[y+u-1][x+v-1]).
+// One thread per (slab, token, 4 channels).
 template <typename T>
-__global__ void bwd_tail_kernel(BwdArgs p, const float* da, const void* gov, const void* wdv, float* dq, float* dv) {
-    const size_t total = (size_t)p.slabs * p.N * p.d;
+__global__ void __launch_bounds__(256) bwd_tail_kernel(BwdArgs p, const float* da, const void* gov, const void* wdv,
+                                                       float* dq, float* dv) {
+    const int d4 = p.d >> 2;
+    const size_t total = (size_t)p.slabs * p.N * d4;
     const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= total) return;
-    const int c = (int)(i % p.d);
-    const int tok = (int)((i / p.d) % p.N);
-    const int slab = (int)(i / ((size_t)p.d * p.N));
+    const int c = (int)(i % d4) * 4;
+    const size_t st = i / d4;                                    // slab * N + token
+    const int tok = (int)(st % p.N);
+    const int slab = (int)(st / p.N);
     const int y = tok / p.W, x = tok - y * p.W;
     const int ayc = (y * p.ph) / p.H, axc = (x * p.pw) / p.W;
-    float g = 0.f;
+    float4 g = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int ay = max(ayc - 1, 0); ay <= min(ayc + 1, p.ph - 1); ++ay) {
         const int y0 = (ay * p.H) / p.ph, y1 = ((ay + 1) * p.H + p.ph - 1) / p.ph;
         if (y < y0 || y >= y1) continue;
         for (int ax = max(axc - 1, 0); ax <= min(axc + 1, p.pw - 1); ++ax) {
             const int x0 = (ax * p.W) / p.pw, x1 = ((ax + 1) * p.W + p.pw - 1) / p.pw;
             if (x < x0 || x >= x1) continue;
-            g += da[((size_t)slab * p.n + ay * p.pw + ax) * p.d + c] / (float)((y1 - y0) * (x1 - x0));
+            const float cnt = (float)((y1 - y0) * (x1 - x0));
+            const float4 a = *reinterpret_cast<const float4*>(da + ((size_t)slab * p.n + ay * p.pw + ax) * p.d + c);
+            g.x += a.x / cnt; g.y += a.y / cnt; g.z += a.z / cnt; g.w += a.w / cnt;
         }
     }
-    dq[i] += g;
+    float4* qo = reinterpret_cast<float4*>(dq + st * p.d + c);
+    float4 qv = *qo;
+    qv.x += g.x; qv.y += g.y; qv.z += g.z; qv.w += g.w;
+    *qo = qv;
     if (wdv) {
         const int head = slab % p.heads;
-        const T* w = static_cast<const T*>(wdv) + ((size_t)head * p.d + c) * 9;
+        const T* w = static_cast<const T*>(wdv) + ((size_t)head * p.d + c) * 9;     // [4 channels][9 taps]
         const T* go = static_cast<const T*>(gov) + (size_t)slab * p.N * p.d;
-        float acc = 0.f;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
         for (int u = 0; u < 3; ++u)
+#pragma unroll
             for (int v = 0; v < 3; ++v) {
                 const int yo = y - u + 1, xo = x - v + 1;          // the output token whose tap (u, v) is (y, x)
                 if (yo < 0 || yo >= p.H || xo < 0 || xo >= p.W) continue;
-                acc = fmaf(ld_f32(w, u * 3 + v), ld_f32(go, ((size_t)yo * p.W + xo) * p.d + c), acc);
+                const float4 gv = ld4_f32<T>(go + ((size_t)yo * p.W + xo) * p.d + c);
+                const int k = u * 3 + v;
+                acc.x = fmaf(ld_f32(w, k), gv.x, acc.x);      acc.y = fmaf(ld_f32(w, 9 + k), gv.y, acc.y);
+                acc.z = fmaf(ld_f32(w, 18 + k), gv.z, acc.z); acc.w = fmaf(ld_f32(w, 27 + k), gv.w, acc.w);
             }
-        dv[i] += acc;
+        float4* vo = reinterpret_cast<float4*>(dv + st * p.d + c);
+        float4 vv = *vo;
+        vv.x += acc.x; vv.y += acc.y; vv.z += acc.z; vv.w += acc.w;
+        *vo = vv;
     }
 }
 
 // dWd[head][c][u][v] = sum over batch and output tokens of dO[y][x][c] * V[y+u-1][x+v-1][c].
 // Block = (slab, token chunk); thread = (token lane, channel); per-block sums are added with atomics.
 template <typename T>
-__global__ void __launch_bounds__(256) bwd_dwd_kernel(BwdArgs p, const void* gov, const void* vv, float* dwd, int chunks) {
-    __shared__ float red[256 * 9];
+__global__ void __launch_bounds__(512) bwd_dwd_kernel(BwdArgs p, const void* gov, const void* vv, float* dwd, int chunks) {
+    __shared__ float red[512 * 9];
     const int slab = blockIdx.x / chunks, chunk = blockIdx.x - slab * chunks;
     const int head = slab % p.heads;
-    const int lanes = 256 / p.d > 0 ? 256 / p.d : 1;              // token lanes (d <= 128: at least 2)
+    const int lanes = 512 / p.d;                                  // token lanes (d <= 128: at least 4)
     const int c = threadIdx.x % p.d, tlane = threadIdx.x / p.d;
     const int per = (p.N + chunks - 1) / chunks;
     const int t0 = chunk * per, t1 = min(t0 + per, p.N);
@@ -401,14 +470,26 @@ __global__ void __launch_bounds__(256) bwd_dwd_kernel(BwdArgs p, const void* gov
     }
 }
 
-template <typename T, int MODE>
-cudaError_t launch_tile(const BwdArgs& a, cudaStream_t st) {
+template <typename T, int MODE, int NT, int KOUT, int TOK>
+cudaError_t launch_tile_cfg(const BwdArgs& a, cudaStream_t st) {
     const bool m1 = MODE == kBcast2 || MODE == kAgg1;
     const size_t smem = ((size_t)a.d * a.np * (m1 ? 2 : 1) + 2 * (size_t)a.tile * a.d + 2 * (size_t)a.tile * a.np) * sizeof(float);
-    cudaError_t e = cudaFuncSetAttribute(bwd_tile_kernel<T, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(bwd_tile_kernel<T, MODE, NT, KOUT, TOK>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    bwd_tile_kernel<T, MODE><<<a.slabs * a.chunks, kBwdThreads, smem, st>>>(a);
+    bwd_tile_kernel<T, MODE, NT, KOUT, TOK><<<a.slabs * a.chunks, kBwdThreads, smem, st>>>(a);
     return cudaGetLastError();
+}
+
+// Three register budgets: few agents (four tokens per warp at once, two blocks per SM), up to 128 agents,
+// and the general case.
+template <typename T, int MODE>
+cudaError_t launch_tile(const BwdArgs& a, cudaStream_t st) {
+    switch (backward_variant(a.n, a.d)) {
+        case 0:  return launch_tile_cfg<T, MODE, 2, 4, 4>(a, st);
+        case 1:  return launch_tile_cfg<T, MODE, 4, 8, 2>(a, st);
+        default: return launch_tile_cfg<T, MODE, kMaxLaneAgents, kMaxOuter, 1>(a, st);
+    }
 }
 
 template <typename T>
@@ -445,12 +526,12 @@ cudaError_t backward_typed(const BwdCall& c, BwdArgs a, cudaStream_t st) {
     a.outer0 = nullptr; a.outer1 = c.ws_da; a.row0 = c.dk; a.row1 = c.dv; a.dbias = c.db1;
     AA_TRY((launch_tile<T, kAgg1>(a, st)));
     // pooling and depthwise terms
-    bwd_tail_kernel<T><<<(unsigned)((tok_elems + 255) / 256), 256, 0, st>>>(a, c.ws_da, c.d_out, c.wd, c.dq, c.dv);
+    bwd_tail_kernel<T><<<(unsigned)((tok_elems / 4 + 255) / 256), 256, 0, st>>>(a, c.ws_da, c.d_out, c.wd, c.dq, c.dv);
     AA_TRY(cudaGetLastError());
     if (c.dwd) {
-        int chunks = (2 * c.sm_count + a.slabs - 1) / a.slabs;
+        int chunks = (4 * c.sm_count + a.slabs - 1) / a.slabs;          // short loops (they are load-latency bound), few atomics
         chunks = max(1, min(chunks, (a.N + 63) / 64));
-        bwd_dwd_kernel<T><<<a.slabs * chunks, 256, 0, st>>>(a, c.d_out, c.v, c.dwd, chunks);
+        bwd_dwd_kernel<T><<<a.slabs * chunks, 512, 0, st>>>(a, c.d_out, c.v, c.dwd, chunks);
         AA_TRY(cudaGetLastError());
     }
 #undef AA_TRY
@@ -474,7 +555,9 @@ bool plan_backward(int slabs, int n, int N, int d, int sm_count, BwdPlan* out) {
     pl.tile = tile;
     pl.np = (n + 31) / 32 * 32 + 1;
     pl.tiles = (N + tile - 1) / tile;
-    int chunks = (2 * sm_count + slabs - 1) / slabs;            // about two blocks per SM over all slabs
+    // one wave of blocks where the slabs allow it: two blocks per SM fit for few agents, else one
+    const int slots = sm_count * (backward_variant(n, d) == 0 ? 2 : 1);
+    int chunks = slots >= slabs ? slots / slabs : 1;
     chunks = max(1, min(chunks, pl.tiles));
     pl.tiles_per_chunk = (pl.tiles + chunks - 1) / chunks;
     pl.chunks = (pl.tiles + pl.tiles_per_chunk - 1) / pl.tiles_per_chunk;
