@@ -53,3 +53,41 @@ def test_pins_catch_mutant(tmp_path, name, old, new):
                         os.path.join(ROOT, "tests", "test_oracle_pins.py")],
                        env=env, cwd=ROOT, stdout=subprocess.PIPE, stderr=subprocess.STDOUT)
     assert r.returncode != 0, f"pins did not notice mutant '{name}'"
+
+
+# The same for the backward oracle: each mutant must fail the backward pins (finite differences of the
+# forward oracle, the adjoint identity, the closed forms).
+BACKWARD_PINS = os.path.join(ROOT, "tests", "test_oracle_backward_pins.py")
+BACKWARD_MUTANTS = [
+    ("bwd_broadcast_softmax_jacobian_without_row_term",
+     "p2[(size_t)i * n + r] * (ds[(size_t)i * n + r] - dot)", "p2[(size_t)i * n + r] * (ds[(size_t)i * n + r])"),
+    ("bwd_aggregation_softmax_jacobian_without_row_term",
+     "p1[(size_t)r * N + j] * (ds[(size_t)r * N + j] - dot)", "p1[(size_t)r * N + j] * (ds[(size_t)r * N + j])"),
+    ("bwd_dq_wrong_scale", "gq[(size_t)i * d + c] = scale2 * acc;", "gq[(size_t)i * d + c] = scale1 * acc;"),
+    ("bwd_dk_wrong_scale", "gk[(size_t)j * d + c] = scale1 * gk_acc;", "gk[(size_t)j * d + c] = scale2 * gk_acc;"),
+    ("bwd_agent_gradient_loses_broadcast_term",
+     "da[(size_t)r * d + c] += scale1 * acc;", "da[(size_t)r * d + c] = scale1 * acc;"),
+    ("bwd_dv_uses_logit_gradient",
+     "gv_acc += p1[(size_t)r * N + j] * dva[(size_t)r * d + c];", "gv_acc += ds[(size_t)r * N + j] * dva[(size_t)r * d + c];"),
+    ("bwd_depthwise_not_transposed",
+     "const int yy = y + u - 1, xx = x + t - 1;", "const int yy = y - u + 1, xx = x - t + 1;"),
+    ("bwd_pooling_sum_not_mean",
+     "da[(size_t)(ay * pw + ax) * d + c] * inv;", "da[(size_t)(ay * pw + ax) * d + c] * 1.0;"),
+    ("bwd_bias_gradient_not_summed_over_batch",
+     "if (dB2) dB2[head * nN + (size_t)i * n + r] += g;", "if (dB2) dB2[head * nN + (size_t)i * n + r] = g;"),
+]
+
+
+@pytest.mark.parametrize("name,old,new", BACKWARD_MUTANTS, ids=[m[0] for m in BACKWARD_MUTANTS])
+def test_backward_pins_catch_mutant(tmp_path, name, old, new):
+    src = open(SRC).read()
+    assert src.count(old) == 1, "mutation site must be unique in the oracle source"
+    mutated = tmp_path / "mutant.c"
+    mutated.write_text(src.replace(old, new))
+    lib = tmp_path / "libmutant.so"
+    subprocess.check_call(["gcc", "-O1", "-fopenmp", "-shared", "-fPIC", "-o", str(lib),
+                           str(mutated), "-lm"])
+    env = dict(os.environ, AGENT_ATTENTION_ORACLE_LIB=str(lib))
+    r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-p", "no:cacheprovider", BACKWARD_PINS],
+                       env=env, cwd=ROOT, stdout=subprocess.PIPE, stderr=subprocess.STDOUT)
+    assert r.returncode != 0, f"backward pins did not notice mutant '{name}'"
