@@ -591,6 +591,9 @@ int agent_attn_backward(agent_attn_handle* h, const void* Q, const void* K, cons
     c.slabs = h->cfg.batch * h->cfg.heads; c.heads = h->cfg.heads; c.H = grid_h; c.W = grid_w;
     c.d = h->cfg.head_dim; c.n = n_agents; c.p = p; c.sm_count = h->sm_count;
     c.scale1 = h->scale1; c.scale2 = h->scale2;
+    c.dtype = h->cfg.dtype;
+    c.use_mma = h->cfg.path == AA_PATH_AUTO && backward_mma_eligible(h->cfg.dtype, n_agents, h->cfg.head_dim);
+    if (c.use_mma) c.plan_mma = plan_backward_mma(c.slabs, N, h->sm_count);
     cudaError_t e = launch_backward(h->cfg.dtype, c, (cudaStream_t)stream);
     if (e != cudaSuccess) return fail(h, AA_ERR_CUDA, "backward launch failed: %s", cudaGetErrorString(e));
     h->launches = backward_launch_count(c.dwd != nullptr);

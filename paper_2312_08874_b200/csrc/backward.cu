@@ -517,14 +517,28 @@ cudaError_t backward_typed(const BwdCall& c, BwdArgs a, cudaStream_t st) {
     // broadcast backward
     a.x = c.q; a.y = c.d_out; a.bias = c.b2; a.m0 = c.ws_a; a.m1 = c.ws_va; a.scale = c.scale2;
     a.outer0 = c.ws_dva; a.outer1 = c.ws_da; a.row0 = c.dq; a.row1 = nullptr; a.dbias = c.db2;
-    AA_TRY((launch_tile<T, kBcast2>(a, st)));
+    if (c.use_mma) {
+        BwdArgs m = a;
+        m.np = c.plan_mma.np; m.tile = c.plan_mma.tile; m.tiles = c.plan_mma.tiles;
+        m.chunks = c.plan_mma.chunks; m.tiles_per_chunk = c.plan_mma.tiles_per_chunk;
+        AA_TRY(launch_backward_mma(c.dtype, true, m, st));
+    } else {
+        AA_TRY((launch_tile<T, kBcast2>(a, st)));
+    }
     bwd_dot_kernel<<<(unsigned)((sn + 255) / 256), 256, 0, st>>>(a, c.ws_va, c.ws_dva, c.ws_dot);
     AA_TRY(cudaGetLastError());
     // aggregation backward
     a.x = c.k; a.y = c.v; a.bias = c.b1; a.m0 = c.ws_a; a.m1 = c.ws_dva; a.scale = c.scale1;
     a.lse = c.ws_lse; a.dot = c.ws_dot;
     a.outer0 = nullptr; a.outer1 = c.ws_da; a.row0 = c.dk; a.row1 = c.dv; a.dbias = c.db1;
-    AA_TRY((launch_tile<T, kAgg1>(a, st)));
+    if (c.use_mma) {
+        BwdArgs m = a;
+        m.np = c.plan_mma.np; m.tile = c.plan_mma.tile; m.tiles = c.plan_mma.tiles;
+        m.chunks = c.plan_mma.chunks; m.tiles_per_chunk = c.plan_mma.tiles_per_chunk;
+        AA_TRY(launch_backward_mma(c.dtype, false, m, st));
+    } else {
+        AA_TRY((launch_tile<T, kAgg1>(a, st)));
+    }
     // pooling and depthwise terms
     bwd_tail_kernel<T><<<(unsigned)((tok_elems / 4 + 255) / 256), 256, 0, st>>>(a, c.ws_da, c.d_out, c.wd, c.dq, c.dv);
     AA_TRY(cudaGetLastError());

@@ -174,9 +174,16 @@ struct BwdCall {
     int slabs, heads, H, W, d, n, p, sm_count;
     float scale1, scale2;
     BwdPlan plan;
+    int dtype;                                // element type of the inputs (kF32, kBF16, kF16)
+    int use_mma;                              // the two gradient stages run on the tensor-core kernels
+    BwdPlan plan_mma;                         // their tiling
 };
 bool plan_backward(int slabs, int n, int N, int d, int sm_count, BwdPlan* out);   // false: shape not supported
 int backward_launch_count(bool with_dwd);
 cudaError_t launch_backward(int dtype, const BwdCall& c, cudaStream_t st);
+// Tensor-core kernels of the two gradient stages (16-bit inputs, n <= 64, d = 64)
+bool backward_mma_eligible(int dtype, int n, int d);
+BwdPlan plan_backward_mma(int slabs, int N, int sm_count);
+cudaError_t launch_backward_mma(int dtype, bool broadcast_stage, const BwdArgs& a, cudaStream_t st);
 
 }  // namespace aa
