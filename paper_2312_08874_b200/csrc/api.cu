@@ -524,7 +524,12 @@ bool bwd_layout(const agent_attn_handle* h, int N, int n, BwdPlan* pl, BwdLayout
     const size_t sn = align_up((size_t)slabs * n * sizeof(float), 256);
     w->a = 0; w->va = snd; w->dva = 2 * snd; w->da = 3 * snd;
     w->lse = 4 * snd; w->dot = w->lse + sn; w->part = w->dot + sn;
-    w->total = w->part + align_up((size_t)slabs * pl->chunks * n * 2 * sizeof(float), 256);
+    size_t part_floats = (size_t)slabs * pl->chunks * n * 2;
+    if (backward_mma_eligible(h->cfg.dtype, n, h->cfg.head_dim)) {      // partials of the tensor-core stage 1
+        const size_t mma_floats = backward_mma_part_floats(slabs, plan_backward_mma(slabs, N, h->sm_count));
+        if (part_floats < mma_floats) part_floats = mma_floats;
+    }
+    w->total = w->part + align_up(part_floats * sizeof(float), 256);
     return true;
 }
 }  // namespace
@@ -596,7 +601,7 @@ int agent_attn_backward(agent_attn_handle* h, const void* Q, const void* K, cons
     if (c.use_mma) c.plan_mma = plan_backward_mma(c.slabs, N, h->sm_count);
     cudaError_t e = launch_backward(h->cfg.dtype, c, (cudaStream_t)stream);
     if (e != cudaSuccess) return fail(h, AA_ERR_CUDA, "backward launch failed: %s", cudaGetErrorString(e));
-    h->launches = backward_launch_count(c.dwd != nullptr);
+    h->launches = backward_launch_count(c.dwd != nullptr, c.use_mma != 0);
     return AA_OK;
 }
 

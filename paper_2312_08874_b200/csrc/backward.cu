@@ -509,11 +509,19 @@ cudaError_t backward_typed(const BwdCall& c, BwdArgs a, cudaStream_t st) {
     // aggregation forward: row statistics, then V_A
     a.x = c.k; a.y = c.v; a.bias = c.b1; a.m0 = c.ws_a; a.m1 = nullptr; a.scale = c.scale1;
     a.part = c.ws_part; a.dbias = nullptr;
-    AA_TRY((launch_tile<T, kStats1>(a, st)));
-    bwd_lse_kernel<<<(unsigned)((sn + 255) / 256), 256, 0, st>>>(a, c.ws_lse);
-    AA_TRY(cudaGetLastError());
-    a.lse = c.ws_lse; a.outer0 = c.ws_va;
-    AA_TRY((launch_tile<T, kVa1>(a, st)));
+    if (c.use_mma) {
+        BwdArgs m = a;
+        m.np = c.plan_mma.np; m.tile = c.plan_mma.tile; m.tiles = c.plan_mma.tiles;
+        m.chunks = c.plan_mma.chunks; m.tiles_per_chunk = c.plan_mma.tiles_per_chunk;
+        AA_TRY(launch_backward_fwd1_mma(c.dtype, m, c.ws_va, c.ws_lse, st));
+        a.lse = c.ws_lse;
+    } else {
+        AA_TRY((launch_tile<T, kStats1>(a, st)));
+        bwd_lse_kernel<<<(unsigned)((sn + 255) / 256), 256, 0, st>>>(a, c.ws_lse);
+        AA_TRY(cudaGetLastError());
+        a.lse = c.ws_lse; a.outer0 = c.ws_va;
+        AA_TRY((launch_tile<T, kVa1>(a, st)));
+    }
     // broadcast backward
     a.x = c.q; a.y = c.d_out; a.bias = c.b2; a.m0 = c.ws_a; a.m1 = c.ws_va; a.scale = c.scale2;
     a.outer0 = c.ws_dva; a.outer1 = c.ws_da; a.row0 = c.dq; a.row1 = nullptr; a.dbias = c.db2;
@@ -579,7 +587,7 @@ bool plan_backward(int slabs, int n, int N, int d, int sm_count, BwdPlan* out) {
     return true;
 }
 
-int backward_launch_count(bool with_dwd) { return 9 + (with_dwd ? 1 : 0); }
+int backward_launch_count(bool with_dwd, bool use_mma) { return (use_mma ? 8 : 9) + (with_dwd ? 1 : 0); }
 
 cudaError_t launch_backward(int dtype, const BwdCall& c, cudaStream_t st) {
     BwdArgs a;

@@ -281,6 +281,160 @@ __global__ void __launch_bounds__(kThreads, 3) bwd_mma_kernel(BwdArgs p) {
     }
 }
 
+// Floats per agent row of a stage-1 partial: running max (log2 domain), running sum, 64 accumulators.
+constexpr int kPartRow = 2 + kD;
+
+// Aggregation stage recomputed (flash-attention style, agents as rows): per block, the running max and sum of
+// the logits of each agent over the block's tokens and the unnormalised sum of exp(S - max) V.  Warp w owns
+// agents 16w..16w+15; P enters the product with V as two 16-bit terms, so that V_A keeps fp32-level accuracy
+// (its small differences between agents are what the broadcast stage's gradient is made of).
+template <typename T>
+__global__ void __launch_bounds__(kThreads, 3) bwd_fwd1_mma_kernel(BwdArgs p) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    T* sA = reinterpret_cast<T*>(smem_raw);      // [agent][c]
+    T* sX = sA + kMat;                           // [token][c]  K
+    T* sY = sX + kMat;                           // [token][c]  V
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int g = lane >> 2, t4 = lane & 3;
+    const int slab = blockIdx.x / p.chunks, chunk = blockIdx.x - slab * p.chunks;
+    const int head = slab % p.heads;
+    const int n = p.n, N = p.N;
+    for (int i = tid; i < kNP * kD; i += kThreads) {
+        const int r = i >> 6, c = i & 63;
+        sA[r * kPA + c] = Elem<T>::from_f32(r < n ? p.m0[((size_t)slab * n + r) * kD + c] : 0.f);
+    }
+    __syncthreads();
+    const int r0 = warp * 16;
+    uint32_t af[4][4];
+#pragma unroll
+    for (int ks = 0; ks < 4; ++ks)
+        ldmatrix_x4(af[ks][0], af[ks][1], af[ks][2], af[ks][3],
+                    sA + (r0 + (lane & 7) + ((lane >> 3) & 1) * 8) * kPA + ks * 16 + (lane >> 4) * 8);
+    const int ag_a = r0 + g, ag_b = ag_a + 8;
+    float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+    float acc[8][4];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[j][0] = acc[j][1] = acc[j][2] = acc[j][3] = 0.f;
+
+    const T* xg = static_cast<const T*>(p.x) + (size_t)slab * N * kD;
+    const T* yg = static_cast<const T*>(p.y) + (size_t)slab * N * kD;
+    const T* bias = static_cast<const T*>(p.bias);
+    const float scale_log2 = p.scale * kLog2e;
+    const int tile_end = min((chunk + 1) * p.tiles_per_chunk, p.tiles);
+    for (int tile = chunk * p.tiles_per_chunk; tile < tile_end; ++tile) {
+        const int tok0 = tile * kTT;
+        __syncthreads();
+        for (int e = tid; e < kTT * (kD / 8); e += kThreads) {
+            const int r = e >> 3, ch = e & 7;
+            const bool ok = tok0 + r < N;
+            const size_t off = ok ? ((size_t)(tok0 + r) * kD + ch * 8) : 0;
+            cp_async16(sX + r * kPA + ch * 8, xg + off, ok ? 16 : 0);
+            cp_async16(sY + r * kPA + ch * 8, yg + off, ok ? 16 : 0);
+        }
+        cp_async_commit();
+        cp_async_wait<0>();
+        __syncthreads();
+        float sc[8][4];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) sc[j][0] = sc[j][1] = sc[j][2] = sc[j][3] = 0.f;
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks)
+#pragma unroll
+            for (int np = 0; np < 4; ++np) {
+                uint32_t b0, b1, b2, b3;
+                ldmatrix_x4(b0, b1, b2, b3,
+                            sX + (np * 16 + (lane & 7) + (lane >> 4) * 8) * kPA + ks * 16 + ((lane >> 3) & 1) * 8);
+                mma16816<T>(sc[2 * np], af[ks], b0, b1);
+                mma16816<T>(sc[2 * np + 1], af[ks], b2, b3);
+            }
+        float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int tok = tok0 + 8 * j + 2 * t4 + (e & 1);
+                const int ag = (e & 2) ? ag_b : ag_a;
+                const bool ok = ag < n && tok < N;
+                float b = 0.f;
+                if (bias && ok) b = Elem<T>::to_f32(bias[((size_t)head * n + ag) * N + tok]);
+                sc[j][e] = ok ? fmaf(sc[j][e], scale_log2, b * kLog2e) : -INFINITY;
+                if (e & 2) mx1 = fmaxf(mx1, sc[j][e]); else mx0 = fmaxf(mx0, sc[j][e]);
+            }
+        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+        const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
+        const bool live0 = mn0 > -INFINITY, live1 = mn1 > -INFINITY;     // rows past n never come alive
+        const float c0 = live0 ? fast_exp2(m0 - mn0) : 1.f, c1 = live1 ? fast_exp2(m1 - mn1) : 1.f;
+        m0 = mn0; m1 = mn1;
+        l0 *= c0; l1 *= c1;
+        uint32_t hi[8][2], lo[8][2];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            acc[j][0] *= c0; acc[j][1] *= c0; acc[j][2] *= c1; acc[j][3] *= c1;
+            const float p0 = live0 ? fast_exp2(sc[j][0] - mn0) : 0.f, p1 = live0 ? fast_exp2(sc[j][1] - mn0) : 0.f;
+            const float p2 = live1 ? fast_exp2(sc[j][2] - mn1) : 0.f, p3 = live1 ? fast_exp2(sc[j][3] - mn1) : 0.f;
+            l0 += p0 + p1;
+            l1 += p2 + p3;
+            hi[j][0] = pack2<T>(p0, p1);
+            hi[j][1] = pack2<T>(p2, p3);
+            const float2 h0 = unpack2<T>(hi[j][0]), h1 = unpack2<T>(hi[j][1]);
+            lo[j][0] = pack2<T>(p0 - h0.x, p1 - h0.y);
+            lo[j][1] = pack2<T>(p2 - h1.x, p3 - h1.y);
+        }
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {
+            const uint32_t ah[4] = {hi[2 * kk][0], hi[2 * kk][1], hi[2 * kk + 1][0], hi[2 * kk + 1][1]};
+            const uint32_t al[4] = {lo[2 * kk][0], lo[2 * kk][1], lo[2 * kk + 1][0], lo[2 * kk + 1][1]};
+#pragma unroll
+            for (int np = 0; np < 4; ++np) {
+                uint32_t b0, b1, b2, b3;
+                ldmatrix_x4_trans(b0, b1, b2, b3,
+                                  sY + (kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * kPA + np * 16 + (lane >> 4) * 8);
+                mma16816<T>(acc[2 * np], ah, b0, b1);
+                mma16816<T>(acc[2 * np + 1], ah, b2, b3);
+                mma16816<T>(acc[2 * np], al, b0, b1);
+                mma16816<T>(acc[2 * np + 1], al, b2, b3);
+            }
+        }
+    }
+    l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
+    l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+    l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
+    l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+    float* pa = p.part + (((size_t)slab * p.chunks + chunk) * kNP + ag_a) * kPartRow;
+    float* pb = p.part + (((size_t)slab * p.chunks + chunk) * kNP + ag_b) * kPartRow;
+    if (t4 == 0) { pa[0] = m0; pa[1] = l0; pb[0] = m1; pb[1] = l1; }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const int col = 2 + 8 * j + 2 * t4;
+        *reinterpret_cast<float2*>(pa + col) = make_float2(acc[j][0], acc[j][1]);
+        *reinterpret_cast<float2*>(pb + col) = make_float2(acc[j][2], acc[j][3]);
+    }
+}
+
+// Merge of the stage-1 partials in chunk order: V_A (fp32) and the natural-log sum-exp of each agent's logits.
+__global__ void bwd_fwd1_merge_kernel(BwdArgs p, float* va, float* lse) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;       // (slab * n + r) * 64 + c
+    if (i >= (size_t)p.slabs * p.n * kD) return;
+    const int c = (int)(i & 63);
+    const size_t sr = i >> 6;
+    const int r = (int)(sr % p.n), slab = (int)(sr / p.n);
+    const float* base = p.part + ((size_t)slab * p.chunks * kNP + r) * kPartRow;
+    const size_t stride = (size_t)kNP * kPartRow;
+    float M = -INFINITY;
+    for (int ch = 0; ch < p.chunks; ++ch) M = fmaxf(M, base[ch * stride]);
+    float L = 0.f, v = 0.f;
+    for (int ch = 0; ch < p.chunks; ++ch) {
+        const float w = exp2f(base[ch * stride] - M);
+        L = fmaf(base[ch * stride + 1], w, L);
+        v = fmaf(base[ch * stride + 2 + c], w, v);
+    }
+    va[i] = v / L;
+    if (c == 0) lse[sr] = (M + log2f(L)) * 0.6931471805599453f;
+}
+
 constexpr size_t kSmemBytes = 7 * (size_t)kMat * 2 + 2 * kNP * sizeof(float);
 
 template <typename T, bool BCAST>
@@ -293,6 +447,28 @@ cudaError_t launch(const BwdArgs& a, cudaStream_t st) {
 }
 
 }  // namespace
+
+size_t backward_mma_part_floats(int slabs, const BwdPlan& pl) { return (size_t)slabs * pl.chunks * kNP * kPartRow; }
+
+cudaError_t launch_backward_fwd1_mma(int dtype, const BwdArgs& a, float* va, float* lse, cudaStream_t st) {
+    const size_t smem = 3 * (size_t)kMat * 2;
+    if (dtype == kBF16) {
+        cudaError_t e = cudaFuncSetAttribute(bwd_fwd1_mma_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        bwd_fwd1_mma_kernel<__nv_bfloat16><<<a.slabs * a.chunks, kThreads, smem, st>>>(a);
+    } else if (dtype == kF16) {
+        cudaError_t e = cudaFuncSetAttribute(bwd_fwd1_mma_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        bwd_fwd1_mma_kernel<__half><<<a.slabs * a.chunks, kThreads, smem, st>>>(a);
+    } else {
+        return cudaErrorInvalidValue;
+    }
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    const size_t total = (size_t)a.slabs * a.n * kD;
+    bwd_fwd1_merge_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(a, va, lse);
+    return cudaGetLastError();
+}
 
 bool backward_mma_eligible(int dtype, int n, int d) { return (dtype == kBF16 || dtype == kF16) && n <= kNP && d == kD; }
 

@@ -179,11 +179,14 @@ struct BwdCall {
     BwdPlan plan_mma;                         // their tiling
 };
 bool plan_backward(int slabs, int n, int N, int d, int sm_count, BwdPlan* out);   // false: shape not supported
-int backward_launch_count(bool with_dwd);
+int backward_launch_count(bool with_dwd, bool use_mma);
 cudaError_t launch_backward(int dtype, const BwdCall& c, cudaStream_t st);
 // Tensor-core kernels of the two gradient stages (16-bit inputs, n <= 64, d = 64)
 bool backward_mma_eligible(int dtype, int n, int d);
 BwdPlan plan_backward_mma(int slabs, int N, int sm_count);
 cudaError_t launch_backward_mma(int dtype, bool broadcast_stage, const BwdArgs& a, cudaStream_t st);
+// aggregation stage recomputed: per-block partials into a.part, then V_A and the log-sum-exp per agent
+cudaError_t launch_backward_fwd1_mma(int dtype, const BwdArgs& a, float* va, float* lse, cudaStream_t st);
+size_t backward_mma_part_floats(int slabs, const BwdPlan& pl);
 
 }  // namespace aa
