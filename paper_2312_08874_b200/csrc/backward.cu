@@ -376,18 +376,25 @@ template <> __device__ __forceinline__ float4 ld4_f32<__half>(const __half* p) {
 
 // Token-wise tail: dQ += Pooling^T(dA) (each window spreads its agent's gradient evenly over its
 // tokens) and dV += DWC^T(dO) (tap (u, v) of output token (y, x) read V[y+u-1][x+v-1]).
-// One thread per (slab, token, 4 channels).
+// blockIdx.y = slab; one thread per (token, 4 channels); the head's filter sits in shared memory as [tap][c].
 template <typename T>
 __global__ void __launch_bounds__(256) bwd_tail_kernel(BwdArgs p, const float* da, const void* gov, const void* wdv,
                                                        float* dq, float* dv) {
+    __shared__ __align__(16) float sw[9 * 128];
+    const int slab = blockIdx.y, head = slab % p.heads;
+    if (wdv) {
+        const T* w = static_cast<const T*>(wdv) + (size_t)head * p.d * 9;
+        for (int i = threadIdx.x; i < p.d * 9; i += 256) {
+            const int c = i / 9, k = i - c * 9;
+            sw[k * p.d + c] = ld_f32(w, i);
+        }
+        __syncthreads();
+    }
     const int d4 = p.d >> 2;
-    const size_t total = (size_t)p.slabs * p.N * d4;
-    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= total) return;
-    const int c = (int)(i % d4) * 4;
-    const size_t st = i / d4;                                    // slab * N + token
-    const int tok = (int)(st % p.N);
-    const int slab = (int)(st / p.N);
+    const int i = blockIdx.x * 256 + threadIdx.x;                 // token * d4 + channel group
+    if (i >= p.N * d4) return;
+    const int tok = i / d4, c = (i - tok * d4) * 4;
+    const size_t st = (size_t)slab * p.N + tok;
     const int y = tok / p.W, x = tok - y * p.W;
     const int ayc = (y * p.ph) / p.H, axc = (x * p.pw) / p.W;
     float4 g = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -407,10 +414,9 @@ __global__ void __launch_bounds__(256) bwd_tail_kernel(BwdArgs p, const float* d
     qv.x += g.x; qv.y += g.y; qv.z += g.z; qv.w += g.w;
     *qo = qv;
     if (wdv) {
-        const int head = slab % p.heads;
-        const T* w = static_cast<const T*>(wdv) + ((size_t)head * p.d + c) * 9;     // [4 channels][9 taps]
         const T* go = static_cast<const T*>(gov) + (size_t)slab * p.N * p.d;
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        float4* vo = reinterpret_cast<float4*>(dv + st * p.d + c);
+        float4 acc = *vo;
 #pragma unroll
         for (int u = 0; u < 3; ++u)
 #pragma unroll
@@ -418,55 +424,60 @@ __global__ void __launch_bounds__(256) bwd_tail_kernel(BwdArgs p, const float* d
                 const int yo = y - u + 1, xo = x - v + 1;          // the output token whose tap (u, v) is (y, x)
                 if (yo < 0 || yo >= p.H || xo < 0 || xo >= p.W) continue;
                 const float4 gv = ld4_f32<T>(go + ((size_t)yo * p.W + xo) * p.d + c);
-                const int k = u * 3 + v;
-                acc.x = fmaf(ld_f32(w, k), gv.x, acc.x);      acc.y = fmaf(ld_f32(w, 9 + k), gv.y, acc.y);
-                acc.z = fmaf(ld_f32(w, 18 + k), gv.z, acc.z); acc.w = fmaf(ld_f32(w, 27 + k), gv.w, acc.w);
+                const float4 wv = *reinterpret_cast<const float4*>(sw + (u * 3 + v) * p.d + c);
+                acc.x = fmaf(wv.x, gv.x, acc.x); acc.y = fmaf(wv.y, gv.y, acc.y);
+                acc.z = fmaf(wv.z, gv.z, acc.z); acc.w = fmaf(wv.w, gv.w, acc.w);
             }
-        float4* vo = reinterpret_cast<float4*>(dv + st * p.d + c);
-        float4 vv = *vo;
-        vv.x += acc.x; vv.y += acc.y; vv.z += acc.z; vv.w += acc.w;
-        *vo = vv;
+        *vo = acc;
     }
 }
 
 // dWd[head][c][u][v] = sum over batch and output tokens of dO[y][x][c] * V[y+u-1][x+v-1][c].
-// Block = (slab, token chunk); thread = (token lane, channel); per-block sums are added with atomics.
+// Block = (slab, token chunk); thread = (token lane, 4 channels); per-block sums are added with atomics.
 template <typename T>
-__global__ void __launch_bounds__(512) bwd_dwd_kernel(BwdArgs p, const void* gov, const void* vv, float* dwd, int chunks) {
-    __shared__ float red[512 * 9];
+__global__ void __launch_bounds__(256) bwd_dwd_kernel(BwdArgs p, const void* gov, const void* vv, float* dwd, int chunks) {
+    __shared__ float4 red[256 * 9];
     const int slab = blockIdx.x / chunks, chunk = blockIdx.x - slab * chunks;
     const int head = slab % p.heads;
-    const int lanes = 512 / p.d;                                  // token lanes (d <= 128: at least 4)
-    const int c = threadIdx.x % p.d, tlane = threadIdx.x / p.d;
+    const int d4 = p.d >> 2;
+    const int lanes = 256 / d4;                                   // token lanes (d <= 128: at least 8)
+    const int c4 = threadIdx.x % d4, tlane = threadIdx.x / d4;
     const int per = (p.N + chunks - 1) / chunks;
     const int t0 = chunk * per, t1 = min(t0 + per, p.N);
-    const T* go = static_cast<const T*>(gov) + (size_t)slab * p.N * p.d;
-    const T* v = static_cast<const T*>(vv) + (size_t)slab * p.N * p.d;
-    float acc[9];
+    const T* go = static_cast<const T*>(gov) + (size_t)slab * p.N * p.d + 4 * c4;
+    const T* v = static_cast<const T*>(vv) + (size_t)slab * p.N * p.d + 4 * c4;
+    float4 acc[9];
 #pragma unroll
-    for (int k = 0; k < 9; ++k) acc[k] = 0.f;
+    for (int k = 0; k < 9; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
     if (tlane < lanes)
         for (int tok = t0 + tlane; tok < t1; tok += lanes) {
             const int y = tok / p.W, x = tok - y * p.W;
-            const float g = ld_f32(go, (size_t)tok * p.d + c);
+            const float4 g = ld4_f32<T>(go + (size_t)tok * p.d);
 #pragma unroll
             for (int u = 0; u < 3; ++u)
 #pragma unroll
                 for (int w = 0; w < 3; ++w) {
                     const int yy = y + u - 1, xx = x + w - 1;
-                    if (yy >= 0 && yy < p.H && xx >= 0 && xx < p.W)
-                        acc[u * 3 + w] = fmaf(g, ld_f32(v, ((size_t)yy * p.W + xx) * p.d + c), acc[u * 3 + w]);
+                    if (yy >= 0 && yy < p.H && xx >= 0 && xx < p.W) {
+                        const float4 t = ld4_f32<T>(v + ((size_t)yy * p.W + xx) * p.d);
+                        float4& a = acc[u * 3 + w];
+                        a.x = fmaf(g.x, t.x, a.x); a.y = fmaf(g.y, t.y, a.y);
+                        a.z = fmaf(g.z, t.z, a.z); a.w = fmaf(g.w, t.w, a.w);
+                    }
                 }
         }
 #pragma unroll
     for (int k = 0; k < 9; ++k) red[threadIdx.x * 9 + k] = acc[k];
     __syncthreads();
-    if (threadIdx.x < p.d) {
-        for (int k = 0; k < 9; ++k) {
-            float s = 0.f;
-            for (int l = 0; l < lanes; ++l) s += red[(l * p.d + threadIdx.x) * 9 + k];
-            atomicAdd(dwd + ((size_t)head * p.d + threadIdx.x) * 9 + k, s);
+    for (int o = threadIdx.x; o < p.d * 9; o += 256) {           // o = c * 9 + tap, the layout of dWd
+        const int c = o / 9, k = o - c * 9;
+        const int q4 = c >> 2, e = c & 3;
+        float s = 0.f;
+        for (int l = 0; l < lanes; ++l) {
+            const float4 t = red[(l * d4 + q4) * 9 + k];
+            s += e == 0 ? t.x : e == 1 ? t.y : e == 2 ? t.z : t.w;
         }
+        atomicAdd(dwd + (size_t)head * p.d * 9 + o, s);
     }
 }
 
@@ -495,7 +506,6 @@ cudaError_t launch_tile(const BwdArgs& a, cudaStream_t st) {
 template <typename T>
 cudaError_t backward_typed(const BwdCall& c, BwdArgs a, cudaStream_t st) {
     const size_t sn = (size_t)a.slabs * a.n, snd = sn * a.d;
-    const size_t tok_elems = (size_t)a.slabs * a.N * a.d;
     cudaError_t e;
 #define AA_TRY(x) do { e = (x); if (e != cudaSuccess) return e; } while (0)
     AA_TRY(cudaMemsetAsync(c.ws_va, 0, c.clear_bytes, st));               // V_A, dV_A, dA are contiguous
@@ -548,12 +558,15 @@ cudaError_t backward_typed(const BwdCall& c, BwdArgs a, cudaStream_t st) {
         AA_TRY((launch_tile<T, kAgg1>(a, st)));
     }
     // pooling and depthwise terms
-    bwd_tail_kernel<T><<<(unsigned)((tok_elems / 4 + 255) / 256), 256, 0, st>>>(a, c.ws_da, c.d_out, c.wd, c.dq, c.dv);
-    AA_TRY(cudaGetLastError());
+    {
+        const dim3 grid((unsigned)(((size_t)a.N * (a.d / 4) + 255) / 256), (unsigned)a.slabs);
+        bwd_tail_kernel<T><<<grid, 256, 0, st>>>(a, c.ws_da, c.d_out, c.wd, c.dq, c.dv);
+        AA_TRY(cudaGetLastError());
+    }
     if (c.dwd) {
         int chunks = (4 * c.sm_count + a.slabs - 1) / a.slabs;          // short loops (they are load-latency bound), few atomics
         chunks = max(1, min(chunks, (a.N + 63) / 64));
-        bwd_dwd_kernel<T><<<a.slabs * chunks, 512, 0, st>>>(a, c.d_out, c.v, c.dwd, chunks);
+        bwd_dwd_kernel<T><<<a.slabs * chunks, 256, 0, st>>>(a, c.d_out, c.v, c.dwd, chunks);
         AA_TRY(cudaGetLastError());
     }
 #undef AA_TRY
@@ -570,6 +583,7 @@ static size_t bwd_smem_bytes(int n, int d, int tile) {
 
 bool plan_backward(int slabs, int n, int N, int d, int sm_count, BwdPlan* out) {
     if (n > 32 * kMaxLaneAgents || (size_t)n * d > (size_t)4 * kMaxOuter * kBwdThreads || d % 4) return false;
+    if (slabs > 65535 || d > 128) return false;                 // the token-wise tail indexes slabs with gridDim.y
     int tile = 32;
     while (tile >= 8 && bwd_smem_bytes(n, d, tile) > 227u * 1024u) tile >>= 1;
     if (tile < 8) return false;
