@@ -511,11 +511,11 @@ int agent_attn_query_status(agent_attn_handle* h, void* stream) {
     return AA_OK;
 }
 
-// Workspace of the backward pass: [A | V_A | dV_A | dA | lse | dot | partial (max, sum)], fp32, each
+// Workspace of the backward pass: [A | V_A | dV_A | dA | lse | dot | window table | partial (max, sum)], fp32, each
 // region 256-byte aligned (V_A, dV_A and dA are cleared with one memset, so their regions have one size).
 namespace {
 struct BwdLayout {
-    size_t a, va, dva, da, lse, dot, part, total;
+    size_t a, va, dva, da, lse, dot, tab, part, total;
 };
 bool bwd_layout(const agent_attn_handle* h, int N, int n, BwdPlan* pl, BwdLayout* w) {
     const int slabs = h->cfg.batch * h->cfg.heads;
@@ -523,7 +523,8 @@ bool bwd_layout(const agent_attn_handle* h, int N, int n, BwdPlan* pl, BwdLayout
     const size_t snd = align_up((size_t)slabs * n * h->cfg.head_dim * sizeof(float), 256);
     const size_t sn = align_up((size_t)slabs * n * sizeof(float), 256);
     w->a = 0; w->va = snd; w->dva = 2 * snd; w->da = 3 * snd;
-    w->lse = 4 * snd; w->dot = w->lse + sn; w->part = w->dot + sn;
+    w->lse = 4 * snd; w->dot = w->lse + sn; w->tab = w->dot + sn;
+    w->part = w->tab + align_up((size_t)N * 48, 256);
     size_t part_floats = (size_t)slabs * pl->chunks * n * 2;
     if (backward_mma_eligible(h->cfg.dtype, n, h->cfg.head_dim)) {      // partials of the tensor-core stage 1
         const size_t mma_floats = backward_mma_part_floats(slabs, plan_backward_mma(slabs, N, h->sm_count));
@@ -592,6 +593,7 @@ int agent_attn_backward(agent_attn_handle* h, const void* Q, const void* K, cons
     c.ws_dva = reinterpret_cast<float*>(ws + w.dva); c.ws_da = reinterpret_cast<float*>(ws + w.da);
     c.ws_lse = reinterpret_cast<float*>(ws + w.lse); c.ws_dot = reinterpret_cast<float*>(ws + w.dot);
     c.ws_part = reinterpret_cast<float*>(ws + w.part);
+    c.ws_tab = reinterpret_cast<int4*>(ws + w.tab);
     c.clear_bytes = w.lse - w.va;
     c.slabs = h->cfg.batch * h->cfg.heads; c.heads = h->cfg.heads; c.H = grid_h; c.W = grid_w;
     c.d = h->cfg.head_dim; c.n = n_agents; c.p = p; c.sm_count = h->sm_count;
@@ -601,7 +603,7 @@ int agent_attn_backward(agent_attn_handle* h, const void* Q, const void* K, cons
     if (c.use_mma) c.plan_mma = plan_backward_mma(c.slabs, N, h->sm_count);
     cudaError_t e = launch_backward(h->cfg.dtype, c, (cudaStream_t)stream);
     if (e != cudaSuccess) return fail(h, AA_ERR_CUDA, "backward launch failed: %s", cudaGetErrorString(e));
-    h->launches = backward_launch_count(c.dwd != nullptr, c.use_mma != 0);
+    h->launches = backward_launch_count(c.use_mma != 0);
     return AA_OK;
 }
 

@@ -374,104 +374,115 @@ template <> __device__ __forceinline__ float4 ld4_f32<__half>(const __half* p) {
     return make_float4(a.x, a.y, b.x, b.y);
 }
 
-// Token-wise tail: dQ += Pooling^T(dA) (each window spreads its agent's gradient evenly over its
-// tokens) and dV += DWC^T(dO) (tap (u, v) of output token (y, x) read V[y+u-1][x+v-1]).
-// blockIdx.y = slab; one thread per (token, 4 channels); the head's filter sits in shared memory as [tap][c].
-template <typename T>
-__global__ void __launch_bounds__(256) bwd_tail_kernel(BwdArgs p, const float* da, const void* gov, const void* wdv,
-                                                       float* dq, float* dv) {
-    __shared__ __align__(16) float sw[9 * 128];
-    const int slab = blockIdx.y, head = slab % p.heads;
-    if (wdv) {
-        const T* w = static_cast<const T*>(wdv) + (size_t)head * p.d * 9;
-        for (int i = threadIdx.x; i < p.d * 9; i += 256) {
-            const int c = i / 9, k = i - c * 9;
-            sw[k * p.d + c] = ld_f32(w, i);
-        }
-        __syncthreads();
-    }
-    const int d4 = p.d >> 2;
-    const int i = blockIdx.x * 256 + threadIdx.x;                 // token * d4 + channel group
-    if (i >= p.N * d4) return;
-    const int tok = i / d4, c = (i - tok * d4) * 4;
-    const size_t st = (size_t)slab * p.N + tok;
+// Per token of the grid (the same for every slab): the pooled cells whose window contains it (at most two per
+// axis; bounds as in bwd_pool_kernel), the reciprocal of each window's size, and the token's grid position.
+// Three int4 per token: (count, agent0, agent1, agent2), (agent3, inv0, inv1, inv2), (inv3, y, x, -).
+__global__ void bwd_window_table_kernel(BwdArgs p, int4* tab) {
+    const int tok = blockIdx.x * blockDim.x + threadIdx.x;
+    if (tok >= p.N) return;
     const int y = tok / p.W, x = tok - y * p.W;
+    int ays[2], hy[2], axs[2], wx[2], ny = 0, nx = 0;
     const int ayc = (y * p.ph) / p.H, axc = (x * p.pw) / p.W;
-    float4 g = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int ay = max(ayc - 1, 0); ay <= min(ayc + 1, p.ph - 1); ++ay) {
+    for (int ay = ayc; ay <= min(ayc + 1, p.ph - 1); ++ay) {
         const int y0 = (ay * p.H) / p.ph, y1 = ((ay + 1) * p.H + p.ph - 1) / p.ph;
-        if (y < y0 || y >= y1) continue;
-        for (int ax = max(axc - 1, 0); ax <= min(axc + 1, p.pw - 1); ++ax) {
-            const int x0 = (ax * p.W) / p.pw, x1 = ((ax + 1) * p.W + p.pw - 1) / p.pw;
-            if (x < x0 || x >= x1) continue;
-            const float cnt = (float)((y1 - y0) * (x1 - x0));
-            const float4 a = *reinterpret_cast<const float4*>(da + ((size_t)slab * p.n + ay * p.pw + ax) * p.d + c);
-            g.x += a.x / cnt; g.y += a.y / cnt; g.z += a.z / cnt; g.w += a.w / cnt;
+        if (y >= y0 && y < y1) { ays[ny] = ay; hy[ny] = y1 - y0; ++ny; }
+    }
+    for (int ax = axc; ax <= min(axc + 1, p.pw - 1); ++ax) {
+        const int x0 = (ax * p.W) / p.pw, x1 = ((ax + 1) * p.W + p.pw - 1) / p.pw;
+        if (x >= x0 && x < x1) { axs[nx] = ax; wx[nx] = x1 - x0; ++nx; }
+    }
+    int agent[4] = {0, 0, 0, 0};
+    float inv[4] = {0.f, 0.f, 0.f, 0.f};
+    int cnt = 0;
+    for (int a = 0; a < ny; ++a)
+        for (int b = 0; b < nx; ++b) {
+            agent[cnt] = ays[a] * p.pw + axs[b];
+            inv[cnt] = 1.f / (float)(hy[a] * wx[b]);
+            ++cnt;
         }
-    }
-    float4* qo = reinterpret_cast<float4*>(dq + st * p.d + c);
-    float4 qv = *qo;
-    qv.x += g.x; qv.y += g.y; qv.z += g.z; qv.w += g.w;
-    *qo = qv;
-    if (wdv) {
-        const T* go = static_cast<const T*>(gov) + (size_t)slab * p.N * p.d;
-        float4* vo = reinterpret_cast<float4*>(dv + st * p.d + c);
-        float4 acc = *vo;
-#pragma unroll
-        for (int u = 0; u < 3; ++u)
-#pragma unroll
-            for (int v = 0; v < 3; ++v) {
-                const int yo = y - u + 1, xo = x - v + 1;          // the output token whose tap (u, v) is (y, x)
-                if (yo < 0 || yo >= p.H || xo < 0 || xo >= p.W) continue;
-                const float4 gv = ld4_f32<T>(go + ((size_t)yo * p.W + xo) * p.d + c);
-                const float4 wv = *reinterpret_cast<const float4*>(sw + (u * 3 + v) * p.d + c);
-                acc.x = fmaf(wv.x, gv.x, acc.x); acc.y = fmaf(wv.y, gv.y, acc.y);
-                acc.z = fmaf(wv.z, gv.z, acc.z); acc.w = fmaf(wv.w, gv.w, acc.w);
-            }
-        *vo = acc;
-    }
+    tab[3 * tok] = make_int4(cnt, agent[0], agent[1], agent[2]);
+    tab[3 * tok + 1] = make_int4(agent[3], __float_as_int(inv[0]), __float_as_int(inv[1]), __float_as_int(inv[2]));
+    tab[3 * tok + 2] = make_int4(__float_as_int(inv[3]), y, x, 0);
 }
 
-// dWd[head][c][u][v] = sum over batch and output tokens of dO[y][x][c] * V[y+u-1][x+v-1][c].
-// Block = (slab, token chunk); thread = (token lane, 4 channels); per-block sums are added with atomics.
+// Token-wise tail, one pass over the tokens:
+//   dQ  += Pooling^T(dA)   each window spreads its agent's gradient evenly over its tokens
+//   dV  += DWC^T(dO)       tap (u, v) of output token (y - u + 1, x - v + 1) read V[y][x]
+//   dWd += corr(dO, V)     dWd[c][u][v] = sum over tokens of dO[y - u + 1][x - v + 1][c] * V[y][x][c]
+// (the last two use the same nine neighbours of dO).  Block = (slab, token chunk); thread = (token lane,
+// 4 channels); the filter gradient is summed per thread, reduced per block and added with atomics.
 template <typename T>
-__global__ void __launch_bounds__(256) bwd_dwd_kernel(BwdArgs p, const void* gov, const void* vv, float* dwd, int chunks) {
+__global__ void __launch_bounds__(256) bwd_tail_kernel(BwdArgs p, const int4* tab, const float* da, const void* gov,
+                                                       const void* vv, const void* wdv, float* dq, float* dv,
+                                                       float* dwd, int chunks) {
+    __shared__ __align__(16) float sw[9 * 128];
     __shared__ float4 red[256 * 9];
     const int slab = blockIdx.x / chunks, chunk = blockIdx.x - slab * chunks;
     const int head = slab % p.heads;
     const int d4 = p.d >> 2;
     const int lanes = 256 / d4;                                   // token lanes (d <= 128: at least 8)
-    const int c4 = threadIdx.x % d4, tlane = threadIdx.x / d4;
+    const int c4 = threadIdx.x % d4, tlane = threadIdx.x / d4, c = 4 * c4;
     const int per = (p.N + chunks - 1) / chunks;
     const int t0 = chunk * per, t1 = min(t0 + per, p.N);
-    const T* go = static_cast<const T*>(gov) + (size_t)slab * p.N * p.d + 4 * c4;
-    const T* v = static_cast<const T*>(vv) + (size_t)slab * p.N * p.d + 4 * c4;
-    float4 acc[9];
+    if (wdv) {
+        const T* w = static_cast<const T*>(wdv) + (size_t)head * p.d * 9;
+        for (int i = threadIdx.x; i < p.d * 9; i += 256) {
+            const int cc = i / 9, k = i - cc * 9;
+            sw[k * p.d + cc] = ld_f32(w, i);
+        }
+        __syncthreads();
+    }
+    const T* go = static_cast<const T*>(gov) + (size_t)slab * p.N * p.d + c;
+    const T* v = static_cast<const T*>(vv) + (size_t)slab * p.N * p.d + c;
+    float4 accw[9];
 #pragma unroll
-    for (int k = 0; k < 9; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int k = 0; k < 9; ++k) accw[k] = make_float4(0.f, 0.f, 0.f, 0.f);
     if (tlane < lanes)
         for (int tok = t0 + tlane; tok < t1; tok += lanes) {
-            const int y = tok / p.W, x = tok - y * p.W;
-            const float4 g = ld4_f32<T>(go + (size_t)tok * p.d);
+            const int4 e0 = tab[3 * tok], e1 = tab[3 * tok + 1], e2 = tab[3 * tok + 2];
+            const int agent[4] = {e0.y, e0.z, e0.w, e1.x};
+            const float inv[4] = {__int_as_float(e1.y), __int_as_float(e1.z), __int_as_float(e1.w), __int_as_float(e2.x)};
+            const size_t st = (size_t)slab * p.N + tok;
+            float4* qo = reinterpret_cast<float4*>(dq + st * p.d + c);
+            float4 qv = *qo;
 #pragma unroll
-            for (int u = 0; u < 3; ++u)
-#pragma unroll
-                for (int w = 0; w < 3; ++w) {
-                    const int yy = y + u - 1, xx = x + w - 1;
-                    if (yy >= 0 && yy < p.H && xx >= 0 && xx < p.W) {
-                        const float4 t = ld4_f32<T>(v + ((size_t)yy * p.W + xx) * p.d);
-                        float4& a = acc[u * 3 + w];
-                        a.x = fmaf(g.x, t.x, a.x); a.y = fmaf(g.y, t.y, a.y);
-                        a.z = fmaf(g.z, t.z, a.z); a.w = fmaf(g.w, t.w, a.w);
-                    }
+            for (int k = 0; k < 4; ++k)
+                if (k < e0.x) {
+                    const float4 a = *reinterpret_cast<const float4*>(da + ((size_t)slab * p.n + agent[k]) * p.d + c);
+                    qv.x = fmaf(a.x, inv[k], qv.x); qv.y = fmaf(a.y, inv[k], qv.y);
+                    qv.z = fmaf(a.z, inv[k], qv.z); qv.w = fmaf(a.w, inv[k], qv.w);
                 }
-        }
+            *qo = qv;
+            if (wdv) {
+                const int y = e2.y, x = e2.z;
+                float4* vo = reinterpret_cast<float4*>(dv + st * p.d + c);
+                float4 acc = *vo;
+                float4 vt = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (dwd) vt = ld4_f32<T>(v + (size_t)tok * p.d);
 #pragma unroll
-    for (int k = 0; k < 9; ++k) red[threadIdx.x * 9 + k] = acc[k];
+                for (int u = 0; u < 3; ++u)
+#pragma unroll
+                    for (int w = 0; w < 3; ++w) {
+                        const int yo = y - u + 1, xo = x - w + 1;
+                        if (yo < 0 || yo >= p.H || xo < 0 || xo >= p.W) continue;
+                        const float4 gv = ld4_f32<T>(go + ((size_t)yo * p.W + xo) * p.d);
+                        const float4 wv = *reinterpret_cast<const float4*>(sw + (u * 3 + w) * p.d + c);
+                        acc.x = fmaf(wv.x, gv.x, acc.x); acc.y = fmaf(wv.y, gv.y, acc.y);
+                        acc.z = fmaf(wv.z, gv.z, acc.z); acc.w = fmaf(wv.w, gv.w, acc.w);
+                        float4& a = accw[u * 3 + w];
+                        a.x = fmaf(gv.x, vt.x, a.x); a.y = fmaf(gv.y, vt.y, a.y);
+                        a.z = fmaf(gv.z, vt.z, a.z); a.w = fmaf(gv.w, vt.w, a.w);
+                    }
+                *vo = acc;
+            }
+        }
+    if (!dwd) return;
+#pragma unroll
+    for (int k = 0; k < 9; ++k) red[threadIdx.x * 9 + k] = accw[k];
     __syncthreads();
     for (int o = threadIdx.x; o < p.d * 9; o += 256) {           // o = c * 9 + tap, the layout of dWd
-        const int c = o / 9, k = o - c * 9;
-        const int q4 = c >> 2, e = c & 3;
+        const int cc = o / 9, k = o - cc * 9;
+        const int q4 = cc >> 2, e = cc & 3;
         float s = 0.f;
         for (int l = 0; l < lanes; ++l) {
             const float4 t = red[(l * d4 + q4) * 9 + k];
@@ -516,6 +527,8 @@ cudaError_t backward_typed(const BwdCall& c, BwdArgs a, cudaStream_t st) {
 
     bwd_pool_kernel<T><<<(unsigned)((snd + 255) / 256), 256, 0, st>>>(a, c.q, c.ws_a);
     AA_TRY(cudaGetLastError());
+    bwd_window_table_kernel<<<(unsigned)((a.N + 255) / 256), 256, 0, st>>>(a, c.ws_tab);
+    AA_TRY(cudaGetLastError());
     // aggregation forward: row statistics, then V_A
     a.x = c.k; a.y = c.v; a.bias = c.b1; a.m0 = c.ws_a; a.m1 = nullptr; a.scale = c.scale1;
     a.part = c.ws_part; a.dbias = nullptr;
@@ -559,14 +572,10 @@ cudaError_t backward_typed(const BwdCall& c, BwdArgs a, cudaStream_t st) {
     }
     // pooling and depthwise terms
     {
-        const dim3 grid((unsigned)(((size_t)a.N * (a.d / 4) + 255) / 256), (unsigned)a.slabs);
-        bwd_tail_kernel<T><<<grid, 256, 0, st>>>(a, c.ws_da, c.d_out, c.wd, c.dq, c.dv);
-        AA_TRY(cudaGetLastError());
-    }
-    if (c.dwd) {
         int chunks = (4 * c.sm_count + a.slabs - 1) / a.slabs;          // short loops (they are load-latency bound), few atomics
         chunks = max(1, min(chunks, (a.N + 63) / 64));
-        bwd_dwd_kernel<T><<<a.slabs * chunks, 256, 0, st>>>(a, c.d_out, c.v, c.dwd, chunks);
+        bwd_tail_kernel<T><<<a.slabs * chunks, 256, 0, st>>>(a, c.ws_tab, c.ws_da, c.d_out, c.v, c.wd, c.dq, c.dv, c.dwd,
+                                                              chunks);
         AA_TRY(cudaGetLastError());
     }
 #undef AA_TRY
@@ -601,7 +610,7 @@ bool plan_backward(int slabs, int n, int N, int d, int sm_count, BwdPlan* out) {
     return true;
 }
 
-int backward_launch_count(bool with_dwd, bool use_mma) { return (use_mma ? 8 : 9) + (with_dwd ? 1 : 0); }
+int backward_launch_count(bool use_mma) { return use_mma ? 8 : 9; }
 
 cudaError_t launch_backward(int dtype, const BwdCall& c, cudaStream_t st) {
     BwdArgs a;

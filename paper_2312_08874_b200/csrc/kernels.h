@@ -170,6 +170,7 @@ struct BwdCall {
     float *ws_a, *ws_va, *ws_dva, *ws_da;     // [slabs][n][d] each; V_A, dV_A, dA contiguous in this order
     float *ws_lse, *ws_dot;                   // [slabs][n]
     float* ws_part;                           // [slabs][chunks][n][2]
+    int4* ws_tab;                             // [N][3]: pooling windows of each token
     size_t clear_bytes;                       // bytes from ws_va to the end of ws_da
     int slabs, heads, H, W, d, n, p, sm_count;
     float scale1, scale2;
@@ -179,7 +180,7 @@ struct BwdCall {
     BwdPlan plan_mma;                         // their tiling
 };
 bool plan_backward(int slabs, int n, int N, int d, int sm_count, BwdPlan* out);   // false: shape not supported
-int backward_launch_count(bool with_dwd, bool use_mma);
+int backward_launch_count(bool use_mma);
 cudaError_t launch_backward(int dtype, const BwdCall& c, cudaStream_t st);
 // Tensor-core kernels of the two gradient stages (16-bit inputs, n <= 64, d = 64)
 bool backward_mma_eligible(int dtype, int n, int d);
