@@ -162,9 +162,13 @@ size_t agent_attn_backward_workspace_bytes(const agent_attn_handle* h, int grid_
  *   grads            host struct of fp32 device buffers (see agent_attn_grads)
  *   workspace        device, >= agent_attn_backward_workspace_bytes(...)
  * n_agents must be a perfect square p*p with p <= min(grid_h, grid_w), and n_agents * head_dim <= 16384.
- * All arithmetic is fp32 on CUDA cores for every element type and path setting.  Sums over tokens
- * and over the batch are accumulated with floating-point atomics, so the low-order bits of the results
- * may differ from run to run (the one exception to the reproducibility rule above).
+ * Arithmetic: handles created with AA_PATH_AUTO run the three attention stages on the tensor cores for 16-bit
+ * element types with n_agents <= 64 and head_dim == 64 (A, the probabilities and the logit gradients are
+ * rounded to the element type before they enter a product, as in the forward pass; V_A, dV_A and the
+ * probabilities that form V_A are carried as two 16-bit terms); every other shape, fp32 inputs, and handles
+ * created with AA_PATH_SIMT or AA_PATH_UNFUSED compute in fp32 on CUDA cores throughout.  Sums over tokens
+ * and over the batch are accumulated with floating-point atomics, so the low-order bits of the results may
+ * differ from run to run (the one exception to the reproducibility rule above).
  * Errors: AA_ERR_INVALID_ARG (null, misaligned or aliasing buffers, n not a square, dwd without a
  * filter), AA_ERR_UNSUPPORTED (shape limits), AA_ERR_WORKSPACE, AA_ERR_CUDA.  No host synchronisation,
  * no allocation. */
