@@ -74,8 +74,9 @@ __device__ __forceinline__ unsigned ld_acquire(const unsigned* p) {
     return v;
 }
 // Thread 0 polls until *ctr >= target; gives up after kSpinLimit polls and records `code`.
-__device__ __forceinline__ void wait_counter(const unsigned* ctr, unsigned target, int* status, int code) {
-    if (threadIdx.x == 0) {
+// `known` (read by thread 0 only): thread 0 has already seen the counter at its target (acquire load).
+__device__ __forceinline__ void wait_counter(const unsigned* ctr, unsigned target, int* status, int code, bool known = false) {
+    if (threadIdx.x == 0 && !known) {
         unsigned spins = 0;
         while (ld_acquire(ctr) < target) {
             if (++spins > kSpinLimit) { atomicExch(status, code); break; }
@@ -168,7 +169,7 @@ using ShapeAny = FusedShape<0, 0, 0, false>;
 // ---------------------------------------------------------------------------------- G task
 template <typename T, typename SH>
 __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub, unsigned char* smem,
-                                           BlockState& st, int* s_flag, int slot) {
+                                           BlockState& st, int* s_flag, int slot, int& next_task) {
     constexpr int NWK = 2, KW = KT / NWK;
     constexpr int cpr = DK / 8;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -472,6 +473,8 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
     unsigned* arrived = p.counters + p.slabs + slab;
     publish_add(arrived);
     wait_counter(arrived, (unsigned)p.plan.g_tasks, p.status, kTimeoutAgents);
+    // no wait lies ahead in this task: take the next ticket now, so that the queue's round trip runs under the merge
+    if (tid == 0) next_task = (int)atomicAdd(p.counters + 3 * (size_t)p.slabs, 1u);
     {
         const int rows_per = (n + p.plan.g_tasks - 1) / p.plan.g_tasks;
         const int rb = sub * rows_per, re = min(n, rb + rows_per);
@@ -515,7 +518,7 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
 // depthwise term (Eq. 6), round once and store.
 template <typename T, typename SH>
 __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int tile, unsigned char* smem,
-                                           BlockState& st, int* s_whead, float (*s_red)[128], int slot) {
+                                           BlockState& st, int* s_whead, float (*s_red)[128], int slot, int& next_task) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int head = slab % p.heads;
     const int H = SH::kFixed ? SH::kH : p.H, W = SH::kFixed ? SH::kW : p.W;
@@ -604,7 +607,7 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
 
     TRACE(slot, 1);
     // 2. wait for the slab's agent features, then fetch A and V_A (L2)
-    wait_counter(va_flag, va_target, p.status, kTimeoutFeatures);
+    wait_counter(va_flag, va_target, p.status, kTimeoutFeatures, early);
     TRACE(slot, 2);
     if (tid == 0 && has_dwc) *s_whead = head;
     if (!early) issue_agents();
@@ -720,6 +723,8 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
     }
     __syncthreads();
     TRACE(slot, 4);
+    // the rest of the task waits for nothing: take the next ticket now, so that the queue's round trip runs under it
+    if (tid == 0) next_task = (int)atomicAdd(p.counters + 3 * (size_t)p.slabs, 1u);
 
     // 4. depthwise 3x3 term + store: thread = (tile row r, 4-channel group cq, x-segment)
     {
@@ -824,8 +829,9 @@ __global__ void __launch_bounds__(NT, 2) fused_kernel(const __grid_constant__ Fu
     const int total = S * (G + B);
     unsigned* queue = p.counters + 3 * (size_t)S;
     int slot = 0;
+    int next_task = -1;                 // thread 0: ticket taken ahead by the previous task
     for (;;) {
-        if (tid == 0) s_task = (int)atomicAdd(queue, 1u);
+        if (tid == 0) s_task = next_task >= 0 ? next_task : (int)atomicAdd(queue, 1u);
         __syncthreads();
         const int task = s_task;
         __syncthreads();
@@ -846,8 +852,9 @@ __global__ void __launch_bounds__(NT, 2) fused_kernel(const __grid_constant__ Fu
             const int step = t / B;
             slab = S - Lg + step; sub = t - step * B; is_g = false;
         }
-        if (is_g) run_g_task<T, SH>(p, slab, sub, smem, st, &s_flag, slot);
-        else      run_b_task<T, SH>(p, slab, sub, smem, st, &s_whead, s_red, slot);
+        next_task = -1;
+        if (is_g) run_g_task<T, SH>(p, slab, sub, smem, st, &s_flag, slot, next_task);
+        else      run_b_task<T, SH>(p, slab, sub, smem, st, &s_whead, s_red, slot, next_task);
 #ifdef AA_FUSED_TRACE
         if (tid == 0 && g_trace && slot < 16) {
             g_trace[((size_t)blockIdx.x * 16 + slot) * 8 + 6] = is_g ? 1 : 2;
