@@ -505,9 +505,7 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
         }
     }
     publish_add(p.counters + 2 * p.slabs + slab);
-    fence_proxy_async();   // this task's plain shared-memory writes precede the next task's TMA writes
-    __syncthreads();       // the ring is free for the next task
-    TRACE(slot, 5);
+    // (the caller closes the task: proxy fence and block barrier, after which the ring is free)
 }
 
 // ---------------------------------------------------------------------------------- B task
@@ -548,7 +546,7 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
     const bool early = ld_acquire(va_flag) >= va_target;      // usual case: the slab's aggregation is long done
     auto issue_agents = [&]() {
         if (tid == 0) {
-            mbar_arrive_expect_tx(bar_agents(st), 2 * kTileBytes);
+            mbar_arrive_expect_tx(bar_agents(st), kTileBytes + (uint32_t)n * 128u);     // A: 64-row box, V_A: n-row box
             tma_load_2d(smem_u32(sA), &p.tm_a, 0, slab * n, bar_agents(st));
             tma_load_2d(smem_u32(sVA), &p.tm_va, 0, slab * n, bar_agents(st));
         }
@@ -618,11 +616,7 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
         st.ph ^= 1u << kBitBin;
     }
     __syncthreads();
-    // rows >= n of the V_A tile hold foreign rows: they must be zero, since 0 * NaN is not 0
-    for (int e = tid; e < (RP - n) * 8; e += NT)
-        *(reinterpret_cast<uint4*>(sVA + (n + e / 8) * 128) + (e & 7)) = make_uint4(0, 0, 0, 0);
-    fence_proxy_async();          // the tensor core reads V_A through the async proxy
-    __syncthreads();
+    // (rows >= n of the V_A tile are zero: the copy brings n rows and the kernel cleared the rest at its start)
 
     TRACE(slot, 3);
     // 3. attention part on the 5th-generation tensor cores: logits S = Q A^T accumulate in tensor
@@ -795,16 +789,14 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
             }
         }
     }
-    fence_proxy_async();   // this task's plain shared-memory writes precede the next task's TMA writes
-    __syncthreads();       // shared memory is free for the next task
-    TRACE(slot, 5);
+    // (the caller closes the task: proxy fence and block barrier, after which shared memory is free)
 }
 
 // ---------------------------------------------------------------------------------- kernel
 template <typename T, typename SH>
 __global__ void __launch_bounds__(NT, 2) fused_kernel(const __grid_constant__ FusedArgs p) {
     extern __shared__ unsigned char smem_raw[];
-    __shared__ int s_task, s_flag, s_whead;
+    __shared__ int s_task[2], s_flag, s_whead;
     __shared__ uint32_t s_tmem;
     __shared__ float s_red[4][128];     // per query row: partial maxima and partial sums of the two column halves
     // TMA tiles with the 128-byte swizzle want a 1024-byte aligned base
@@ -818,6 +810,10 @@ __global__ void __launch_bounds__(NT, 2) fused_kernel(const __grid_constant__ Fu
         for (int i = 0; i < kNumBars; ++i) mbar_init(st.bar_base + 8 * i, 1);
         mbar_fence_init();
     }
+    // rows >= n of the V_A tile never receive data (its copies bring n rows): zero, since 0 * NaN is not 0
+    for (int e = tid; e < (RP - p.n) * 8; e += NT)
+        *(reinterpret_cast<uint4*>(smem + OFF_VA + (p.n + e / 8) * 128) + (e & 7)) = make_uint4(0, 0, 0, 0);
+    fence_proxy_async();          // the tensor core reads V_A through the async proxy
     // tensor memory for the broadcast MMAs: warp 0 allocates (and frees at the end)
     if (tid < 32) tmem_alloc<kTmemCols>(smem_u32(&s_tmem));
     tc_fence_before_sync();
@@ -829,12 +825,13 @@ __global__ void __launch_bounds__(NT, 2) fused_kernel(const __grid_constant__ Fu
     const int total = S * (G + B);
     unsigned* queue = p.counters + 3 * (size_t)S;
     int slot = 0;
-    int next_task = -1;                 // thread 0: ticket taken ahead by the previous task
-    for (;;) {
-        if (tid == 0) s_task = next_task >= 0 ? next_task : (int)atomicAdd(queue, 1u);
-        __syncthreads();
-        const int task = s_task;
-        __syncthreads();
+    // Every task takes the ticket of the block's next task at the start of its wait-free tail (thread 0) and
+    // the ticket is handed to the block through s_task[] before the task's closing barrier, so no barrier of
+    // its own is spent on the queue.  Two slots: a slot is rewritten two tasks after it was read.
+    if (tid == 0) s_task[0] = (int)atomicAdd(queue, 1u);
+    __syncthreads();
+    for (int par = 0;; par ^= 1) {
+        const int task = s_task[par];
         if (task >= total) break;
         // queue order: step i holds the G tasks of slab i (i < S) and the B tasks of slab i - lag (i >= lag)
         int slab, sub;
@@ -852,9 +849,13 @@ __global__ void __launch_bounds__(NT, 2) fused_kernel(const __grid_constant__ Fu
             const int step = t / B;
             slab = S - Lg + step; sub = t - step * B; is_g = false;
         }
-        next_task = -1;
+        int next_task = total;          // thread 0: set by the task
         if (is_g) run_g_task<T, SH>(p, slab, sub, smem, st, &s_flag, slot, next_task);
         else      run_b_task<T, SH>(p, slab, sub, smem, st, &s_whead, s_red, slot, next_task);
+        if (tid == 0) s_task[par ^ 1] = next_task;
+        fence_proxy_async();   // this task's plain shared-memory writes precede the next task's TMA writes
+        __syncthreads();       // shared memory is free for the next task, and its ticket is visible
+        TRACE(slot, 5);
 #ifdef AA_FUSED_TRACE
         if (tid == 0 && g_trace && slot < 16) {
             g_trace[((size_t)blockIdx.x * 16 + slot) * 8 + 6] = is_g ? 1 : 2;

@@ -133,7 +133,7 @@ bool fused_make_maps(FusedArgs* a) {
         !make_map_tok_u16(&a->tm_vrow, &a->hf_vrow, a->v, a->lin, batch, a->heads, (long long)N, DK, (uint32_t)a->W, false))
         return false;
     if (!make_map_2d_u16(&a->tm_a, a->a_ws, S * a->n, DK, RP, DK)) return false;
-    if (!make_map_2d_u16(&a->tm_va, a->va_ws, S * a->n, DK, RP, DK)) return false;
+    if (!make_map_2d_u16(&a->tm_va, a->va_ws, S * a->n, DK, (uint32_t)a->n, DK)) return false;    // box of n rows
     a->b1_tma = 0;
     if (a->b1 && N % 8 == 0 && ((uint64_t)a->plan.rows_per_g * a->W) % 8 == 0 && N >= KT)
         a->b1_tma = make_map_2d_u16(&a->tm_b1, a->b1, (uint64_t)a->heads * a->n, N, RP, KT) ? 1 : 0;
