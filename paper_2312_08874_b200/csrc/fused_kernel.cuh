@@ -104,6 +104,14 @@ __device__ __forceinline__ void wait_bar(uint32_t bar, uint32_t parity, int* sta
         }
     }
 }
+// Every thread waits (bounded) for a phase of an mbarrier itself, parked by the suspended form of try_wait: no
+// block barrier is needed to pass the completion on.  On expiry the thread records `code` and goes on.
+__device__ __forceinline__ void wait_bar_all(uint32_t bar, uint32_t parity, int* status, int code) {
+    if (mbar_try_wait_suspend(bar, parity, 2000u)) return;
+    for (unsigned tries = 0; tries < (1u << 20); ++tries)
+        if (mbar_try_wait_suspend(bar, parity, 2000u)) return;
+    atomicExch(status, code);
+}
 // Byte offset of element (row, col) in a swizzled [rows][64] tile of 16-bit elements: the 16-byte
 // chunk index is XORed with the row index modulo 8 (the TMA 128-byte swizzle).
 __device__ __forceinline__ int swz(int row, int col) {
@@ -638,9 +646,8 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
                 umma_f16(tS, umma_desc_sw128(smem_u32(sQt) + kk * 32), umma_desc_sw128(smem_u32(sA) + kk * 32), idesc, kk > 0);
             umma_commit(bar_mma(st));
         }
-        wait_bar(bar_mma(st), (st.ph >> kBitMma) & 1u, p.status, kTimeoutLoads);
+        wait_bar_all(bar_mma(st), (st.ph >> kBitMma) & 1u, p.status, kTimeoutLoads);
         st.ph ^= 1u << kBitMma;
-        __syncthreads();
         tc_fence_after_sync();
         float s[32];
         {
@@ -697,9 +704,8 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
                 umma_f16(tO, umma_desc_sw128(smem_u32(sPt) + kk * 32), umma_desc_sw128(smem_u32(sVA) + kk * 2048), idesc, kk > 0);
             umma_commit(bar_mma(st));
         }
-        wait_bar(bar_mma(st), (st.ph >> kBitMma) & 1u, p.status, kTimeoutLoads);
+        wait_bar_all(bar_mma(st), (st.ph >> kBitMma) & 1u, p.status, kTimeoutLoads);
         st.ph ^= 1u << kBitMma;
-        __syncthreads();
         tc_fence_after_sync();
         const float inv = 1.f / (s_red[2][row] + s_red[3][row]);
         float* prow = sPatchAll + row * PO + c0;
