@@ -73,18 +73,19 @@ __device__ __forceinline__ unsigned ld_acquire(const unsigned* p) {
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
-// Thread 0 polls until *ctr >= target; gives up after kSpinLimit polls and records `code`.
-// `known` (read by thread 0 only): thread 0 has already seen the counter at its target (acquire load).
-__device__ __forceinline__ void wait_counter(const unsigned* ctr, unsigned target, int* status, int code, bool known = false) {
-    if (threadIdx.x == 0 && !known) {
-        unsigned spins = 0;
-        while (ld_acquire(ctr) < target) {
-            if (++spins > kSpinLimit) { atomicExch(status, code); break; }
-            // once any block has given up, the others stop waiting too
-            if ((spins & 255u) == 0 && ld_acquire(reinterpret_cast<const unsigned*>(status)) != 0u) break;
-            __nanosleep(40);
-        }
+// The calling thread polls until *ctr >= target; gives up after kSpinLimit polls and records `code`.
+__device__ __forceinline__ void poll_counter(const unsigned* ctr, unsigned target, int* status, int code) {
+    unsigned spins = 0;
+    while (ld_acquire(ctr) < target) {
+        if (++spins > kSpinLimit) { atomicExch(status, code); break; }
+        // once any block has given up, the others stop waiting too
+        if ((spins & 255u) == 0 && ld_acquire(reinterpret_cast<const unsigned*>(status)) != 0u) break;
+        __nanosleep(40);
     }
+}
+// Thread 0 polls, then a block barrier passes the result on.
+__device__ __forceinline__ void wait_counter(const unsigned* ctr, unsigned target, int* status, int code) {
+    if (threadIdx.x == 0) poll_counter(ctr, target, status, code);
     __syncthreads();
 }
 // Publish: all of this block's prior global writes become visible before the counter moves.
@@ -613,9 +614,9 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
 
     TRACE(slot, 1);
     // 2. wait for the slab's agent features, then fetch A and V_A (L2)
-    wait_counter(va_flag, va_target, p.status, kTimeoutFeatures, early);
+    //    (thread 0 alone: the barrier below passes everything on; a flag already seen set is not read again)
+    if (tid == 0 && !early) poll_counter(va_flag, va_target, p.status, kTimeoutFeatures);
     TRACE(slot, 2);
-    if (tid == 0 && has_dwc) *s_whead = head;
     if (!early) issue_agents();
     wait_bar(bar_agents(st), (st.ph >> kBitAgents) & 1u, p.status, kTimeoutLoads);
     st.ph ^= 1u << kBitAgents;
@@ -624,6 +625,7 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
         st.ph ^= 1u << kBitBin;
     }
     __syncthreads();
+    if (tid == 0 && has_dwc) *s_whead = head;      // every thread has compared the old value before the barrier
     // (rows >= n of the V_A tile are zero: the copy brings n rows and the kernel cleared the rest at its start)
 
     TRACE(slot, 3);
