@@ -61,7 +61,7 @@ constexpr int OFF_B2 = OFF_HALO + kHaloBytes;
 constexpr int kB2Bytes = QT * RP * 2 + 16;              // + one spare vector: pairs are read as two words
 constexpr int kBBytes = kPatchBytes + kHaloBytes + kB2Bytes;
 constexpr int OFF_BAR = OFF_UNION + (kGBytes > kBBytes ? kGBytes : kBBytes);   // mbarriers (8 bytes each)
-constexpr int kNumBars = STAGES + 3;                    // ring stages, agents, broadcast inputs, MMA completion
+constexpr int kNumBars = STAGES + 4;                    // ring stages, agents, Q tile, MMA completion, V rows + B2 tile
 constexpr int kTmemCols = 128;                          // per block: 64 columns of logits + 64 of output
 static_assert(kPatchBytes >= 2 * QT * 128, "the Q and P operand tiles alias the patch");
 constexpr int kSmemBytes = OFF_BAR + 8 * kNumBars + 1024;   // + slack to align the base to 1024
@@ -156,11 +156,12 @@ struct BlockState {
     uint32_t ph;                // parity to wait for next: bit s = ring stage s, then agents, broadcast inputs, MMA
     uint32_t tmem;              // base address of this block's tensor-memory columns
 };
-constexpr int kBitAgents = STAGES, kBitBin = STAGES + 1, kBitMma = STAGES + 2;
+constexpr int kBitAgents = STAGES, kBitBin = STAGES + 1, kBitMma = STAGES + 2, kBitVb = STAGES + 3;
 __device__ __forceinline__ uint32_t bar_full(const BlockState& st, int s) { return st.bar_base + 8 * s; }
 __device__ __forceinline__ uint32_t bar_agents(const BlockState& st) { return st.bar_base + 8 * STAGES; }
 __device__ __forceinline__ uint32_t bar_bin(const BlockState& st) { return st.bar_base + 8 * (STAGES + 1); }
 __device__ __forceinline__ uint32_t bar_mma(const BlockState& st) { return st.bar_base + 8 * (STAGES + 2); }
+__device__ __forceinline__ uint32_t bar_vb(const BlockState& st) { return st.bar_base + 8 * (STAGES + 3); }
 // barrier among the 128 threads of warps 0-3 (the threads that own TMEM lanes in the broadcast)
 __device__ __forceinline__ void sync_rows() { asm volatile("bar.sync 1, 128;\n" ::: "memory"); }
 }  // namespace
@@ -566,12 +567,18 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
     const bool b2_bulk = has_b2 && ((reinterpret_cast<uintptr_t>(b2src) & 15u) == 0) && ((b2bytes & 15) == 0);
     int vrows = 0;
     if (has_dwc) vrows = min(H, y0 + rows + 1) - max(0, y0 - 1);
-    const uint32_t bin_bytes = (uint32_t)QT * DK * 2 + (uint32_t)vrows * W * DK * 2 + (b2_bulk ? b2bytes : 0);
+    // Two threads share the issue work, each with a barrier of its own: thread 0 brings the Q tile (and A, V_A below),
+    // lane 0 of warp 1 the V rows and the B2 tile, so that neither instruction stream waits for the other.
+    const uint32_t vb_bytes = (uint32_t)vrows * W * DK * 2 + (b2_bulk ? b2bytes : 0);
     if (tid == 0) {
         const uint32_t bar = bar_bin(st);
-        mbar_arrive_expect_tx(bar, bin_bytes);
+        mbar_arrive_expect_tx(bar, (uint32_t)QT * DK * 2);
         // Q tile: 128 rows from the tile's first token (rows past the tile feed rows that are never stored)
         load_tokens(smem_u32(smem + OFF_PATCH), &p.tm_q, SH::kDense ? 1 : p.dense_in, p.hf_q, q0, head, slab / p.heads, slab * N, bar);
+    }
+    if (tid == 32 && vb_bytes) {
+        const uint32_t bar = bar_vb(st);
+        mbar_arrive_expect_tx(bar, vb_bytes);
         if (has_dwc) {
             for (int hr = 0; hr < rows + 2; ++hr) {
                 const int y = y0 - 1 + hr;
@@ -620,9 +627,11 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
     if (!early) issue_agents();
     wait_bar(bar_agents(st), (st.ph >> kBitAgents) & 1u, p.status, kTimeoutLoads);
     st.ph ^= 1u << kBitAgents;
-    if (bin_bytes) {
-        wait_bar(bar_bin(st), (st.ph >> kBitBin) & 1u, p.status, kTimeoutLoads);
-        st.ph ^= 1u << kBitBin;
+    wait_bar(bar_bin(st), (st.ph >> kBitBin) & 1u, p.status, kTimeoutLoads);
+    st.ph ^= 1u << kBitBin;
+    if (vb_bytes) {
+        wait_bar(bar_vb(st), (st.ph >> kBitVb) & 1u, p.status, kTimeoutLoads);
+        st.ph ^= 1u << kBitVb;
     }
     __syncthreads();
     if (tid == 0 && has_dwc) *s_whead = head;      // every thread has compared the old value before the barrier
