@@ -42,6 +42,23 @@ def test_largest_config_matches_oracle_on_sampled_slabs():
         assert_close(out[b:b + 1, h:h + 1], ref, w.dtype, f"cfg5b slab {(b, h)}")
 
 
+def test_more_slabs_than_the_queue_lag_interleaves_task_kinds():
+    """With more slabs than the queue's lag (the L2 budget: 83 slabs of this shape) aggregation and broadcast tasks
+    alternate in the queue, so blocks take tickets of one kind while finishing a task of the other and broadcast
+    tasks may find their slab's flag not yet set: sampled slabs against the oracle, repeatable bit for bit, and no
+    bounded wait expired."""
+    w = WORKLOADS["cfg3_pvt_bf16"].scaled(batch=160, seed=77)
+    inp = make_inputs(w)
+    mod = make_module(w)
+    out = gpu_forward(mod, w, inp).clone()
+    again = gpu_forward(mod, w, inp)
+    assert torch.equal(out, again)
+    assert torch.isfinite(out.float()).all()
+    slabs = [(0, 0), (82, 0), (83, 0), (121, 0), (159, 0)]
+    for (b, h), ref in zip(slabs, oracle_forward(w, inp, slabs=slabs)):
+        assert_close(out[b:b + 1, h:h + 1], ref, w.dtype, f"slab {(b, h)} of 160")
+
+
 # ------------------------------------------------------- attention term must not hide under DWC
 @pytest.mark.parametrize("name", ["cfg3_pvt_bf16", "cfg5a_hires_bf16"])
 @pytest.mark.parametrize("variant", ["no_dwc", "shifted_v"])
