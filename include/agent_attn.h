@@ -50,10 +50,13 @@ typedef enum {
 } aa_status;
 
 typedef enum {
-    AA_PATH_AUTO = 0,         /* tensor-core kernels for bf16/f16 (one fused persistent kernel where the
-                                 shape allows it), fp32 FMA kernels for f32 */
+    AA_PATH_AUTO = 0,         /* tensor-core kernels for bf16/f16: three streaming kernels for long token grids
+                                 with few agents (n <= 64, d = 64, N >= 1024), one persistent task-queue kernel
+                                 for short ones, tensor-memory kernels for n > 64; fp32 FMA kernels for f32 */
     AA_PATH_SIMT = 1,         /* fp32 FMA kernels for every dtype (slow; for cross-checks) */
-    AA_PATH_UNFUSED = 2       /* like AUTO, but always one kernel per step (pool, aggregate, broadcast) */
+    AA_PATH_UNFUSED = 2,      /* like AUTO, but always one kernel per step (pool, aggregate, broadcast) */
+    AA_PATH_QUEUE = 3         /* like AUTO, but without the streaming kernels: the task-queue kernel wherever it
+                                 applies (n <= 64, d = 64, W <= 64), whatever the number of tokens */
 } aa_path;
 
 typedef struct {

@@ -15,7 +15,7 @@ import torch
 from .build import LIB_PATH, build_library
 
 AA_F32, AA_BF16, AA_F16 = 0, 1, 2
-AA_PATH_AUTO, AA_PATH_SIMT, AA_PATH_UNFUSED = 0, 1, 2
+AA_PATH_AUTO, AA_PATH_SIMT, AA_PATH_UNFUSED, AA_PATH_QUEUE = 0, 1, 2, 3
 STATUS_NAMES = {0: "AA_OK", 1: "AA_ERR_INVALID_ARG", 2: "AA_ERR_UNSUPPORTED", 3: "AA_ERR_WORKSPACE",
                 4: "AA_ERR_CUDA", 5: "AA_ERR_TIMEOUT"}
 _DTYPES = {torch.float32: AA_F32, torch.bfloat16: AA_BF16, torch.float16: AA_F16}

@@ -17,10 +17,15 @@ struct agent_attn_handle {
     float scale1, scale2;
     int sm_count;
     int elem_bytes;
-    int* d_status;          // one device word: bounded waits report here (none of the current kernels wait)
+    int* d_status;          // one device word: the kernels' bounded waits (mbarriers, flags) report here
     int launches;
     int fused_key[3];       // (grid_h, grid_w, n_agents) that fused_plan was made for
     FusedPlan fused_plan;
+    int stream_key[4];      // (grid_h, grid_w, n_agents, pooled) that stream_plan was made for
+    StreamPlan stream_plan;
+    StreamArgs stream_args; // last call of the streaming path: its tensor maps are reused while the pointers repeat
+    bool stream_args_valid;
+    unsigned poll_limit;    // flag-poll limit of the task-queue kernel (test hook; 0xffffffff = the kernel's own)
     char err[512];
 };
 
@@ -41,6 +46,9 @@ int fail(agent_attn_handle* h, int code, const char* fmt, ...) {
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
 
+// AA_PATH_QUEUE differs from AA_PATH_AUTO only in skipping the streaming kernels.
+bool auto_like(const agent_attn_handle* h) { return h->cfg.path == AA_PATH_AUTO || h->cfg.path == AA_PATH_QUEUE; }
+
 bool use_simt(const agent_attn_handle* h) {
     return h->cfg.dtype == AA_F32 || h->cfg.path == AA_PATH_SIMT;
 }
@@ -48,7 +56,7 @@ bool use_simt(const agent_attn_handle* h) {
 // Large agent counts go to the tensor-memory kernel (the shape rule does not depend on the bias, so
 // that the workspace size is the same with and without one).
 bool use_umma(const agent_attn_handle* h, int n_tokens, int n_agents) {
-    return !use_simt(h) && h->cfg.path == AA_PATH_AUTO &&
+    return !use_simt(h) && auto_like(h) &&
            aggregate_umma_eligible(h->cfg.dtype, n_agents, n_tokens, h->cfg.head_dim, true);
 }
 
@@ -60,9 +68,25 @@ AggPlan plan_for(const agent_attn_handle* h, int n_tokens, int n_agents) {
                        : plan_aggregate_mma(slabs, n_agents, n_tokens, h->cfg.head_dim, h->sm_count);
 }
 
-// Workspace layout: [A | V_A | partials | tickets], each region 256-byte aligned.
+// Plan of the streaming path for a call shape (cached in the handle); ok = false where it does not apply.
+const StreamPlan& stream_plan_for(agent_attn_handle* h, int grid_h, int grid_w, int n_agents, bool pooled) {
+    if (h->stream_key[0] != grid_h || h->stream_key[1] != grid_w || h->stream_key[2] != n_agents ||
+        h->stream_key[3] != (pooled ? 1 : 2)) {
+        h->stream_plan = (h->cfg.path == AA_PATH_AUTO && h->cfg.dtype != AA_F32)
+                             ? plan_stream(h->cfg.dtype, h->cfg.batch * h->cfg.heads, grid_h, grid_w, h->cfg.head_dim,
+                                           n_agents, pooled, h->sm_count)
+                             : StreamPlan{};
+        h->stream_key[0] = grid_h; h->stream_key[1] = grid_w; h->stream_key[2] = n_agents;
+        h->stream_key[3] = pooled ? 1 : 2;
+        h->stream_args_valid = false;
+    }
+    return h->stream_plan;
+}
+
+// Workspace layout: [A | V_A | partials | tickets | streaming path: scaled agents, prepared biases], each region
+// 256-byte aligned.
 struct WsLayout {
-    size_t a_off, va_off, part_off, ticket_off, total;
+    size_t a_off, va_off, part_off, ticket_off, extra_off, total;
 };
 WsLayout ws_layout(const agent_attn_handle* h, int n_tokens, int n_agents, int grid_h = 0, int grid_w = 0) {
     const size_t slabs = (size_t)h->cfg.batch * h->cfg.heads;
@@ -74,13 +98,27 @@ WsLayout ws_layout(const agent_attn_handle* h, int n_tokens, int n_agents, int g
     w.part_off = 2 * av;
     // sized for either launch plan (per-step kernels or the fused kernel)
     size_t part_floats = slabs * pl.parts * partial_floats(pl.rows_pad, pl.dpad);
-    if (grid_h > 0 && h->cfg.path == AA_PATH_AUTO) {
+    if (grid_h > 0 && auto_like(h)) {
         const size_t fused_floats = slabs * (size_t)fused_parts_per_slab(h->cfg.dtype, grid_h, grid_w, h->cfg.head_dim, n_agents) *
                                     partial_floats(64, h->cfg.head_dim);
         if (part_floats < fused_floats) part_floats = fused_floats;
     }
+    size_t extra = 0;
+    if (grid_h > 0) {
+        // the larger of the plans for pooled and for caller-supplied agents (the size must not depend on A)
+        for (int pooled = 0; pooled < 2; ++pooled) {
+            const StreamPlan sp = (h->cfg.path == AA_PATH_AUTO && h->cfg.dtype != AA_F32)
+                                      ? plan_stream(h->cfg.dtype, (int)slabs, grid_h, grid_w, h->cfg.head_dim, n_agents, pooled != 0, h->sm_count)
+                                      : StreamPlan{};
+            if (!sp.ok) continue;
+            const size_t sf = slabs * (size_t)sp.splits * partial_floats(64, 64);
+            if (part_floats < sf) part_floats = sf;
+            extra = stream_extra_bytes((int)slabs, h->cfg.heads, n_tokens, n_agents);
+        }
+    }
     w.ticket_off = w.part_off + align_up(part_floats * sizeof(float), 256);
-    w.total = w.ticket_off + align_up(fused_counter_words((int)slabs) * sizeof(unsigned), 256);
+    w.extra_off = w.ticket_off + align_up(fused_counter_words((int)slabs) * sizeof(unsigned), 256);
+    w.total = w.extra_off + extra;
     return w;
 }
 
@@ -166,7 +204,7 @@ int do_broadcast(agent_attn_handle* h, const void* Q, const void* A, const void*
     a.lin = cl ? cl->in : dense_layout(h->cfg.heads, (long long)gh * gw, h->cfg.head_dim);
     a.lout = cl ? cl->out : a.lin;
     a.strided = cl && cl->strided;
-    const bool umma = !use_simt(h) && h->cfg.path == AA_PATH_AUTO &&
+    const bool umma = !use_simt(h) && auto_like(h) &&
                       broadcast_umma_eligible(h->cfg.dtype, n, gh * gw, h->cfg.head_dim);
     if (a.strided && !umma)
         return fail(h, AA_ERR_UNSUPPORTED, "strided Q, V and out need the fused or the tensor-memory kernels (16-bit, d <= 64, n a multiple of 8 up to 256)");
@@ -200,7 +238,8 @@ int agent_attn_create(agent_attn_handle** out, const agent_attn_config* cfg) {
         cfg->max_agents <= 0 || cfg->scale1 < 0.f || cfg->scale2 < 0.f)
         return AA_ERR_INVALID_ARG;
     if (cfg->dtype != AA_F32 && cfg->dtype != AA_BF16 && cfg->dtype != AA_F16) return AA_ERR_UNSUPPORTED;
-    if (cfg->path != AA_PATH_AUTO && cfg->path != AA_PATH_SIMT && cfg->path != AA_PATH_UNFUSED) return AA_ERR_UNSUPPORTED;
+    if (cfg->path != AA_PATH_AUTO && cfg->path != AA_PATH_SIMT && cfg->path != AA_PATH_UNFUSED && cfg->path != AA_PATH_QUEUE)
+        return AA_ERR_UNSUPPORTED;
     const int es = cfg->dtype == AA_F32 ? 4 : 2;
     if (cfg->head_dim > 128 || cfg->head_dim < 8 || (cfg->head_dim * es) % 16 != 0) return AA_ERR_UNSUPPORTED;
     if (cfg->max_agents > 256) return AA_ERR_UNSUPPORTED;
@@ -226,6 +265,7 @@ int agent_attn_create(agent_attn_handle** out, const agent_attn_config* cfg) {
     const float def = 1.0f / std::sqrt((float)cfg->head_dim);
     h->scale1 = cfg->scale1 > 0.f ? cfg->scale1 : def;
     h->scale2 = cfg->scale2 > 0.f ? cfg->scale2 : def;
+    h->poll_limit = 0xffffffffu;
     if (cudaMalloc(&h->d_status, sizeof(int)) != cudaSuccess || cudaMemset(h->d_status, 0, sizeof(int)) != cudaSuccess) {
         delete h;
         return AA_ERR_CUDA;
@@ -308,8 +348,6 @@ int agent_attn_broadcast(agent_attn_handle* h, const void* Q, const void* A, con
     return do_broadcast(h, Q, A, VA, V, b2, dwc_weight, grid_h, grid_w, n_agents, out, (cudaStream_t)stream);
 }
 
-static bool fused_layout_ok(const CallLayout&) { return true; }
-
 static int forward_impl(agent_attn_handle* h, const void* Q, const void* K, const void* V, const void* A,
                         int grid_h, int grid_w, int n_agents, const agent_attn_bias* bias, const void* dwc_weight,
                         void* out, void* workspace, size_t workspace_bytes, void* stream, const CallLayout* clp) {
@@ -344,14 +382,47 @@ static int forward_impl(agent_attn_handle* h, const void* Q, const void* K, cons
     cudaStream_t st = (cudaStream_t)stream;
     char* ws = static_cast<char*>(workspace);
     const CallLayout cl = clp ? *clp : dense_call(h, N);
-    if (!A && h->cfg.path == AA_PATH_AUTO && h->cfg.dtype != AA_F32) {
+    if (h->cfg.path == AA_PATH_AUTO && h->cfg.dtype != AA_F32 && !cl.strided) {
+        // long token grids with few agents: three streaming kernels, phase by phase over the batch
+        const StreamPlan& sp = stream_plan_for(h, grid_h, grid_w, n_agents, A == nullptr);
+        if (sp.ok) {
+            const int slabs = h->cfg.batch * h->cfg.heads;
+            StreamArgs sa;
+            memset(&sa, 0, sizeof(sa));
+            sa.q = Q; sa.k = K; sa.v = V; sa.a_user = A; sa.b1 = b1; sa.b2 = b2; sa.dwc_w = dwc_weight; sa.out = out;
+            sa.a_ws = ws + w.a_off; sa.va_ws = ws + w.va_off;
+            const size_t av = align_up((size_t)slabs * n_agents * 64 * 2, 256);
+            sa.a1s = ws + w.extra_off; sa.a2s = ws + w.extra_off + av;
+            sa.b1c = ws + w.extra_off + 2 * av;
+            sa.b2p = ws + w.extra_off + 2 * av + align_up((size_t)h->cfg.heads * N * 64 * 2, 256);
+            sa.partials = reinterpret_cast<float*>(ws + w.part_off);
+            sa.tickets = reinterpret_cast<unsigned*>(ws + w.ticket_off);
+            sa.status = h->d_status;
+            sa.slabs = slabs; sa.heads = h->cfg.heads; sa.H = grid_h; sa.W = grid_w; sa.n = n_agents; sa.p = p;
+            sa.scale1 = h->scale1; sa.scale2 = h->scale2; sa.sm_count = h->sm_count; sa.plan = sp;
+            // the tensor maps depend on the pointers and the shape only: reuse them while both repeat
+            const size_t key_bytes = offsetof(StreamArgs, tm_k);
+            if (h->stream_args_valid && memcmp(&sa, &h->stream_args, key_bytes) == 0) {
+                sa = h->stream_args;
+            } else {
+                if (!stream_make_maps(&sa)) return fail(h, AA_ERR_CUDA, "tensor map encoding failed");
+                h->stream_args = sa;
+                h->stream_args_valid = true;
+            }
+            cudaError_t e = launch_stream(h->cfg.dtype, sa, st);
+            if (e != cudaSuccess) return fail(h, AA_ERR_CUDA, "streaming launch failed: %s", cudaGetErrorString(e));
+            h->launches = 3;
+            return AA_OK;
+        }
+    }
+    if (!A && auto_like(h) && h->cfg.dtype != AA_F32) {
         // one persistent kernel for the whole module where the shape allows it
         if (h->fused_key[0] != grid_h || h->fused_key[1] != grid_w || h->fused_key[2] != n_agents) {
             h->fused_plan = plan_fused(h->cfg.dtype, h->cfg.batch * h->cfg.heads, grid_h, grid_w, h->cfg.head_dim,
                                        n_agents, h->sm_count);
             h->fused_key[0] = grid_h; h->fused_key[1] = grid_w; h->fused_key[2] = n_agents;
         }
-        if (h->fused_plan.ok && fused_layout_ok(cl)) {
+        if (h->fused_plan.ok) {
             const int slabs = h->cfg.batch * h->cfg.heads;
             unsigned* counters = reinterpret_cast<unsigned*>(ws + w.ticket_off);
             cudaError_t e = cudaMemsetAsync(counters, 0, fused_counter_words(slabs) * sizeof(unsigned), st);
@@ -599,7 +670,7 @@ int agent_attn_backward(agent_attn_handle* h, const void* Q, const void* K, cons
     c.d = h->cfg.head_dim; c.n = n_agents; c.p = p; c.sm_count = h->sm_count;
     c.scale1 = h->scale1; c.scale2 = h->scale2;
     c.dtype = h->cfg.dtype;
-    c.use_mma = h->cfg.path == AA_PATH_AUTO && backward_mma_eligible(h->cfg.dtype, n_agents, h->cfg.head_dim);
+    c.use_mma = auto_like(h) && backward_mma_eligible(h->cfg.dtype, n_agents, h->cfg.head_dim);
     if (c.use_mma) c.plan_mma = plan_backward_mma(c.slabs, N, h->sm_count);
     cudaError_t e = launch_backward(h->cfg.dtype, c, (cudaStream_t)stream);
     if (e != cudaSuccess) return fail(h, AA_ERR_CUDA, "backward launch failed: %s", cudaGetErrorString(e));

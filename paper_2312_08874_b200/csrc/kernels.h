@@ -143,6 +143,47 @@ cudaError_t launch_fused(int dtype, const FusedArgs& a, cudaStream_t st);
 int fused_parts_per_slab(int dtype, int H, int W, int d, int n_agents);   // 0 if the shape is not eligible
 inline size_t fused_counter_words(int slabs) { return 3 * (size_t)slabs + 4; }
 
+// Whole module (Eq. 6) for small agent counts and long token grids (n <= 64, d = 64, N >= 1024, dense tensors)
+// as three streaming kernels, phase by phase over the batch (the second reads of Q and V come from L2):
+//   prep       agents A = Pooling(Q) (or the caller's A), scaled copies for the two logit products, biases
+//              clamped to finite values (B2 also padded to 64 columns), arrival counters cleared
+//   aggregate  V_A = softmax(scale1 A K^T + B1) V: grid (splits, slabs), tcgen05 with the agents and the
+//              probabilities as tensor-memory operands, bias added inside the contraction
+//   broadcast  O = softmax(scale2 Q A^T + B2) V_A + DWC(V): persistent blocks over runs of row tiles
+struct StreamPlan {
+    bool ok;
+    int splits;          // aggregation blocks per slab
+    int tiles_per_split; // 128-token tiles per aggregation block
+    int rows_b;          // grid rows per broadcast tile (rows_b * W <= 128 tokens)
+    int tiles_b;         // broadcast tiles per slab
+    int grid_b;          // broadcast blocks (persistent)
+    int halo_stages;     // ring depth of the depthwise window's V rows
+    int smem_b;          // dynamic shared memory of a broadcast block
+};
+struct StreamArgs {
+    const void *q, *k, *v, *a_user, *b1, *b2, *dwc_w;
+    void* out;
+    void *a_ws, *va_ws;        // [slabs][n][64] agents and agent features (element type)
+    void *a1s, *a2s;           // [slabs][n][64] agents times scale1 / scale2
+    void *b1c, *b2p;           // [heads][N][64] clamped, transposed, padded B1; [heads or 1][N][64] clamped, padded B2
+    float* partials;           // [slabs][splits][partial_floats(64, 64)]
+    unsigned* tickets;         // [slabs]
+    int* status;
+    int slabs, heads, H, W, n, p;
+    float scale1, scale2;
+    int sm_count;
+    StreamPlan plan;
+    alignas(64) CUtensorMap tm_k, tm_v, tm_b1, tm_q, tm_b2, tm_h, tm_a2, tm_va;
+};
+StreamPlan plan_stream(int dtype, int slabs, int H, int W, int d, int n_agents, bool pooled, int sm_count);
+// workspace beyond A and V_A: bytes of (a1s | a2s | b1c | b2p), each 256-byte aligned, in this order
+size_t stream_extra_bytes(int slabs, int heads, int N, int n_agents);
+bool stream_make_maps(StreamArgs* a);
+cudaError_t launch_stream(int dtype, const StreamArgs& a, cudaStream_t st);
+cudaError_t launch_stream_prep(int dtype, const StreamArgs& a, cudaStream_t st);
+cudaError_t launch_stream_aggregate(int dtype, const StreamArgs& a, cudaStream_t st);
+cudaError_t launch_stream_broadcast(int dtype, const StreamArgs& a, cudaStream_t st);
+
 // ------------------------------------------------------------------------------ backward pass
 // Tiling of the backward kernels: tiles of `tile` tokens, `chunks` blocks per slab, each block
 // walking `tiles_per_chunk` consecutive tiles; np = agents padded to a multiple of 32, plus 1.
