@@ -18,10 +18,12 @@
 //       store them back over the logits.  No maximum is taken on this path: a probability >= 2 shows in the
 //       top exponent bit of the packed pairs (one OR per pair); only then the reference moves up (true
 //       maximum of the tile plus a margin) and the thread rescales its accumulator row.
-// At the end the two token halves of a row meet in shared memory, the block writes one partial state, and
-// the slab's last block merges the partial states in a fixed order (bit-reproducible).
-// Every wait is bounded.  No TMA multicast, no clusters.
-#include "merge.cuh"
+// The blocks of a slab form a thread-block cluster.  At the end the two token halves of a row meet in shared
+// memory, and after a cluster barrier every block merges its share of the agent rows from the partial states
+// in its siblings' shared memory (plain distributed-shared-memory loads, fixed order of the blocks:
+// bit-reproducible) and writes those rows of V_A.  No partial state goes through global memory.
+// Every mbarrier wait is bounded; every block reaches both cluster barriers whatever happened before.
+// No TMA multicast.
 #include "stream_common.cuh"
 
 namespace aa {
@@ -84,51 +86,31 @@ __device__ __forceinline__ uint32_t row_probs(const uint32_t (&sa)[32], const ui
     return orr;
 }
 
-// Merge of the slab's partial states (m[64] in log2 units | l[64] | acc[64][64] each) into V_A, in the fixed
-// order of the parts; all loads of an output group are issued before the arithmetic (at most 8 parts).
-template <typename T>
-__device__ __forceinline__ void merge_parts(const float* base, int parts, int n, T* out, int tid, int nthreads) {
-    const size_t pf = partial_floats(64, 64);
-    for (int e = tid; e < n * 16; e += nthreads) {
-        const int r = e >> 4, c4 = e & 15;
-        float m[8], l[8];
-        float4 a[8];
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            m[q] = -INFINITY; l[q] = 0.f; a[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (q < parts) {
-                const float* pq = base + q * pf;
-                m[q] = __ldcg(pq + r);
-                l[q] = __ldcg(pq + 64 + r);
-                a[q] = __ldcg(reinterpret_cast<const float4*>(pq + 128 + (size_t)r * 64) + c4);
-            }
-        }
-        float mm = m[0];
-#pragma unroll
-        for (int q = 1; q < 8; ++q) mm = fmaxf(mm, m[q]);
-        const float bs = (mm == -INFINITY) ? 0.f : mm;
-        float den = 0.f;
-        float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            const float wq = exp2f(m[q] - bs);               // 0 for a part without tokens
-            den = fmaf(l[q], wq, den);
-            num.x = fmaf(a[q].x, wq, num.x); num.y = fmaf(a[q].y, wq, num.y);
-            num.z = fmaf(a[q].z, wq, num.z); num.w = fmaf(a[q].w, wq, num.w);
-        }
-        const float inv = 1.f / den;
-        uint2 o;
-        o.x = pack2<T>(num.x * inv, num.y * inv);
-        o.y = pack2<T>(num.z * inv, num.w * inv);
-        *(reinterpret_cast<uint2*>(out + (size_t)r * 64) + c4) = o;
-    }
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;\n" ::: "memory");
+}
+// shared-memory address of the same variable in block `rank` of the cluster
+__device__ __forceinline__ uint32_t cluster_map(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ float4 ld_cluster_f4(uint32_t addr) {
+    float4 v;
+    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ float2 ld_cluster_f2(uint32_t addr) {
+    float2 v;
+    asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr));
+    return v;
 }
 }  // namespace
 
 template <typename T>
 __global__ void __launch_bounds__(NT, 1) stream_aggregate_kernel(const __grid_constant__ StreamArgs p) {
     extern __shared__ unsigned char smem_raw[];
-    __shared__ int s_dead, s_flag;
+    __shared__ int s_dead;
     __shared__ uint32_t s_tmem;
     unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     constexpr int fmt = Elem<T>::kIsBf16 ? 1 : 0;
@@ -157,19 +139,29 @@ __global__ void __launch_bounds__(NT, 1) stream_aggregate_kernel(const __grid_co
     __syncthreads();
     tc_fence_after_sync();
     pp.tmem = s_tmem;
-    pdl_wait();              // scaled agents, prepared bias and cleared counters come from the preceding kernel
-
     const uint32_t ring = smem_u32(smem + OFF_RING);
-    const size_t pf = partial_floats(64, 64);
-    float* slab_parts = p.partials + (size_t)slab * p.plan.splits * pf;
+    pdl_launch_dependents();     // the broadcast kernel may set itself up on idle SMs; it waits for this grid to finish
 
     if (warp == 4) {
         // ------------------------------------------------------------------ producer
         if (lane == 0) {
             const uint32_t tx = (has_bias ? 3u : 2u) * kTile;
-            for (int i = 0; i < tiles; ++i) {
+            // K and V are inputs of the call: the first ring stages are requested before the wait for the
+            // preceding kernel, whose results (scaled agents, prepared bias) are only needed after it
+            const int first = min(tiles, STAGES);
+            for (int i = 0; i < first; ++i) {
+                const uint32_t bar = pipe_bar(pp, BAR_FULL + i), dst = ring + i * kStage;
+                mbar_arrive_expect_tx(bar, tx);
+                tma_load_3d(dst, &p.tm_k, 0, (t0 + i) * TK, slab, bar);
+                tma_load_3d(dst + kTile, &p.tm_v, 0, (t0 + i) * TK, slab, bar);
+            }
+            pdl_wait();
+            if (has_bias)
+                for (int i = 0; i < first; ++i)
+                    tma_load_3d(ring + i * kStage + 2 * kTile, &p.tm_b1, 0, (t0 + i) * TK, head, pipe_bar(pp, BAR_FULL + i));
+            for (int i = first; i < tiles; ++i) {
                 const int s = i % STAGES, c0 = (t0 + i) * TK;
-                if (i >= STAGES) wait_par(pp, BAR_EMPTY + s, (i / STAGES) - 1, kTimeoutRole);
+                wait_par(pp, BAR_EMPTY + s, (i / STAGES) - 1, kTimeoutRole);
                 const uint32_t bar = pipe_bar(pp, BAR_FULL + s), dst = ring + s * kStage;
                 mbar_arrive_expect_tx(bar, tx);
                 tma_load_3d(dst, &p.tm_k, 0, c0, slab, bar);
@@ -228,6 +220,7 @@ __global__ void __launch_bounds__(NT, 1) stream_aggregate_kernel(const __grid_co
         // ------------------------------------------------------------------ row warps
         const int r = tid & 63, h = tid >> 6;              // agent row (padded), token half
         const uint32_t lane_base = ((uint32_t)(32 * warp)) << 16;
+        pdl_wait();          // the scaled agents come from the preceding kernel
         {
             // this lane's row of the A operand: 64 channels of scale1 * A, then the identity row that picks
             // the agent's own bias (rows past n stay zero: their logits are 0 and their results unused)
@@ -345,28 +338,65 @@ __global__ void __launch_bounds__(NT, 1) stream_aggregate_kernel(const __grid_co
         }
         asm volatile("bar.sync 1, %0;\n" ::"n"(NROW) : "memory");
         if (h == 0) {
+            // this block's partial state of row r stays in shared memory: row, reference (log2 units), sum
             const float om = sX[64], ol = sX[65];
             const float mm = fmaxf(m_ref, om);
             const float bs = (mm == -INFINITY) ? 0.f : mm;
             const float wa = fast_exp2(m_ref - bs), wb = fast_exp2(om - bs);
-            float* part = slab_parts + (size_t)split * pf;
-            part[r] = mm;
-            part[64 + r] = l * wa + ol * wb;
-            float* pacc = part + 128 + (size_t)r * 64;
 #pragma unroll
             for (int k = 0; k < 16; ++k) {
                 const float4 xv = *reinterpret_cast<const float4*>(sX + 4 * k);
-                *reinterpret_cast<float4*>(pacc + 4 * k) =
+                *reinterpret_cast<float4*>(sX + 4 * k) =
                     make_float4(o[4 * k] * wa + xv.x * wb, o[4 * k + 1] * wa + xv.y * wb,
                                 o[4 * k + 2] * wa + xv.z * wb, o[4 * k + 3] * wa + xv.w * wb);
             }
+            sX[64] = mm; sX[65] = l * wa + ol * wb;
         }
     }
-    // the slab's last block merges the partial states, in the fixed order of the splits
+    // every block of the slab has its partial state in shared memory; each merges its share of the agent rows
     tc_fence_before_sync();
-    const bool last = arrive_is_last(p.tickets + slab, (unsigned)p.plan.splits, &s_flag);
-    if (last) merge_parts<T>(slab_parts, p.plan.splits, n, static_cast<T*>(p.va_ws) + (size_t)slab * n * 64, tid, NT);
-    __syncthreads();
+    cluster_sync_all();
+    {
+        const int splits = p.plan.splits;
+        const int rows_per = (n + splits - 1) / splits;
+        const int rb = split * rows_per, re = min(n, rb + rows_per);
+        const uint32_t sx0 = ring;                          // [64][68] floats at the start of the ring, in every block
+        T* va = static_cast<T*>(p.va_ws) + (size_t)slab * n * 64;
+        for (int e = tid; e < (re - rb) * 16; e += NT) {
+            const int r = rb + (e >> 4), c4 = e & 15;
+            float m[8], l[8];
+            float4 a[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                m[q] = -INFINITY; l[q] = 0.f; a[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (q < splits) {
+                    const uint32_t row = cluster_map(sx0 + (uint32_t)r * 272u, (uint32_t)q);
+                    const float2 ml = ld_cluster_f2(row + 256u);
+                    m[q] = ml.x; l[q] = ml.y;
+                    a[q] = ld_cluster_f4(row + 16u * c4);
+                }
+            }
+            float mm = m[0];
+#pragma unroll
+            for (int q = 1; q < 8; ++q) mm = fmaxf(mm, m[q]);
+            const float bs = (mm == -INFINITY) ? 0.f : mm;
+            float den = 0.f;
+            float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                const float wq = exp2f(m[q] - bs);           // 0 for a block without tokens
+                den = fmaf(l[q], wq, den);
+                num.x = fmaf(a[q].x, wq, num.x); num.y = fmaf(a[q].y, wq, num.y);
+                num.z = fmaf(a[q].z, wq, num.z); num.w = fmaf(a[q].w, wq, num.w);
+            }
+            const float inv = 1.f / den;
+            uint2 o2;
+            o2.x = pack2<T>(num.x * inv, num.y * inv);
+            o2.y = pack2<T>(num.z * inv, num.w * inv);
+            *(reinterpret_cast<uint2*>(va + (size_t)r * 64) + c4) = o2;
+        }
+    }
+    cluster_sync_all();            // no block leaves while a sibling may still read its shared memory
     if (warp == 0) tmem_dealloc<512>(pp.tmem);
 }
 
@@ -377,11 +407,15 @@ cudaError_t launch_stream_aggregate(int dtype, const StreamArgs& a, cudaStream_t
     cfg.blockDim = dim3(NT);
     cfg.dynamicSmemBytes = kSmemBytes;
     cfg.stream = st;
-    cudaLaunchAttribute at[1];
+    cudaLaunchAttribute at[2];
     at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     at[0].val.programmaticStreamSerializationAllowed = 1;
+    at[1].id = cudaLaunchAttributeClusterDimension;       // the blocks of a slab exchange their partial states
+    at[1].val.clusterDim.x = (unsigned)a.plan.splits;
+    at[1].val.clusterDim.y = 1;
+    at[1].val.clusterDim.z = 1;
     cfg.attrs = at;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     cudaError_t e;
     if (dtype == kBF16) {
         auto kern = stream_aggregate_kernel<__nv_bfloat16>;

@@ -100,6 +100,14 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
 }
 
+// 4-D tiled load of a [slab][y][x][64] view: box at (0, x, y, slab); coordinates outside the grid (x = -1, x = W,
+// y = -1, y = H) are zero-filled, which is the zero padding of the depthwise window.
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int c, int x, int y, int z, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];\n"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
+}
+
 // Programmatic dependent launch: a kernel launched with the attribute may start before its predecessor in
 // the stream has finished; it must pass pdl_wait() before it touches anything the predecessor writes.
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;\n" ::: "memory"); }
@@ -118,6 +126,20 @@ inline bool make_map_rows3d_u16(CUtensorMap* out, const void* base, uint64_t zs,
     return fn(out, CU_TENSOR_MAP_DATA_TYPE_UINT16, 3, const_cast<void*>(base), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
               CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Host: map of a dense [z][H][W][64] tensor of 16-bit elements with a box of 64 x box_w x box_h x 1, no swizzle.
+inline bool make_map_grid4d_u16(CUtensorMap* out, const void* base, uint64_t zs, uint64_t H, uint64_t W, uint32_t box_h, uint32_t box_w) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    if ((reinterpret_cast<uintptr_t>(base) & 15u) || box_h > 256 || box_w > 256 || box_h < 1 || box_w < 1) return false;
+    const cuuint64_t dims[4] = {64, W, H, zs};
+    const cuuint64_t strides[3] = {128, W * 128, H * W * 128};
+    const cuuint32_t box[4] = {64, box_w, box_h, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    return fn(out, CU_TENSOR_MAP_DATA_TYPE_UINT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 }  // namespace aa

@@ -16,14 +16,15 @@ namespace {
 constexpr int NT = 256;
 
 template <typename T>
-__global__ void __launch_bounds__(NT) stream_prep_kernel(const StreamArgs p, int pool_blocks) {
+__global__ void __launch_bounds__(NT) stream_prep_kernel(const StreamArgs p, int bias_blocks) {
     pdl_launch_dependents();          // the aggregation kernel may set itself up while this one runs
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int N = p.H * p.W, n = p.n;
     if (blockIdx.x == 0)
         for (int e = tid; e < p.slabs; e += NT) p.tickets[e] = 0u;
-    if ((int)blockIdx.x < pool_blocks) {
-        const long long wi = (long long)blockIdx.x * (NT / 32) + warp;
+    // the bias blocks come first in the grid: they are few, latency-bound, and would otherwise form the kernel's tail
+    if ((int)blockIdx.x >= bias_blocks) {
+        const long long wi = (long long)(blockIdx.x - bias_blocks) * (NT / 32) + warp;
         if (wi >= (long long)p.slabs * n) return;
         const int slab = (int)(wi / n), a = (int)(wi - (long long)slab * n);
         const int c = lane & 7, ts = lane >> 3;
@@ -36,27 +37,33 @@ __global__ void __launch_bounds__(NT) stream_prep_kernel(const StreamArgs p, int
         } else {
             const int win_h = p.H / p.p, win_w = p.W / p.p, cnt = win_h * win_w;
             const int y0 = (a / p.p) * win_h, x0 = (a % p.p) * win_w;
-            const T* gq = static_cast<const T*>(p.q) + (size_t)slab * N * 64;
+            // lane (c, ts) walks the window's tokens ts, ts + 4, ... in row-major order; (wy, wx) is kept
+            // incrementally, so the sixteen loads of a batch cost an add and a compare each
+            const uint4* gq = reinterpret_cast<const uint4*>(static_cast<const T*>(p.q) + ((size_t)slab * N + (size_t)y0 * p.W + x0) * 64) + c;
             inv = 1.f / (float)cnt;
+            int wy = ts / win_w, wx = ts - wy * win_w;
+            float2 acc2[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) acc2[k] = make_float2(0.f, 0.f);
             for (int ib = ts; ib < cnt; ib += 64) {
                 uint4 raw[16];
 #pragma unroll
                 for (int u = 0; u < 16; ++u) {
-                    const int i = ib + 4 * u;
                     raw[u] = make_uint4(0u, 0u, 0u, 0u);
-                    if (i < cnt) {
-                        const int wy = i / win_w, wx = i - wy * win_w;
-                        raw[u] = __ldg(reinterpret_cast<const uint4*>(gq + ((size_t)(y0 + wy) * p.W + (x0 + wx)) * 64) + c);
-                    }
+                    if (ib + 4 * u < cnt) raw[u] = __ldg(gq + ((size_t)wy * p.W + wx) * 8);
+                    wx += 4;
+                    while (wx >= win_w) { wx -= win_w; ++wy; }
                 }
 #pragma unroll
                 for (int u = 0; u < 16; ++u) {
-                    float f[8];
-                    unpack16<T>(raw[u], f);
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) acc[k] += f[k];
+                    acc2[0] = fadd2(acc2[0], unpack2<T>(raw[u].x));
+                    acc2[1] = fadd2(acc2[1], unpack2<T>(raw[u].y));
+                    acc2[2] = fadd2(acc2[2], unpack2<T>(raw[u].z));
+                    acc2[3] = fadd2(acc2[3], unpack2<T>(raw[u].w));
                 }
             }
+#pragma unroll
+            for (int k = 0; k < 4; ++k) { acc[2 * k] = acc2[k].x; acc[2 * k + 1] = acc2[k].y; }
         }
 #pragma unroll
         for (int o = 8; o < 32; o <<= 1) {
@@ -75,8 +82,7 @@ __global__ void __launch_bounds__(NT) stream_prep_kernel(const StreamArgs p, int
         return;
     }
     // ---- bias blocks
-    const long long nb = gridDim.x - pool_blocks;
-    const long long t0 = ((long long)blockIdx.x - pool_blocks) * NT + tid, step = nb * NT;
+    const long long t0 = (long long)blockIdx.x * NT + tid, step = (long long)bias_blocks * NT;
     if (p.b1) {
         // B1 [heads][n][N] -> transposed, padded [heads][N][64] (pad columns zero): a K-major operand tile per 128 tokens
         const long long vecs = (long long)p.heads * N * 8;
@@ -122,12 +128,12 @@ cudaError_t launch_stream_prep(int dtype, const StreamArgs& a, cudaStream_t st) 
     const int pool_blocks = (int)((windows + NT / 32 - 1) / (NT / 32));
     const long long N = (long long)a.H * a.W;
     const long long items = (a.b1 ? (long long)a.heads * N * 8 : 0) + (long long)(a.b2 ? a.heads : 1) * N * 8;
-    long long bias_blocks = (items + NT * 4 - 1) / (NT * 4);
-    if (bias_blocks > 4LL * a.sm_count) bias_blocks = 4LL * a.sm_count;
+    long long bias_blocks = (items + NT - 1) / NT;            // one output vector per thread where the grid allows it
+    if (bias_blocks > 8LL * a.sm_count) bias_blocks = 8LL * a.sm_count;
     if (bias_blocks < 1) bias_blocks = 1;
     const unsigned grid = (unsigned)(pool_blocks + bias_blocks);
-    if (dtype == kBF16) stream_prep_kernel<__nv_bfloat16><<<grid, NT, 0, st>>>(a, pool_blocks);
-    else if (dtype == kF16) stream_prep_kernel<__half><<<grid, NT, 0, st>>>(a, pool_blocks);
+    if (dtype == kBF16) stream_prep_kernel<__nv_bfloat16><<<grid, NT, 0, st>>>(a, (int)bias_blocks);
+    else if (dtype == kF16) stream_prep_kernel<__half><<<grid, NT, 0, st>>>(a, (int)bias_blocks);
     else return cudaErrorInvalidValue;
     return cudaGetLastError();
 }
