@@ -395,6 +395,7 @@ static int forward_impl(agent_attn_handle* h, const void* Q, const void* K, cons
             sa.a1s = ws + w.extra_off; sa.a2s = ws + w.extra_off + av;
             sa.b1c = ws + w.extra_off + 2 * av;
             sa.b2p = ws + w.extra_off + 2 * av + align_up((size_t)h->cfg.heads * N * 64 * 2, 256);
+            sa.wt = ws + w.extra_off + 2 * av + 2 * align_up((size_t)h->cfg.heads * N * 64 * 2, 256);
             sa.partials = reinterpret_cast<float*>(ws + w.part_off);
             sa.tickets = reinterpret_cast<unsigned*>(ws + w.ticket_off);
             sa.status = h->d_status;

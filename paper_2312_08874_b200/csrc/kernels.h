@@ -166,6 +166,7 @@ struct StreamArgs {
     void *a_ws, *va_ws;        // [slabs][n][64] agents and agent features (element type)
     void *a1s, *a2s;           // [slabs][n][64] agents times scale1 / scale2
     void *b1c, *b2p;           // [heads][N][64] clamped, transposed, padded B1; [heads or 1][N][64] clamped, padded B2
+    void* wt;                  // [heads][9][16][128 B] diagonal slices of the depthwise filter, as swizzled operand tiles
     float* partials;           // [slabs][splits][partial_floats(64, 64)]
     unsigned* tickets;         // [slabs]
     int* status;

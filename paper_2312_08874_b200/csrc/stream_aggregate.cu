@@ -6,7 +6,8 @@
 // agent rows are stacked twice so that all 128 tensor-memory lanes carry a row: lane r + 64 h owns agent r
 // and the token half h of every tile, with its own reference maximum, row sum and accumulator row.
 //   warp 4 "producer":  one lane issues every TMA copy, ahead of the others through full/empty mbarriers.
-//   warp 5 "MMA issuer": one lane.  S = [A | I] [K | B1^T]^T: the agents (times scale1) and an identity block
+//   warps 5, 6 "MMA issuers": one lane each, one for the logits and one for the products, so that neither
+//       instruction stream waits behind the other's barriers.  S = [A | I] [K | B1^T]^T: the agents (times scale1) and an identity block
 //       sit in tensor memory as the A operand, so the bias is added inside the contraction and the logits
 //       arrive complete, in natural units; eight instructions of 128 columns per tile, one tile ahead.  Then
 //       D += P V with the probabilities read from tensor memory too.  (An instruction of this kind takes about
@@ -32,7 +33,7 @@ namespace {
 constexpr int TK = 128;                // tokens per tile
 constexpr int STAGES = 4;
 constexpr int NROW = 128;              // row-warp threads
-constexpr int NT = NROW + 64;          // + producer warp + MMA issuer warp
+constexpr int NT = NROW + 96;          // + producer warp + two MMA issuer warps (logits; products)
 constexpr int kTile = TK * 128;        // swizzled [128][64] tile of 16-bit elements
 constexpr int kStage = 3 * kTile;      // K | V | B1^T
 constexpr float kMargin = 4.f;         // a new reference sits this far (log2 units) above the tile's maximum
@@ -51,11 +52,12 @@ constexpr int BAR_S_FULL = 8;     // [2]       commit         row warps
 constexpr int BAR_P_FULL = 10;    // [2]       row threads    MMA issuer
 constexpr int BAR_PV = 12;        // [2]       commit         row warps (only when a reference moves, and at the end)
 constexpr int BAR_A = 14;         //           row threads    MMA issuer      the agent operand is in tensor memory
-constexpr int kBars = 15;
+constexpr int BAR_S_EMPTY = 15;   // [2]       row threads    MMA issuer      the logits have been read
+constexpr int kBars = 17;
 
-// tensor memory columns: logits 2 x 128 (the probabilities overwrite the first 64 of their buffer),
-// accumulator 64, agent operand 32 (64 channels) + 32 (identity, 64 agents)
-constexpr uint32_t TM_S = 0, TM_D = 256, TM_A = 320;
+// tensor memory columns: logits 2 x 128, probabilities 2 x 64 (16-bit pairs), accumulator 64,
+// agent operand 32 (64 channels) + 32 (identity, 64 agents)
+constexpr uint32_t TM_S = 0, TM_P = 256, TM_D = 384, TM_A = 448;
 
 // Probabilities of one thread's 64 logits relative to the reference (nb = minus the reference, log2 units):
 // packed pairs in pk, their fp32 sum in `sum`; returns the OR of the pairs.  Columns >= valid weigh nothing.
@@ -131,7 +133,7 @@ __global__ void __launch_bounds__(NT, 1) stream_aggregate_kernel(const __grid_co
     if (tid == 0) {
         s_dead = 0;
         for (int i = 0; i < kBars; ++i)
-            mbar_init(pp.bars + 8 * i, ((i >= BAR_P_FULL && i < BAR_PV) || i == BAR_A) ? (uint32_t)NROW : 1u);
+            mbar_init(pp.bars + 8 * i, ((i >= BAR_P_FULL && i < BAR_PV) || i >= BAR_A) ? (uint32_t)NROW : 1u);
         mbar_fence_init();
     }
     if (warp == 0) tmem_alloc<512>(smem_u32(&s_tmem));
@@ -161,7 +163,7 @@ __global__ void __launch_bounds__(NT, 1) stream_aggregate_kernel(const __grid_co
                     tma_load_3d(ring + i * kStage + 2 * kTile, &p.tm_b1, 0, (t0 + i) * TK, head, pipe_bar(pp, BAR_FULL + i));
             for (int i = first; i < tiles; ++i) {
                 const int s = i % STAGES, c0 = (t0 + i) * TK;
-                wait_par(pp, BAR_EMPTY + s, (i / STAGES) - 1, kTimeoutRole);
+                wait_spin(pp, BAR_EMPTY + s, (i / STAGES) - 1, kTimeoutRole);
                 const uint32_t bar = pipe_bar(pp, BAR_FULL + s), dst = ring + s * kStage;
                 mbar_arrive_expect_tx(bar, tx);
                 tma_load_3d(dst, &p.tm_k, 0, c0, slab, bar);
@@ -171,46 +173,61 @@ __global__ void __launch_bounds__(NT, 1) stream_aggregate_kernel(const __grid_co
         }
         __syncwarp();
     } else if (warp == 5) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            const uint32_t idS = umma_idesc(fmt, 128, 128, 0), idPV = umma_idesc(fmt, 128, 64, 1);
+        // ------------------------------------------------------------------ MMA issuer: logits, up to two tiles ahead
+        // (the whole warp runs the loop; one elected lane issues)
+        {
+            const uint32_t idS = umma_idesc(fmt, 128, 128, 0);
             const uint64_t dRing = umma_desc_sw128(ring);
-            const uint32_t tA = pp.tmem + TM_A, tD = pp.tmem + TM_D, tS = pp.tmem + TM_S;
-            // descriptor start addresses count 16-byte units: + 2 per K-step of a K-major operand (32 bytes),
-            // + 128 per K-step of an MN-major operand (16 rows of 128 bytes).  `s` and `b` are compile-time
-            // constants at every call below (the tile loop is unrolled over the ring).
-            auto issue_S = [&](int i, int s, int b) {
-                wait_par(pp, BAR_FULL + s, i / STAGES, kTimeoutTile);
-                tc_fence_after_sync();
-                const uint64_t dK = dRing + (uint64_t)(s * (kStage >> 4));
-                const uint32_t dd = tS + 128 * b;
-                umma_ts(dd, tA, dK, idS, 0u);
-#pragma unroll
-                for (int k = 1; k < 4; ++k) umma_ts(dd, tA + 8 * k, dK + 2 * k, idS, 1u);
-                if (has_bias) {
-                    const uint64_t dB = dK + (uint64_t)(2 * kTile >> 4);
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) umma_ts(dd, tA + 32 + 8 * k, dB + 2 * k, idS, 1u);
-                }
-                umma_commit(pipe_bar(pp, BAR_S_FULL + b));
-            };
-            wait_par(pp, BAR_A, 0, kTimeoutLoads);
-            issue_S(0, 0, 0);
+            const uint32_t tA = pp.tmem + TM_A, tS = pp.tmem + TM_S;
+            // descriptor start addresses count 16-byte units: + 2 per K-step of a K-major operand (32 bytes).
+            // `u` is a compile-time constant (the tile loop is unrolled over the ring).
+            wait_spin(pp, BAR_A, 0, kTimeoutLoads);
             for (int i0 = 0; i0 < tiles; i0 += STAGES) {
 #pragma unroll
                 for (int u = 0; u < STAGES; ++u) {
                     const int i = i0 + u;
                     if (i < tiles) {
-                        if (i + 1 < tiles) issue_S(i + 1, (u + 1) % STAGES, (u + 1) & 1);
-                        wait_par(pp, BAR_P_FULL + (u & 1), i >> 1, kTimeoutRole);
+                        // the logits buffer is free once the row warps have read tile i - 2 out of it
+                        if (i >= 2) wait_spin(pp, BAR_S_EMPTY + (u & 1), (i >> 1) - 1, kTimeoutRole);
+                        wait_spin(pp, BAR_FULL + u, i / STAGES, kTimeoutTile);
+                        tc_fence_after_sync();
+                        const uint64_t dK = dRing + (uint64_t)(u * (kStage >> 4));
+                        const uint32_t dd = tS + 128 * (u & 1);
+                        umma_ts_w(dd, tA, dK, idS, 0u);
+#pragma unroll
+                        for (int k = 1; k < 4; ++k) umma_ts_w(dd, tA + 8 * k, dK + 2 * k, idS, 1u);
+                        if (has_bias) {
+                            const uint64_t dB = dK + (uint64_t)(2 * kTile >> 4);
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) umma_ts_w(dd, tA + 32 + 8 * k, dB + 2 * k, idS, 1u);
+                        }
+                        umma_commit_w(pipe_bar(pp, BAR_S_FULL + (u & 1)));
+                    }
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 6) {
+        // ------------------------------------------------------------------ MMA issuer: products
+        {
+            const uint32_t idPV = umma_idesc(fmt, 128, 64, 1);
+            const uint64_t dRing = umma_desc_sw128(ring);
+            const uint32_t tD = pp.tmem + TM_D, tPb = pp.tmem + TM_P;
+            // + 128 per K-step of an MN-major operand (16 rows of 128 bytes)
+            for (int i0 = 0; i0 < tiles; i0 += STAGES) {
+#pragma unroll
+                for (int u = 0; u < STAGES; ++u) {
+                    const int i = i0 + u;
+                    if (i < tiles) {
+                        wait_spin(pp, BAR_P_FULL + (u & 1), i >> 1, kTimeoutRole);
                         tc_fence_after_sync();
                         const uint64_t dV = dRing + (uint64_t)(u * (kStage >> 4) + (kTile >> 4));
-                        const uint32_t tP = tS + 128 * (u & 1);
-                        umma_ts(tD, tP, dV, idPV, i > 0 ? 1u : 0u);
+                        const uint32_t tP = tPb + 64 * (u & 1);
+                        umma_ts_w(tD, tP, dV, idPV, i > 0 ? 1u : 0u);
 #pragma unroll
-                        for (int k = 1; k < 8; ++k) umma_ts(tD, tP + 8 * k, dV + 128 * k, idPV, 1u);
-                        umma_commit(pipe_bar(pp, BAR_EMPTY + u));
-                        umma_commit(pipe_bar(pp, BAR_PV + (u & 1)));
+                        for (int k = 1; k < 8; ++k) umma_ts_w(tD, tP + 8 * k, dV + 128 * k, idPV, 1u);
+                        umma_commit_w(pipe_bar(pp, BAR_EMPTY + u));
+                        umma_commit_w(pipe_bar(pp, BAR_PV + (u & 1)));
                     }
                 }
             }
@@ -240,6 +257,11 @@ __global__ void __launch_bounds__(NT, 1) stream_aggregate_kernel(const __grid_co
 #pragma unroll
             for (int j = 0; j < 32; ++j) ra[j] = (j == (r >> 1)) ? one : 0u;
             tmem_st32(pp.tmem + TM_A + 32 + lane_base, ra);
+            // the other token half's share of both probability operands stays zero for the whole kernel
+#pragma unroll
+            for (int j = 0; j < 32; ++j) ra[j] = 0u;
+            tmem_st32(pp.tmem + TM_P + 32 * (1 - h) + lane_base, ra);
+            tmem_st32(pp.tmem + TM_P + 64 + 32 * (1 - h) + lane_base, ra);
             tmem_st_wait();
             tc_fence_before_sync();
             pipe_arrive(pp, BAR_A);
@@ -247,7 +269,7 @@ __global__ void __launch_bounds__(NT, 1) stream_aggregate_kernel(const __grid_co
         const uint32_t tD = pp.tmem + TM_D + lane_base;
         float nb = 0.f;                                    // minus the row's reference, log2 units
         float l = 0.f;                                     // row sum of the probabilities, relative to the reference
-        bool started = false;
+        bool started = false;                              // the accumulator row holds something
         for (int i = 0; i < tiles; ++i) {
             const int b = i & 1;
             const int valid = max(0, min(64, N - ((t0 + i) * TK + 64 * h)));      // tokens of this half: uniform per warp
@@ -260,10 +282,13 @@ __global__ void __launch_bounds__(NT, 1) stream_aggregate_kernel(const __grid_co
                 tmem_ld32(tS + 64 * h, sa);
                 tmem_ld32(tS + 64 * h + 32, sb);
                 tmem_ld_wait();
-                float sum;
-                const uint32_t orr = valid == 64 ? row_probs<T, false>(sa, sb, nb, valid, pk, sum)
-                                                 : row_probs<T, true>(sa, sb, nb, valid, pk, sum);
-                const bool trig = !started || (orr & kPairGe2) != 0u;
+                tc_fence_before_sync();
+                pipe_arrive(pp, BAR_S_EMPTY + b);          // the next logits may land in this buffer
+                float sum = 0.f;
+                uint32_t orr = kPairGe2;
+                if (started)
+                    orr = valid == 64 ? row_probs<T, false>(sa, sb, nb, valid, pk, sum) : row_probs<T, true>(sa, sb, nb, valid, pk, sum);
+                const bool trig = (orr & kPairGe2) != 0u;
                 if (__any_sync(0xffffffffu, trig)) {       // first tile, or rare: some row's logits outgrew its reference
                     float mx = -INFINITY;
 #pragma unroll
@@ -301,14 +326,14 @@ __global__ void __launch_bounds__(NT, 1) stream_aggregate_kernel(const __grid_co
                 l += sum;
                 started = true;
             } else {
+                tc_fence_before_sync();
+                pipe_arrive(pp, BAR_S_EMPTY + b);
 #pragma unroll
                 for (int j = 0; j < 32; ++j) pk[j] = 0u;
             }
-            // probabilities over this half's logits, zeros over the other half's share of the operand
-            tmem_st32(tS + 32 * h, pk);
-#pragma unroll
-            for (int j = 0; j < 32; ++j) pk[j] = 0u;
-            tmem_st32(tS + 32 * (1 - h), pk);
+            // the probability operand of this buffer is free once the product of tile i - 2 has read it
+            if (i >= 2) { wait_par(pp, BAR_PV + b, (i >> 1) - 1, kTimeoutTile); tc_fence_after_sync(); }
+            tmem_st32(pp.tmem + TM_P + 64 * b + 32 * h + lane_base, pk);
             tmem_st_wait();
             tc_fence_before_sync();
             pipe_arrive(pp, BAR_P_FULL + b);

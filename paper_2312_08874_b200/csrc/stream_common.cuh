@@ -18,6 +18,33 @@ __device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64
         ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
 
+// The same instructions for an issuing WARP in uniform control flow: every lane executes the surrounding code
+// (waits, address arithmetic), so that the compiler can keep descriptors and addresses in uniform registers, and
+// one elected lane (the same one every time) issues.  With the issue inside an `if (lane == 0)` region every
+// operand takes a detour through per-thread registers, which costs more than the instruction itself.
+__device__ __forceinline__ void umma_ts_w(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "elect.sync _|q, 0xffffffff;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}\n"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_ss_w(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "elect.sync _|q, 0xffffffff;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}\n"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit_w(uint32_t bar) {
+    asm volatile(
+        "{\n\t.reg .pred q;\n\t"
+        "elect.sync _|q, 0xffffffff;\n\t"
+        "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}\n" ::"r"(bar) : "memory");
+}
+
 // One fp32 column of this thread's tensor-memory row.
 __device__ __forceinline__ uint32_t tmem_ld1(uint32_t taddr) {
     uint32_t r;
@@ -92,6 +119,18 @@ __device__ __forceinline__ void wait_par(Pipe& pp, int i, uint32_t parity, int c
     if (pp.status) atomicCAS(pp.status, 0, code);
 }
 
+// Spinning wait of a single-lane role on the critical path (no back-off: a hand-off costs tens of cycles);
+// bounded like every other wait.
+__device__ __forceinline__ void wait_spin(Pipe& pp, int i, uint32_t parity, int code) {
+    const uint32_t bar = pipe_bar(pp, i);
+    for (unsigned tries = 0; tries < (1u << 24); ++tries) {
+        if (mbar_try_wait(bar, parity & 1u)) return;
+        if ((tries & 1023u) == 1023u && pipe_dead(pp)) return;
+    }
+    *reinterpret_cast<volatile int*>(pp.dead) = 1;
+    if (pp.status) atomicCAS(pp.status, 0, code);
+}
+
 // 3-D tiled load: box at (0, row, z) of a map whose dimensions are (64 channels or columns, rows, slabs or
 // heads).  Rows outside [0, rows) are zero-filled, so a tile never runs into the next slab.
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
@@ -128,8 +167,8 @@ inline bool make_map_rows3d_u16(CUtensorMap* out, const void* base, uint64_t zs,
               CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Host: map of a dense [z][H][W][64] tensor of 16-bit elements with a box of 64 x box_w x box_h x 1, no swizzle.
-inline bool make_map_grid4d_u16(CUtensorMap* out, const void* base, uint64_t zs, uint64_t H, uint64_t W, uint32_t box_h, uint32_t box_w) {
+// Host: map of a dense [z][H][W][64] tensor of 16-bit elements with a box of 64 x box_w x box_h x 1, 128-byte swizzle or none.
+inline bool make_map_grid4d_u16(CUtensorMap* out, const void* base, uint64_t zs, uint64_t H, uint64_t W, uint32_t box_h, uint32_t box_w, bool swizzle) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
     if ((reinterpret_cast<uintptr_t>(base) & 15u) || box_h > 256 || box_w > 256 || box_h < 1 || box_w < 1) return false;
@@ -138,8 +177,8 @@ inline bool make_map_grid4d_u16(CUtensorMap* out, const void* base, uint64_t zs,
     const cuuint32_t box[4] = {64, box_w, box_h, 1};
     const cuuint32_t estr[4] = {1, 1, 1, 1};
     return fn(out, CU_TENSOR_MAP_DATA_TYPE_UINT16, 4, const_cast<void*>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+              CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 }  // namespace aa

@@ -7,6 +7,8 @@
 //     and padded to 64 columns with a large negative value.  The attention kernels add the bias inside the
 //     tensor-core contraction (a product with an identity block), where an infinite entry would turn 0 * inf into NaN for every other agent; and the pad
 //     columns make the agents past n drop out of the broadcast softmax without any masking instructions.
+//   * the depthwise filter as diagonal operand slices: the broadcast kernel evaluates the 3x3 term on the tensor
+//     core as nine products of a shifted V tile with diag(w[:, tap]).
 //   * the arrival counters of the aggregation are cleared.
 #include "stream_common.cuh"
 
@@ -99,6 +101,20 @@ __global__ void __launch_bounds__(NT) stream_prep_kernel(const StreamArgs p, int
                 f[k] = col < n ? fminf(fmaxf(Elem<T>::to_f32(src[((size_t)head * n + col) * N + tok]), -Pair<T>::kBig), Pair<T>::kBig) : 0.f;
             }
             dst[e] = pack16<T>(f);
+        }
+    }
+    if (p.dwc_w) {
+        // depthwise filter -> per tap a [16][64] K-major operand tile (128-byte rows, 128-byte swizzle) holding four
+        // diagonal 16 x 16 slices: row j, column 16 g + k is w[16 g + j][tap] where j == k, else 0
+        const long long elems = (long long)p.heads * 9 * 16 * 64;
+        const T* src = static_cast<const T*>(p.dwc_w);
+        unsigned char* dst = static_cast<unsigned char*>(p.wt);
+        for (long long e = t0; e < elems; e += step) {
+            const int col = (int)(e & 63), j = (int)((e >> 6) & 15);
+            const int ht = (int)(e >> 10), head = ht / 9, tap = ht - head * 9;
+            const int g = col >> 4, k = col & 15;
+            const T v = (j == k) ? src[((size_t)head * 64 + 16 * g + j) * 9 + tap] : Elem<T>::from_f32(0.f);
+            *reinterpret_cast<T*>(dst + (size_t)ht * 2048 + j * 128 + ((((col >> 3) ^ j) & 7) << 4) + (col & 7) * 2) = v;
         }
     }
     {
