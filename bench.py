@@ -30,20 +30,38 @@ from paper_2312_08874_b200.workloads import TORCH_DTYPE  # noqa: E402
 METRIC = "agent-attention fwd tokens/s and % of HBM roofline at N=3136,n=49,d=64"
 UNIT = "tokens/s"
 DEFAULT_WORKLOAD = "cfg3_pvt_bf16"
-L2_BYTES = 126 * 1024 * 1024
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu captures
-# summarised under profiles/ (None where the kernel has changed since its counters were taken)
-NCU_TRAFFIC = {("cfg3_pvt_bf16", "fused_kernel"): 102.76e6, ("cfg5a_hires_bf16", "broadcast_dwc"): 159.54e6}
+# dram__bytes_read.sum + dram__bytes_write.sum per forward pass of the streaming path (three launches), from the ncu
+# capture summarised under profiles/, with the digest of the kernel sources it was taken from: the figure is
+# reported only while those sources are unchanged
+NCU_TRAFFIC = {"cfg3_pvt_bf16": {"bytes": None, "sources_sha256": None}}
+TRAFFIC_SOURCES = ("stream_prep.cu", "stream_aggregate.cu", "stream_broadcast.cu", "stream_common.cuh")
+
+
+def kernel_sources_digest() -> str:
+    import hashlib
+    h = hashlib.sha256()
+    for f in TRAFFIC_SOURCES:
+        with open(os.path.join(ROOT, "paper_2312_08874_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def traffic_of(name: str):
+    t = NCU_TRAFFIC.get(name)
+    if not t or t["bytes"] is None or t["sources_sha256"] != kernel_sources_digest():
+        return None
+    return t["bytes"]
 
 
 def measured_peaks():
-    """(HBM GB/s, source) from the generated peaks file, else the machine's fallback figure."""
+    """(HBM GB/s, sustained bf16 TFLOP/s, source) from the generated peaks file, else the machine's fallback figures."""
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
         with open(path) as f:
-            return float(json.load(f)["hbm_gbs"]), "measured"
+            j = json.load(f)
+        return float(j["hbm_gbs"]), float(j.get("bf16_tflops_sustained", 1400.0)), "measured"
     except Exception:
-        return 6650.0, "fallback"
+        return 6650.0, 1400.0, "fallback"
 
 
 class ClockSampler(threading.Thread):
@@ -116,33 +134,40 @@ def oracle_inputs(w):
     return {k: (None if v is None else v.double().numpy()) for k, v in inp.items()}
 
 
+def oracle_baseline(w, passes: int, warmup: int):
+    """The oracle as it stands on the host cores, the same way for the GPU arm's `cpu_baseline` and for
+    `--impl reference`: one pass = the forward pass over a bounded sample of the workload (as many whole batch
+    entries as there are host threads, one slab per thread); the value is sample tokens / mean pass time."""
+    from oracle import agent_attention_oracle as orc
+    threads = orc.max_threads()
+    sample_batch = max(1, min(w.batch, threads // max(1, w.heads)))
+    ws = w.scaled(batch=sample_batch)
+    inp = oracle_inputs(ws)
+    for _ in range(warmup):
+        oracle_sample_run(ws, inp, threads)
+    t0 = time.perf_counter()
+    used = 1
+    for _ in range(passes):
+        _, used = oracle_sample_run(ws, inp, threads)
+    total = time.perf_counter() - t0
+    sample = f"{ws.batch} of {w.batch} batch entries ({ws.slabs} slabs) of {w.name} per pass, mean of {passes} passes"
+    return {"value": passes * ws.batch * ws.tokens / total, "unit": UNIT, "cores": used, "kind": "oracle",
+            "sample": sample, "ms_per_pass": 1e3 * total / passes}
+
+
 def run_reference(args, w):
     """The oracle as it stands on the host cores; each step is one pass over a bounded sample."""
     rank, _, world = pdist.env_rank()
     if rank != 0:
         return
-    from oracle import agent_attention_oracle as orc
-    threads = orc.max_threads()
-    # sample: as many whole batch entries as there are host threads, capped at the workload's batch
-    sample_batch = max(1, min(w.batch, threads // max(1, w.heads)))
-    ws = w.scaled(batch=sample_batch)
-    inp = oracle_inputs(ws)
-    for _ in range(args.warmup):
-        oracle_sample_run(ws, inp, threads)
-    t0 = time.perf_counter()
-    used = 1
-    for _ in range(args.steps):
-        _, used = oracle_sample_run(ws, inp, threads)
-    total = time.perf_counter() - t0
-    value = args.steps * ws.batch * ws.tokens / total
-    sample = f"{ws.batch} of {w.batch} batch entries ({ws.slabs} slabs) of {w.name} per step"
+    base = oracle_baseline(w, passes=args.steps, warmup=min(args.warmup, 3))
     print(json.dumps({
-        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
+        "impl": "reference", "metric": METRIC, "value": base["value"], "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": base["ms_per_pass"],
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "sample": sample},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": used, "kind": "oracle", "sample": sample},
-        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "config": {"workload": w.name, "sample": base["sample"]},
+        "cpu_baseline": {k: base[k] for k in ("value", "unit", "cores", "kind", "sample")},
+        "e2e": {"value": base["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }))
 
@@ -199,7 +224,7 @@ def run_backward(args, w, mod, sets, rank, local_rank, world):
     tfl = backward_flops(w) / (ms_step * 1e-3) / 1e12
     set_bytes = sum(t.numel() * t.element_size() for t in list(sets[0].values()) + list(g.values()) + [go]
                     if t is not None) - sets[0]["out"].numel() * sets[0]["out"].element_size()
-    hbm_peak, peak_src = measured_peaks()
+    hbm_peak, _, peak_src = measured_peaks()
     gbs = set_bytes / (ms_step * 1e-3) / 1e9
     tensor_path = w.dtype in ("bf16", "f16") and w.agents <= 64 and w.head_dim == 64
     if tensor_path:
@@ -227,14 +252,81 @@ def run_backward(args, w, mod, sets, rank, local_rank, world):
         }))
 
 
+def make_sets(w, dev, n_sets, rank, layout="dense"):
+    """`n_sets` device-resident buffer sets of the workload (distinct contents, same distribution)."""
+    dt = TORCH_DTYPE[w.dtype]
+    host = make_inputs(w, seed=w.seed + 1000 * rank)
+    sets = []
+    for s in range(n_sets):
+        g = torch.Generator(device="cpu").manual_seed(17 + s)
+        roll = int(torch.randint(1, w.tokens, (1,), generator=g))
+        d = {k: (None if v is None else v.to(dev)) for k, v in host.items()}
+        if s:  # a roll along the token axis
+            for k in ("q", "k", "v"):
+                d[k] = torch.roll(d[k], roll, dims=2).contiguous()
+        d["out"] = torch.empty_like(d["q"])
+        if layout != "dense":      # the same values behind token-major storage; views keep the [B,h,N,d] shape
+            if layout == "qkv":
+                packed = torch.stack([d[k].permute(0, 2, 1, 3) for k in ("q", "k", "v")], dim=2).contiguous()
+                for j, k in enumerate(("q", "k", "v")):
+                    d[k] = packed[:, :, j].permute(0, 2, 1, 3)
+            else:
+                for k in ("q", "k", "v"):
+                    d[k] = d[k].permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+            d["out"] = torch.empty((w.batch, w.tokens, w.heads, w.head_dim), dtype=dt, device=dev).permute(0, 2, 1, 3)
+        sets.append(d)
+    return host, sets
+
+
+def n_sets_for(w, l2_bytes):
+    """Rotating buffer sets: together more than 4x the L2, so no step re-reads a resident set."""
+    return max(2, -(-4 * l2_bytes // w.algorithmic_bytes()))
+
+
+def time_forward(mod, w, sets, ws, stream, steps, repeats, layout="dense", min_seconds=0.0, max_repeats=400):
+    """`repeats` timed regions of exactly `steps` forward calls each, between CUDA events on the launching stream
+    (more repeats until `min_seconds` of device time are covered).  Returns the per-step times in ms, one per repeat."""
+    fwd = mod.forward if layout == "dense" else mod.forward_strided
+
+    def step(i):
+        d = sets[i % len(sets)]
+        fwd(d["q"], d["k"], d["v"], w.grid_h, w.grid_w, w.agents, b1=d["b1"], b2=d["b2"],
+            dwc_weight=d["dwc"], out=d["out"], workspace=ws, stream=stream)
+
+    times, i, spent = [], 0, 0.0
+    while len(times) < repeats or (spent < min_seconds and len(times) < max_repeats):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            step(i)
+            i += 1
+        e1.record(stream)
+        e1.synchronize()
+        ms = e0.elapsed_time(e1)
+        times.append(ms / steps)
+        spent += ms * 1e-3
+    return times
+
+
+def bound_of(w, ms_step, hbm_peak, tensor_peak):
+    """Slower of (algorithmic bytes at the HBM peak) and (algorithmic flops at the sustained bf16 tensor peak)."""
+    t_hbm = w.algorithmic_bytes() / (hbm_peak * 1e9)
+    t_tensor = flops_of(w) / (tensor_peak * 1e12)
+    t_bound = max(t_hbm, t_tensor)
+    return {"bound": "hbm" if t_hbm >= t_tensor else "tensor", "t_hbm_us": 1e6 * t_hbm, "t_tensor_us": 1e6 * t_tensor,
+            "frac": t_bound / (ms_step * 1e-3)}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
     ap.add_argument("--e2e-steps", type=int, default=10)
+    ap.add_argument("--repeats", type=int, default=5, help="timed regions of --steps forwards each (median reported)")
+    ap.add_argument("--min-seconds", type=float, default=0.5, help="keep repeating until this much device time is covered")
     ap.add_argument("--layout", choices=["dense", "bnhd", "qkv"], default="dense",
                     help="storage of Q, K, V and out: dense [B,h,N,d]; bnhd = [B,N,h,d] (forward_strided); "
                          "qkv = Q, K, V interleaved as [B,N,3,h,d], out [B,N,h,d] (forward_strided)")
@@ -242,6 +334,7 @@ def main():
                     help="backward: time agent_attn_backward (fp32 gradients of Q, K, V, both biases and the filter) "
                          "instead of the forward pass; prints a line with \"pass\": \"backward\"")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-configs", action="store_true", help="skip the short runs of the other configurations")
     ap.add_argument("--min-warmup-seconds", type=float, default=0.2)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
@@ -258,30 +351,11 @@ def main():
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
     dt = TORCH_DTYPE[w.dtype]
+    l2_bytes = int(torch.cuda.get_device_properties(dev).L2_cache_size)     # cudaDevAttrL2CacheSize
 
-    # Rotating buffer sets: together more than 4x the L2, so no step re-reads a resident set.
     set_bytes = w.algorithmic_bytes()
-    n_sets = max(2, -(-4 * L2_BYTES // set_bytes))
-    host = make_inputs(w, seed=w.seed + 1000 * rank)
-    sets = []
-    for s in range(n_sets):
-        g = torch.Generator(device="cpu").manual_seed(17 + s)
-        roll = int(torch.randint(1, w.tokens, (1,), generator=g))
-        d = {k: (None if v is None else v.to(dev)) for k, v in host.items()}
-        if s:  # distinct contents per set, same distribution (a roll along the token axis)
-            for k in ("q", "k", "v"):
-                d[k] = torch.roll(d[k], roll, dims=2).contiguous()
-        d["out"] = torch.empty_like(d["q"])
-        if args.layout != "dense":      # the same values behind token-major storage; views keep the [B,h,N,d] shape
-            if args.layout == "qkv":
-                packed = torch.stack([d[k].permute(0, 2, 1, 3) for k in ("q", "k", "v")], dim=2).contiguous()
-                for j, k in enumerate(("q", "k", "v")):
-                    d[k] = packed[:, :, j].permute(0, 2, 1, 3)
-            else:
-                for k in ("q", "k", "v"):
-                    d[k] = d[k].permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
-            d["out"] = torch.empty((w.batch, w.tokens, w.heads, w.head_dim), dtype=dt, device=dev).permute(0, 2, 1, 3)
-        sets.append(d)
+    n_sets = n_sets_for(w, l2_bytes)
+    host, sets = make_sets(w, dev, n_sets, rank, args.layout)
     mod = AgentAttention(w.batch, w.heads, w.head_dim, w.tokens, w.agents, dt, device=local_rank)
     ws = mod.workspace(w.grid_h, w.grid_w, w.agents)
     stream = torch.cuda.current_stream()
@@ -292,59 +366,62 @@ def main():
         pdist.shutdown()
         return
 
-    def step(i):
-        d = sets[i % n_sets]
-        fwd = mod.forward if args.layout == "dense" else mod.forward_strided
-        fwd(d["q"], d["k"], d["v"], w.grid_h, w.grid_w, w.agents, b1=d["b1"], b2=d["b2"],
-            dwc_weight=d["dwc"], out=d["out"], workspace=ws, stream=stream)
-
     # warm-up: W steps, and at least 0.2 s so that clocks have ramped
     t_w = time.perf_counter()
-    i = 0
-    while i < args.warmup or time.perf_counter() - t_w < args.min_warmup_seconds:
-        step(i)
-        i += 1
-        if i % 64 == 0:
-            torch.cuda.synchronize()
+    done = 0
+    while done < args.warmup or time.perf_counter() - t_w < args.min_warmup_seconds:
+        time_forward(mod, w, sets, ws, stream, 16, 1, args.layout)
+        done += 16
     torch.cuda.synchronize()
     launches_per_step = mod.last_launch_count()
 
+    # the timed region: `repeats` x exactly `steps` forward calls, device time by CUDA events, max over ranks
     sampler = ClockSampler(local_rank)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     pdist.barrier()
     torch.cuda.synchronize()
     sampler.start()
-    e0.record(stream)
-    for i in range(args.steps):
-        step(i)
-    e1.record(stream)
+    times = time_forward(mod, w, sets, ws, stream, args.steps, args.repeats, args.layout, args.min_seconds)
     torch.cuda.synchronize()
     pdist.barrier()
     clocks = sampler.stop()
-    ms_total = pdist.max_over_ranks(e0.elapsed_time(e1))
-    ms_step = ms_total / args.steps
+    if mod.query_status() != 0:
+        raise SystemExit("a device-side bounded wait expired during the timed region: the timing is void")
+    ms_step = pdist.max_over_ranks(statistics.median(times))
+    ms_min = pdist.max_over_ranks(min(times))
     tokens_per_step = world * w.batch * w.tokens
     value = tokens_per_step / (ms_step * 1e-3)
 
     s = w.elem_bytes
     unit = w.slabs * w.tokens * w.head_dim * s                       # one [B,h,N,d] tensor
     bias_b = w.heads * w.agents * w.tokens * s if w.bias else 0
-    peak, peak_src = measured_peaks()
-    if launches_per_step != 1 and args.layout != "dense":
-        # the step-level entry points take dense tensors only: report the whole path as one unit
+    wd_b = 9 * w.heads * w.head_dim * s if w.dwc else 0
+    peak, tensor_peak, peak_src = measured_peaks()
+    kb_steps = min(args.steps, 200)
+    kern_note = None
+    if launches_per_step == 3 and args.layout == "dense":
+        # three streaming kernels per forward call: each timed by itself between events through the stage mask
+        # (a later stage alone reads what the last full call left in the workspace)
+        names = ("prep", "aggregate", "broadcast_dwc")
+        kern_ms = {}
+        for bit, nm in enumerate(names):
+            mod.set_stage_mask(1 << bit)
+            time_forward(mod, w, sets, ws, stream, 8, 1)
+            kern_ms[nm] = statistics.median(time_forward(mod, w, sets, ws, stream, kb_steps, 3))
+        mod.set_stage_mask(7)
+        # what each kernel itself has to touch (the second reads of Q and V are meant to come from L2)
+        kern_bytes = {"prep": unit + 2 * bias_b + wd_b, "aggregate": 2 * unit + bias_b,
+                      "broadcast_dwc": 3 * unit + bias_b + wd_b}
+        kern_note = ("kernel_ms: each kernel launched alone, back to back with itself (so without the overlap that "
+                     "programmatic dependent launch gives the path); kernel_algorithmic_bytes counts what a kernel "
+                     "touches, second reads of Q and V included, so it sums to more than the path's bytes")
         dominant = "forward_path"
-        kern_ms = {dominant: ms_step}
-        kern_bytes = {dominant: set_bytes}
-    elif launches_per_step == 1:
-        # the whole path is one persistent kernel: its launch duration is the step time (the only other
-        # node on the stream is a few-hundred-byte memset), its algorithmic bytes are the path's
-        dominant = "fused_kernel"
+    elif launches_per_step == 1 or args.layout != "dense":
+        dominant = "fused_kernel" if launches_per_step == 1 else "forward_path"
         kern_ms = {dominant: ms_step}
         kern_bytes = {dominant: set_bytes}
     else:
         # one kernel per step of the path: time each between events on the launching stream, through the
         # step-level entry points
-        kb_steps = min(args.steps, 200)
         evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(kb_steps)]
         a_buf = torch.empty((w.batch, w.heads, w.agents, w.head_dim), dtype=dt, device=dev)
         va_buf = torch.empty_like(a_buf)
@@ -362,21 +439,58 @@ def main():
         torch.cuda.synchronize()
         kern_ms = {nm: statistics.mean(evs[i][j].elapsed_time(evs[i][j + 1]) for i in range(kb_steps))
                    for j, nm in enumerate(("pool", "aggregate", "broadcast_dwc"))}
-        kern_bytes = {"pool": unit, "aggregate": 2 * unit + bias_b,
-                      "broadcast_dwc": unit + bias_b + (9 * w.heads * w.head_dim * s if w.dwc else 0)}
+        kern_bytes = {"pool": unit, "aggregate": 2 * unit + bias_b, "broadcast_dwc": unit + bias_b + wd_b}
         dominant = max(kern_ms, key=kern_ms.get)
-    dom_gbs = kern_bytes[dominant] / (kern_ms[dominant] * 1e-3) / 1e9
     path_gbs = set_bytes / (ms_step * 1e-3) / 1e9
+    if dominant == "forward_path":
+        dom_gbs, dom_ms, dom_bytes = path_gbs, ms_step, set_bytes
+    else:
+        dom_ms, dom_bytes = kern_ms[dominant], kern_bytes[dominant]
+        dom_gbs = dom_bytes / (dom_ms * 1e-3) / 1e9
     roofline = {
         "bound": "hbm", "kernel": dominant, "achieved": dom_gbs, "peak": peak, "unit": "GB/s",
-        "frac": dom_gbs / peak, "traffic": NCU_TRAFFIC.get((w.name, dominant)), "peak_source": peak_src,
+        "frac": dom_gbs / peak, "traffic": traffic_of(w.name) if launches_per_step == 3 else None, "peak_source": peak_src,
+        "launches_per_step": launches_per_step,
         "kernel_ms": kern_ms, "kernel_algorithmic_bytes": kern_bytes,
+        "kernel_frac": {k: kern_bytes[k] / (kern_ms[k] * 1e-3) / 1e9 / peak for k in kern_ms},
         "path_achieved": path_gbs, "path_frac": path_gbs / peak, "path_frac_nominal_8TBs": path_gbs / 8000.0,
         "path_algorithmic_bytes": set_bytes, "path_tflops": flops_of(w) / (ms_step * 1e-3) / 1e12,
     }
+    if kern_note:
+        roofline["note"] = kern_note
+
+    # the other configurations, briefly (same protocol, fewer repeats): tokens/s against N for the high-resolution pair
+    configs = None
+    if not args.no_configs and world == 1 and args.layout == "dense":
+        configs = [{"workload": w.name, "tokens": w.tokens, "agents": w.agents, "dtype": w.dtype, "ms_per_step": ms_step,
+                    "tokens_per_s": value, "algorithmic_bytes": set_bytes, **bound_of(w, ms_step, peak, tensor_peak)}]
+        del sets
+        torch.cuda.empty_cache()
+        for name in ("cfg2_deit_bf16", "cfg4_sd_f16", "cfg5a_hires_bf16", "cfg5b_hires_bf16"):
+            if name == w.name:
+                continue
+            wc = WORKLOADS[name]
+            _, sc = make_sets(wc, dev, n_sets_for(wc, l2_bytes), rank)
+            mc = AgentAttention(wc.batch, wc.heads, wc.head_dim, wc.tokens, wc.agents, TORCH_DTYPE[wc.dtype], device=local_rank)
+            wsc = mc.workspace(wc.grid_h, wc.grid_w, wc.agents)
+            time_forward(mc, wc, sc, wsc, stream, 20, 1)
+            est = statistics.median(time_forward(mc, wc, sc, wsc, stream, 10, 2))
+            k = max(10, min(200, int(0.05 / (est * 1e-3))))
+            tc = time_forward(mc, wc, sc, wsc, stream, k, 3)
+            if mc.query_status() != 0:
+                raise SystemExit(f"a device-side bounded wait expired on {name}")
+            msc = statistics.median(tc)
+            configs.append({"workload": name, "tokens": wc.tokens, "agents": wc.agents, "dtype": wc.dtype, "ms_per_step": msc,
+                            "ms_per_step_min": min(tc), "steps": k, "repeats": 3, "launches_per_step": mc.last_launch_count(),
+                            "tokens_per_s": wc.batch * wc.tokens / (msc * 1e-3), "algorithmic_bytes": wc.algorithmic_bytes(),
+                            **bound_of(wc, msc, peak, tensor_peak)})
+            del sc, mc, wsc
+            torch.cuda.empty_cache()
+        _, sets = make_sets(w, dev, 2, rank)          # (the end-to-end leg below needs no device sets)
 
     # end to end through the host-buffer entry point: pinned inputs in, result out, every step
     e2e = None
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     if args.e2e_steps > 0:
         pin = {k: (None if v is None else v.pin_memory()) for k, v in host.items()}
         out_h = torch.empty_like(pin["q"]).pin_memory()
@@ -401,6 +515,8 @@ def main():
             stream.wait_stream(st)
         e1.record(stream)
         torch.cuda.synchronize()
+        if mod.query_status() != 0:
+            raise SystemExit("a device-side bounded wait expired during the end-to-end region")
         ms_e2e = pdist.max_over_ranks(e0.elapsed_time(e1)) / args.e2e_steps
         h2d = sum(v.numel() * v.element_size() for v in pin.values() if v is not None)
         e2e = {"value": tokens_per_step / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
@@ -409,31 +525,24 @@ def main():
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        from oracle import agent_attention_oracle as orc
-        threads = orc.max_threads()
-        inp_np = {k: (None if v is None else v.double().numpy()) for k, v in host.items()}
-        best, used, reps, spent = None, 1, 0, 0.0
-        while reps < 3 or (spent < 2.0 and reps < 20):
-            t, used = oracle_sample_run(w, inp_np, threads)
-            best = t if best is None else min(best, t)
-            spent += t
-            reps += 1
-        cpu_baseline = {"value": w.batch * w.tokens / best, "unit": UNIT, "cores": used, "kind": "oracle",
-                        "sample": f"the full {w.name} batch ({w.slabs} slabs), best of {reps} passes, "
-                                  f"{spent * used:.0f} core-seconds in total"}
+        base = oracle_baseline(w, passes=3, warmup=1)
+        cpu_baseline = {k: base[k] for k in ("value", "unit", "cores", "kind", "sample")}
 
     if rank == 0:
         print(json.dumps({
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "warmup": args.warmup, "ms_per_step": ms_step, "ms_per_step_min": ms_min, "repeats": len(times),
+            "timed_steps_total": len(times) * args.steps,
+            "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
             "config": {"workload": w.name, "batch_per_gpu": w.batch, "heads": w.heads, "tokens": w.tokens,
                        "grid": [w.grid_h, w.grid_w], "head_dim": w.head_dim, "agents": w.agents,
                        "bias": w.bias, "dwc": w.dwc, "layout": args.layout,
-                       "l2": f"{n_sets} rotating buffer sets of {set_bytes / 1e6:.1f} MB (> 4x the 126 MB L2)",
+                       "l2": f"{n_sets} rotating buffer sets of {set_bytes / 1e6:.1f} MB (> 4x the {l2_bytes / 2**20:.0f} MiB L2)",
+                       "timing": f"median of {len(times)} regions of {args.steps} forward calls each, CUDA events",
                        "parallelism": f"batch-sharded x{world}, no collective"},
-            "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
-            "roofline": roofline, "cpu_baseline": cpu_baseline,
+            "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * len(times) * args.steps,
+            "roofline": roofline, "configs": configs, "cpu_baseline": cpu_baseline,
         }))
     pdist.shutdown()
 

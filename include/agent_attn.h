@@ -92,10 +92,14 @@ int agent_attn_destroy(agent_attn_handle* h);
 const char* agent_attn_last_error(const agent_attn_handle* h);
 
 /* Bytes of device workspace that agent_attn_forward / agent_attn_aggregate need for this
- * grid and agent count (holds A, V_A, the per-split online-softmax partials (max, sum, acc)
- * and one arrival counter per slab).  Returns 0 on invalid arguments.  Its contents need
- * no initialisation and carry nothing from call to call; it may be reused by any number of
- * calls that do not overlap on the GPU. */
+ * grid and agent count (holds A, V_A, the per-split online-softmax partials (max, sum, acc),
+ * one arrival counter per slab and, for the streaming kernels, scaled copies of the agents, the
+ * biases clamped to finite values and re-laid for the tensor core, and the depthwise filter as
+ * diagonal operand slices).  Returns 0 on invalid arguments.  Its contents need no initialisation
+ * and carry nothing from call to call; it may be reused by any number of calls that do not
+ * overlap on the GPU.  After agent_attn_forward the pooled agents A ([B][heads][n][d], element
+ * type) sit at offset 0 and the agent features V_A (same shape) at the next multiple of 256 bytes:
+ * callers may read them (the tests do). */
 size_t agent_attn_workspace_bytes(const agent_attn_handle* h, int grid_h, int grid_w, int n_agents);
 
 /* The whole module, Eq. 6.
@@ -238,6 +242,19 @@ int agent_attn_query_status(agent_attn_handle* h, void* stream);
 
 /* Number of kernels the most recent successful call on this handle enqueued. */
 int agent_attn_last_launch_count(const agent_attn_handle* h);
+
+/* Test hook (no counterpart in the paper): how many times a block of the task-queue kernel polls another block's
+ * counter before its wait gives up; 0xffffffff restores the built-in limit.  With 0 the first unsatisfied poll
+ * expires: the kernel records AA_ERR_TIMEOUT in the status word and carries on with whatever the workspace holds
+ * (a wrong result, every access still inside the caller's buffers; no copy is left in flight, since the mbarrier
+ * waits keep their own limit).  Affects AA_PATH_QUEUE handles and the shapes AA_PATH_AUTO gives to that kernel. */
+int agent_attn_test_set_poll_limit(agent_attn_handle* h, unsigned polls);
+
+/* Measurement hook (no counterpart in the paper): which of the three streaming kernels agent_attn_forward
+ * launches on the shapes it gives to them: bit 0 = prep (pooling, prepared operands), bit 1 = aggregation,
+ * bit 2 = broadcast + depthwise term; 7 (the default) = the whole path.  A later stage launched alone reads what
+ * an earlier full call left in the workspace, so each kernel can be timed by itself between CUDA events. */
+int agent_attn_test_set_stage_mask(agent_attn_handle* h, unsigned mask);
 
 /* Agent aggregation without any caller- or library-side allocation (the paper has no counterpart
  * of this call; it computes exactly what agent_attn_aggregate computes).

@@ -26,7 +26,8 @@ EXPORTS = [
     "agent_attn_staging_bytes", "agent_attn_forward_host", "agent_attn_query_status",
     "agent_attn_last_launch_count", "agent_attn_aggregate_static", "agent_attn_static_scratch_bytes",
     "agent_attn_compose_bias", "agent_attn_forward_strided",
-    "agent_attn_backward_workspace_bytes", "agent_attn_backward",
+    "agent_attn_backward_workspace_bytes", "agent_attn_backward", "agent_attn_test_set_poll_limit",
+    "agent_attn_test_set_stage_mask",
 ]
 
 
@@ -109,6 +110,10 @@ def load_library(build_if_missing: bool = True) -> ctypes.CDLL:
     lib.agent_attn_backward.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ctypes.POINTER(AgentAttnBias), vp,
                                         ctypes.POINTER(AgentAttnGrads), vp, sz, vp]
     lib.agent_attn_backward.restype = ci
+    lib.agent_attn_test_set_stage_mask.argtypes = [vp, ctypes.c_uint]
+    lib.agent_attn_test_set_stage_mask.restype = ci
+    lib.agent_attn_test_set_poll_limit.argtypes = [vp, ctypes.c_uint]
+    lib.agent_attn_test_set_poll_limit.restype = ci
     lib.agent_attn_static_scratch_bytes.argtypes = []
     lib.agent_attn_static_scratch_bytes.restype = sz
     _lib = lib
@@ -176,6 +181,23 @@ class AgentAttention:
         if self._ws is None or self._ws.numel() < need:
             self._ws = torch.empty(need, dtype=torch.uint8, device=self.device)
         return self._ws
+
+    def intermediates(self, workspace: torch.Tensor, n_agents: int):
+        """Views of the agents A and the agent features V_A ([B, heads, n, d] each) that `forward` left in its
+        workspace: A occupies the first B*heads*n*d elements, V_A starts at the next multiple of 256 bytes."""
+        count = self.batch * self.heads * n_agents * self.head_dim
+        nbytes = count * workspace.new_empty(0, dtype=self.dtype).element_size()
+        va_off = (nbytes + 255) // 256 * 256
+        shape = (self.batch, self.heads, n_agents, self.head_dim)
+        return (workspace[:nbytes].view(self.dtype).view(shape), workspace[va_off:va_off + nbytes].view(self.dtype).view(shape))
+
+    def set_stage_mask(self, mask: int):
+        """Measurement hook: which of the three streaming kernels `forward` launches (1 prep | 2 aggregation | 4 broadcast)."""
+        self._check(self.lib.agent_attn_test_set_stage_mask(self._h, mask))
+
+    def set_poll_limit(self, polls: int):
+        """Test hook: polls of another block's counter before a wait of the task-queue kernel gives up."""
+        self._check(self.lib.agent_attn_test_set_poll_limit(self._h, polls & 0xffffffff))
 
     def last_launch_count(self) -> int:
         return int(self.lib.agent_attn_last_launch_count(self._h))

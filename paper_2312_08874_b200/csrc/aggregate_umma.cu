@@ -182,7 +182,7 @@ __global__ void __launch_bounds__(NT, 1) aggregate_umma_kernel(const __grid_cons
         for (int t = 0; t < tiles; ++t) {
             const int b = t & 1, s = t % STAGES;
             const int valid = min(32, N - ((t0 + t) * KT + 32 * c));      // tokens of this thread's half
-            pipe_wait(pp, BAR_S_FULL + 2 * mb + b, kTimeoutTile);
+            pipe_wait_one(pp, BAR_S_FULL + 2 * mb + b, kTimeoutTile);
             tc_fence_after_sync();
             float sv[32];
             {
@@ -248,7 +248,7 @@ __global__ void __launch_bounds__(NT, 1) aggregate_umma_kernel(const __grid_cons
                 started = true;
             }
             // P of the previous tile has been consumed (and every product into this thread's accumulator is done)
-            if (t > 0) { pipe_wait(pp, BAR_PV + mb, kTimeoutTile); tc_fence_after_sync(); }
+            if (t > 0) { pipe_wait_one(pp, BAR_PV + mb, kTimeoutTile); tc_fence_after_sync(); }
             if (__any_sync(0xffffffffu, resc)) {               // rare: the reference maximum of some row moved
                 uint32_t ra[32];
 #pragma unroll
@@ -271,7 +271,7 @@ __global__ void __launch_bounds__(NT, 1) aggregate_umma_kernel(const __grid_cons
             tc_fence_before_sync();
             pipe_arrive(pp, BAR_P_FULL + mb);
         }
-        pipe_wait(pp, BAR_PV + mb, kTimeoutTile);
+        pipe_wait_one(pp, BAR_PV + mb, kTimeoutTile);
         tc_fence_after_sync();
         // both chains are through with the ring before its memory is reused for the exchange below
         asm volatile("bar.sync 3, %0;\n" ::"r"(256 * MB) : "memory");

@@ -26,6 +26,7 @@ struct agent_attn_handle {
     StreamArgs stream_args; // last call of the streaming path: its tensor maps are reused while the pointers repeat
     bool stream_args_valid;
     unsigned poll_limit;    // flag-poll limit of the task-queue kernel (test hook; 0xffffffff = the kernel's own)
+    unsigned stage_mask;    // which of the three streaming kernels a forward call launches (measurement hook; 7 = all)
     char err[512];
 };
 
@@ -266,6 +267,7 @@ int agent_attn_create(agent_attn_handle** out, const agent_attn_config* cfg) {
     h->scale1 = cfg->scale1 > 0.f ? cfg->scale1 : def;
     h->scale2 = cfg->scale2 > 0.f ? cfg->scale2 : def;
     h->poll_limit = 0xffffffffu;
+    h->stage_mask = 7u;
     if (cudaMalloc(&h->d_status, sizeof(int)) != cudaSuccess || cudaMemset(h->d_status, 0, sizeof(int)) != cudaSuccess) {
         delete h;
         return AA_ERR_CUDA;
@@ -287,6 +289,18 @@ int agent_attn_destroy(agent_attn_handle* h) {
 const char* agent_attn_last_error(const agent_attn_handle* h) { return h ? h->err : kNullHandleMsg; }
 
 int agent_attn_last_launch_count(const agent_attn_handle* h) { return h ? h->launches : 0; }
+
+int agent_attn_test_set_stage_mask(agent_attn_handle* h, unsigned mask) {
+    if (!h || (mask & 7u) == 0u) return AA_ERR_INVALID_ARG;
+    h->stage_mask = mask & 7u;
+    return AA_OK;
+}
+
+int agent_attn_test_set_poll_limit(agent_attn_handle* h, unsigned polls) {
+    if (!h) return AA_ERR_INVALID_ARG;
+    h->poll_limit = polls;
+    return AA_OK;
+}
 
 size_t agent_attn_workspace_bytes(const agent_attn_handle* h, int grid_h, int grid_w, int n_agents) {
     if (!h || grid_h <= 0 || grid_w <= 0 || n_agents <= 0) return 0;
@@ -410,9 +424,12 @@ static int forward_impl(agent_attn_handle* h, const void* Q, const void* K, cons
                 h->stream_args = sa;
                 h->stream_args_valid = true;
             }
-            cudaError_t e = launch_stream(h->cfg.dtype, sa, st);
+            cudaError_t e = cudaSuccess;
+            h->launches = 0;
+            if (e == cudaSuccess && (h->stage_mask & 1u)) { e = launch_stream_prep(h->cfg.dtype, sa, st); h->launches++; }
+            if (e == cudaSuccess && (h->stage_mask & 2u)) { e = launch_stream_aggregate(h->cfg.dtype, sa, st); h->launches++; }
+            if (e == cudaSuccess && (h->stage_mask & 4u)) { e = launch_stream_broadcast(h->cfg.dtype, sa, st); h->launches++; }
             if (e != cudaSuccess) return fail(h, AA_ERR_CUDA, "streaming launch failed: %s", cudaGetErrorString(e));
-            h->launches = 3;
             return AA_OK;
         }
     }
@@ -434,6 +451,7 @@ static int forward_impl(agent_attn_handle* h, const void* Q, const void* K, cons
             fa.a_ws = ws + w.a_off; fa.va_ws = ws + w.va_off;
             fa.partials = reinterpret_cast<float*>(ws + w.part_off);
             fa.counters = counters; fa.status = h->d_status;
+            fa.poll_limit = h->poll_limit == 0xffffffffu ? (1u << 20) : h->poll_limit;
             fa.slabs = slabs; fa.heads = h->cfg.heads; fa.H = grid_h; fa.W = grid_w; fa.d = h->cfg.head_dim;
             fa.n = n_agents; fa.p = p; fa.scale1 = h->scale1; fa.scale2 = h->scale2; fa.plan = h->fused_plan;
             fa.lin = cl.in; fa.lout = cl.out;
@@ -444,6 +462,13 @@ static int forward_impl(agent_attn_handle* h, const void* Q, const void* K, cons
             return AA_OK;
         }
     }
+    // strided tensors are read in place only by the task-queue and the tensor-memory kernels: decide before anything
+    // is launched
+    if (cl.strided && !(use_umma(h, N, n_agents) && !use_simt(h) && auto_like(h) &&
+                        broadcast_umma_eligible(h->cfg.dtype, n_agents, N, h->cfg.head_dim)))
+        return fail(h, AA_ERR_UNSUPPORTED,
+                    "strided tensors need the task-queue kernel (16-bit, d = 64, n <= 64, pooled agents, W <= 64) or the "
+                    "tensor-memory kernels (16-bit, d <= 64, n a multiple of 8 in 72..256)");
     const void* agents = A;
     if (!A) {
         if (int rc = do_pool(h, Q, grid_h, grid_w, p, p, ws + w.a_off, st, &cl)) return rc;

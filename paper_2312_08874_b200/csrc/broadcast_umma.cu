@@ -224,7 +224,7 @@ __global__ void __launch_bounds__(NT, 1) broadcast_umma_kernel(const __grid_cons
                 sW[e] = ch < d ? Elem<T>::to_f32(w[ch * 9 + tap]) : 0.f;
             }
         }
-        pipe_wait(pp, BAR_AG, kTimeoutLoads);
+        pipe_wait_one(pp, BAR_AG, kTimeoutLoads);
         for (int e = tid; e < (128 * MB - n) * 8; e += NROW)
             *(reinterpret_cast<uint4*>(smem + OFF_VA + (n + (e >> 3)) * 128) + (e & 7)) = make_uint4(0u, 0u, 0u, 0u);
         fence_proxy_async();
@@ -241,7 +241,7 @@ __global__ void __launch_bounds__(NT, 1) broadcast_umma_kernel(const __grid_cons
                 const int j = i * MB + a, b = j & 1;
                 const int valid = min(32, n - (128 * a + 32 * gq));     // agents of this thread in the step
                 const bool tv = valid > 0;                              // uniform per warp
-                pipe_wait(pp, BAR_S_FULL + b, kTimeoutTile);
+                pipe_wait_one(pp, BAR_S_FULL + b, kTimeoutTile);
                 tc_fence_after_sync();
                 float sv[32];
                 {
@@ -251,7 +251,7 @@ __global__ void __launch_bounds__(NT, 1) broadcast_umma_kernel(const __grid_cons
                     tc_fence_before_sync();
                     pipe_arrive(pp, BAR_S_EMPTY + b);
                     if (has_b2) {                            // logits in natural units: scale2 * q.a + b2
-                        pipe_wait(pp, BAR_B_FULL + b, kTimeoutLoads);
+                        pipe_wait_one(pp, BAR_B_FULL + b, kTimeoutLoads);
                         const unsigned char* sB = smem + OFF_B2 + b * 4 * kTile + (gq >> 1) * 2 * kTile + row * 128;
 #pragma unroll
                         for (int jj = 0; jj < 4; ++jj) {
@@ -307,7 +307,7 @@ __global__ void __launch_bounds__(NT, 1) broadcast_umma_kernel(const __grid_cons
                     started = true;
                 }
                 // the previous step's product is done: P may be overwritten, this thread's accumulator is at rest
-                if (a > 0) { pipe_wait(pp, BAR_PV, kTimeoutTile); tc_fence_after_sync(); }
+                if (a > 0) { pipe_wait_one(pp, BAR_PV, kTimeoutTile); tc_fence_after_sync(); }
                 if (__any_sync(0xffffffffu, resc)) {           // rare: the reference maximum of some row moved
                     uint32_t ra[32];
 #pragma unroll
@@ -337,7 +337,7 @@ __global__ void __launch_bounds__(NT, 1) broadcast_umma_kernel(const __grid_cons
             if (has_dwc) {
                 // tap (u, v) of this thread's token sits at row (row + v) of run u; taps outside the grid
                 // (or in another slab, or past the head dim) contribute nothing
-                pipe_wait(pp, BAR_H_FULL, kTimeoutLoads);
+                pipe_wait_one(pp, BAR_H_FULL, kTimeoutLoads);
                 const int tk = min(tok, N - 1);
                 const int y = tk / W, x = tk - y * W;
                 const bool live = tok < N && nch > 0;
@@ -367,7 +367,7 @@ __global__ void __launch_bounds__(NT, 1) broadcast_umma_kernel(const __grid_cons
                 pipe_arrive(pp, BAR_H_EMPTY);
             }
             sML[gq * 128 + row] = make_float2(started ? m_ref : -INFINITY, started ? l : 0.f);
-            pipe_wait(pp, BAR_PV, kTimeoutTile);
+            pipe_wait_one(pp, BAR_PV, kTimeoutTile);
             tc_fence_after_sync();
             asm volatile("bar.sync 1, %0;\n" ::"n"(NROW) : "memory");
             {

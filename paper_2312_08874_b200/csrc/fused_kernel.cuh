@@ -73,19 +73,19 @@ __device__ __forceinline__ unsigned ld_acquire(const unsigned* p) {
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
-// The calling thread polls until *ctr >= target; gives up after kSpinLimit polls and records `code`.
-__device__ __forceinline__ void poll_counter(const unsigned* ctr, unsigned target, int* status, int code) {
+// The calling thread polls until *ctr >= target; gives up after `limit` polls and records `code`.
+__device__ __forceinline__ void poll_counter(const unsigned* ctr, unsigned target, int* status, int code, unsigned limit) {
     unsigned spins = 0;
     while (ld_acquire(ctr) < target) {
-        if (++spins > kSpinLimit) { atomicExch(status, code); break; }
+        if (++spins > limit) { atomicExch(status, code); break; }
         // once any block has given up, the others stop waiting too
         if ((spins & 255u) == 0 && ld_acquire(reinterpret_cast<const unsigned*>(status)) != 0u) break;
         __nanosleep(40);
     }
 }
 // Thread 0 polls, then a block barrier passes the result on.
-__device__ __forceinline__ void wait_counter(const unsigned* ctr, unsigned target, int* status, int code) {
-    if (threadIdx.x == 0) poll_counter(ctr, target, status, code);
+__device__ __forceinline__ void wait_counter(const unsigned* ctr, unsigned target, int* status, int code, unsigned limit) {
+    if (threadIdx.x == 0) poll_counter(ctr, target, status, code, limit);
     __syncthreads();
 }
 // Publish: all of this block's prior global writes become visible before the counter moves.
@@ -127,22 +127,6 @@ __device__ __forceinline__ void load_tokens(uint32_t dst, const CUtensorMap* map
     else tma_load_tok(dst, map, head_first, tok, head, b, bar);
 }
 
-// Optional per-task phase timestamps (debug builds only): define AA_FUSED_TRACE and hand a device
-// buffer to aa_fused_trace_buffer; record i of a block goes to slot (blockIdx, i).
-#ifdef AA_FUSED_TRACE
-__device__ unsigned long long* g_trace = nullptr;
-__device__ __forceinline__ void trace_mark(int task_slot, int phase) {
-    if (threadIdx.x == 0 && g_trace && task_slot < 16) {
-        unsigned long long t;
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-        g_trace[((size_t)blockIdx.x * 16 + task_slot) * 8 + phase] = t;
-    }
-}
-#define TRACE(slot, phase) trace_mark(slot, phase)
-#else
-#define TRACE(slot, phase)
-#endif
-
 // Flat global -> shared copy of `bytes` (a multiple of 2) by plain loads: the fallback when a
 // bulk copy's alignment rules do not hold.
 __device__ __forceinline__ void copy_flat(unsigned char* dst, const unsigned char* src, int bytes, int tid) {
@@ -179,7 +163,7 @@ using ShapeAny = FusedShape<0, 0, 0, false>;
 // ---------------------------------------------------------------------------------- G task
 template <typename T, typename SH>
 __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub, unsigned char* smem,
-                                           BlockState& st, int* s_flag, int slot, int& next_task) {
+                                           BlockState& st, int* s_flag, int& next_task) {
     constexpr int NWK = 2, KW = KT / NWK;
     constexpr int cpr = DK / 8;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -223,8 +207,6 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
             }
         }
     };
-
-    TRACE(slot, 0);
     // 1. start the ring
     for (int s = 0; s < STAGES - 1; ++s)
         if (s < tiles) issue_tile(s, s);
@@ -308,15 +290,13 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
             }
         }
     }
-    TRACE(slot, 1);
     // 3. publish these agent rows, wait for the slab's other G tasks
     publish_add(p.counters + slab);
-    wait_counter(p.counters + slab, (unsigned)p.plan.g_tasks, p.status, kTimeoutAgents);
-
-    TRACE(slot, 2);
+    wait_counter(p.counters + slab, (unsigned)p.plan.g_tasks, p.status, kTimeoutAgents, p.poll_limit);
     // 4. all agents of the slab -> shared memory (rows >= n receive foreign rows; they only feed
     //    padded agent rows, which are never merged)
     if (tid == 0) {
+        fence_proxy_async_all();       // the siblings' agent rows were written with plain stores
         mbar_arrive_expect_tx(bar_agents(st), kTileBytes);
         tma_load_2d(smem_u32(sA), &p.tm_a, 0, slab * n, bar_agents(st));
     }
@@ -338,8 +318,6 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
     float acc[DK / 8][4], accl[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
     for (int j = 0; j < DK / 8; ++j) { acc[j][0] = acc[j][1] = acc[j][2] = acc[j][3] = 0.f; }
-
-    TRACE(slot, 3);
     // 5. online-softmax aggregation over the range
     for (int it = 0; it < tiles; ++it) {
         const int s = it % STAGES;
@@ -351,6 +329,14 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
         const unsigned char* sV = sK + kTileBytes;
         const unsigned char* sB = sV + kTileBytes;
         const int c0 = t_begin + it * KT;
+        if (c0 + KT > t_end) {
+            // ragged last tile: the rows past the range belong to the next range or slab; their weights are 0, and
+            // 0 * NaN is not 0, so the V rows are cleared before the product
+            unsigned char* vz = ring + s * kStageBytes + kTileBytes;
+            for (int e = tid; e < (c0 + KT - t_end) * 8; e += NT)
+                *(reinterpret_cast<uint4*>(vz + (t_end - c0 + (e >> 3)) * 128) + (e & 7)) = make_uint4(0u, 0u, 0u, 0u);
+            __syncthreads();
+        }
 
         float sc[KW / 8][4];
 #pragma unroll
@@ -438,8 +424,6 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
     // row sums sit in column 0 of the extra product: lanes with t4 == 0 hold them
     const float l0 = __shfl_sync(0xffffffffu, accl[0], lane & ~3);
     const float l1 = __shfl_sync(0xffffffffu, accl[2], lane & ~3);
-
-    TRACE(slot, 4);
     // 6. the two key halves of the block combine through shared memory into one partial state;
     float* sX = reinterpret_cast<float*>(ring);        // [4 row groups][36 values][32 lanes]
     if (wk == 1) {
@@ -482,7 +466,7 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
     //    agent rows (fixed order of the parts: bit-reproducible) and counts itself done
     unsigned* arrived = p.counters + p.slabs + slab;
     publish_add(arrived);
-    wait_counter(arrived, (unsigned)p.plan.g_tasks, p.status, kTimeoutAgents);
+    wait_counter(arrived, (unsigned)p.plan.g_tasks, p.status, kTimeoutAgents, p.poll_limit);
     // no wait lies ahead in this task: take the next ticket now, so that the queue's round trip runs under the merge
     if (tid == 0) next_task = (int)atomicAdd(p.counters + 3 * (size_t)p.slabs, 1u);
     {
@@ -526,12 +510,11 @@ __device__ __forceinline__ void run_g_task(const FusedArgs& p, int slab, int sub
 // depthwise term (Eq. 6), round once and store.
 template <typename T, typename SH>
 __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int tile, unsigned char* smem,
-                                           BlockState& st, int* s_whead, float (*s_red)[128], int slot, int& next_task) {
+                                           BlockState& st, int* s_whead, float (*s_red)[128], int& next_task) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int head = slab % p.heads;
     const int H = SH::kFixed ? SH::kH : p.H, W = SH::kFixed ? SH::kW : p.W;
     const int N = H * W, n = SH::kFixed ? SH::kP * SH::kP : p.n;
-    const int n8 = (n + 7) >> 3;                      // logit column tiles that hold agents
     const int n16 = (n + 15) >> 4;
     const int R = SH::kFixed ? (QT / SH::kW > 16 ? 16 : (QT / SH::kW > SH::kH ? SH::kH : QT / SH::kW)) : p.plan.rows_per_b;
     const int y0 = tile * R;
@@ -540,8 +523,6 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
     const bool has_dwc = SH::kFixed ? true : (p.dwc_w != nullptr);
     const bool has_b2 = SH::kFixed ? true : (p.b2 != nullptr);
     const int HP = W + 2;                             // V-row pitch in tokens (zero columns at both ends)
-    const int g = lane >> 2, t4 = lane & 3, xr = lane & 7;
-
     unsigned char* sA = smem + OFF_A;
     unsigned char* sVA = smem + OFF_VA;
     float* sW = reinterpret_cast<float*>(smem + OFF_W);
@@ -550,12 +531,11 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
     T* sB2 = reinterpret_cast<T*>(smem + OFF_B2);                    // [TQ][n] flat
 
     const unsigned* va_flag = p.counters + 2 * p.slabs + slab;
-
-    TRACE(slot, 0);
     const unsigned va_target = (unsigned)p.plan.g_tasks;   // every G task of the slab merged its rows
     const bool early = ld_acquire(va_flag) >= va_target;      // usual case: the slab's aggregation is long done
     auto issue_agents = [&]() {
         if (tid == 0) {
+            fence_proxy_async_all();   // A and V_A were written by other blocks with plain stores
             mbar_arrive_expect_tx(bar_agents(st), kTileBytes + (uint32_t)n * 128u);     // A: 64-row box, V_A: n-row box
             tma_load_2d(smem_u32(sA), &p.tm_a, 0, slab * n, bar_agents(st));
             tma_load_2d(smem_u32(sVA), &p.tm_va, 0, slab * n, bar_agents(st));
@@ -618,12 +598,9 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
     }
     if (has_b2 && !b2_bulk)
         copy_flat(reinterpret_cast<unsigned char*>(sB2), reinterpret_cast<const unsigned char*>(b2src), b2bytes, tid);
-
-    TRACE(slot, 1);
     // 2. wait for the slab's agent features, then fetch A and V_A (L2)
     //    (thread 0 alone: the barrier below passes everything on; a flag already seen set is not read again)
-    if (tid == 0 && !early) poll_counter(va_flag, va_target, p.status, kTimeoutFeatures);
-    TRACE(slot, 2);
+    if (tid == 0 && !early) poll_counter(va_flag, va_target, p.status, kTimeoutFeatures, p.poll_limit);
     if (!early) issue_agents();
     wait_bar(bar_agents(st), (st.ph >> kBitAgents) & 1u, p.status, kTimeoutLoads);
     st.ph ^= 1u << kBitAgents;
@@ -636,8 +613,6 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
     __syncthreads();
     if (tid == 0 && has_dwc) *s_whead = head;      // every thread has compared the old value before the barrier
     // (rows >= n of the V_A tile are zero: the copy brings n rows and the kernel cleared the rest at its start)
-
-    TRACE(slot, 3);
     // 3. attention part on the 5th-generation tensor cores: logits S = Q A^T accumulate in tensor
     //    memory; two threads share each query row (32 logit columns each: warps w and w+4 own the same
     //    tensor-memory lanes), exchange their partial maxima and sums through shared memory, write the
@@ -733,7 +708,6 @@ __device__ __forceinline__ void run_b_task(const FusedArgs& p, int slab, int til
         tc_fence_before_sync();
     }
     __syncthreads();
-    TRACE(slot, 4);
     // the rest of the task waits for nothing: take the next ticket now, so that the queue's round trip runs under it
     if (tid == 0) next_task = (int)atomicAdd(p.counters + 3 * (size_t)p.slabs, 1u);
 
@@ -841,7 +815,6 @@ __global__ void __launch_bounds__(NT, 2) fused_kernel(const __grid_constant__ Fu
     const int count0 = Lg * G, count1 = (S - Lg) * (G + B);
     const int total = S * (G + B);
     unsigned* queue = p.counters + 3 * (size_t)S;
-    int slot = 0;
     // Every task takes the ticket of the block's next task at the start of its wait-free tail (thread 0) and
     // the ticket is handed to the block through s_task[] before the task's closing barrier, so no barrier of
     // its own is spent on the queue.  Two slots: a slot is rewritten two tasks after it was read.
@@ -867,19 +840,11 @@ __global__ void __launch_bounds__(NT, 2) fused_kernel(const __grid_constant__ Fu
             slab = S - Lg + step; sub = t - step * B; is_g = false;
         }
         int next_task = total;          // thread 0: set by the task
-        if (is_g) run_g_task<T, SH>(p, slab, sub, smem, st, &s_flag, slot, next_task);
-        else      run_b_task<T, SH>(p, slab, sub, smem, st, &s_whead, s_red, slot, next_task);
+        if (is_g) run_g_task<T, SH>(p, slab, sub, smem, st, &s_flag, next_task);
+        else      run_b_task<T, SH>(p, slab, sub, smem, st, &s_whead, s_red, next_task);
         if (tid == 0) s_task[par ^ 1] = next_task;
         fence_proxy_async();   // this task's plain shared-memory writes precede the next task's TMA writes
         __syncthreads();       // shared memory is free for the next task, and its ticket is visible
-        TRACE(slot, 5);
-#ifdef AA_FUSED_TRACE
-        if (tid == 0 && g_trace && slot < 16) {
-            g_trace[((size_t)blockIdx.x * 16 + slot) * 8 + 6] = is_g ? 1 : 2;
-            g_trace[((size_t)blockIdx.x * 16 + slot) * 8 + 7] = (unsigned long long)task;
-        }
-#endif
-        ++slot;
     }
     tc_fence_before_sync();
     __syncthreads();

@@ -21,9 +21,6 @@ cudaError_t launch_fused_s56s(int dtype, const FusedArgs& a, cudaStream_t st);
 cudaError_t launch_fused_s14s(int dtype, const FusedArgs& a, cudaStream_t st);
 
 static int fused_spec_of(int H, int W, int n_agents) {
-#ifdef AA_FUSED_TRACE
-    return 0;                      // debug builds trace the generic kernel
-#endif
     if (H == 56 && W == 56 && n_agents == 49) return 1;
     if (H == 14 && W == 14 && n_agents == 49) return 2;
     return 0;
@@ -152,9 +149,3 @@ cudaError_t launch_fused(int dtype, const FusedArgs& a, cudaStream_t st) {
 }
 
 }  // namespace aa
-
-#ifdef AA_FUSED_TRACE
-extern "C" int aa_fused_trace_buffer(void* device_buffer) {
-    return (int)cudaMemcpyToSymbol(aa::g_trace, &device_buffer, sizeof(void*));
-}
-#endif

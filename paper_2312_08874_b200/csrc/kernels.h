@@ -123,6 +123,7 @@ struct FusedArgs {
     float* partials;      // [slabs][parts][partial_floats(64, d)]
     unsigned* counters;   // zero on entry: a_count[slabs] | tickets[slabs] | va_ready[slabs] | queue[1]
     int* status;          // device status word: set when a bounded wait gives up
+    unsigned poll_limit;  // polls of another block's counter before a wait gives up
     int slabs, heads, H, W, d, n, p;
     float scale1, scale2;
     TokLayout lin, lout;  // strides of Q, K, V and of out
@@ -180,7 +181,6 @@ StreamPlan plan_stream(int dtype, int slabs, int H, int W, int d, int n_agents, 
 // workspace beyond A and V_A: bytes of (a1s | a2s | b1c | b2p), each 256-byte aligned, in this order
 size_t stream_extra_bytes(int slabs, int heads, int N, int n_agents);
 bool stream_make_maps(StreamArgs* a);
-cudaError_t launch_stream(int dtype, const StreamArgs& a, cudaStream_t st);
 cudaError_t launch_stream_prep(int dtype, const StreamArgs& a, cudaStream_t st);
 cudaError_t launch_stream_aggregate(int dtype, const StreamArgs& a, cudaStream_t st);
 cudaError_t launch_stream_broadcast(int dtype, const StreamArgs& a, cudaStream_t st);

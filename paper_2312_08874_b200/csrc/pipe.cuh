@@ -36,11 +36,6 @@ __device__ __forceinline__ void pipe_wait_one(Pipe& pp, int i, int code) {
     *reinterpret_cast<volatile int*>(pp.dead) = 1;
     if (pp.status) atomicCAS(pp.status, 0, code);
 }
-// A whole converged warp waits: every lane runs the same bounded loop (no election, no divergence:
-// a suspended try_wait costs one instruction per attempt).
-__device__ __forceinline__ void pipe_wait(Pipe& pp, int i, int code) {
-    pipe_wait_one(pp, i, code);
-}
 __device__ __forceinline__ void pipe_arrive(const Pipe& pp, int i) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(pipe_bar(pp, i)) : "memory");
 }

@@ -461,12 +461,4 @@ cudaError_t launch_stream_broadcast(int dtype, const StreamArgs& a, cudaStream_t
     return cudaErrorInvalidValue;
 }
 
-cudaError_t launch_stream(int dtype, const StreamArgs& a, cudaStream_t st) {
-    cudaError_t e = launch_stream_prep(dtype, a, st);
-    if (e != cudaSuccess) return e;
-    e = launch_stream_aggregate(dtype, a, st);
-    if (e != cudaSuccess) return e;
-    return launch_stream_broadcast(dtype, a, st);
-}
-
 }  // namespace aa

@@ -68,7 +68,9 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16
 template <typename T> struct Pair;
 template <> struct Pair<__nv_bfloat16> {
     static constexpr uint32_t kOne = 0x3F80u;            // 1.0
-    static constexpr float kBig = 1e30f;                 // finite stand-in for infinity
+    static constexpr float kBig = 30000.f;               // biases are clamped to +-kBig: low enough to remove a key, small
+                                                         // enough that logit arithmetic in fp32 stays exact to 0.01
+    static constexpr float kPad = 60000.f;               // minus this: bias of the agent columns past n
     __device__ static __forceinline__ uint32_t cvt(float lo, float hi) {
         uint32_t d;
         asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
@@ -82,7 +84,8 @@ template <> struct Pair<__nv_bfloat16> {
 };
 template <> struct Pair<__half> {
     static constexpr uint32_t kOne = 0x3C00u;
-    static constexpr float kBig = 60000.f;
+    static constexpr float kBig = 30000.f;
+    static constexpr float kPad = 60000.f;
     __device__ static __forceinline__ uint32_t cvt(float lo, float hi) {
         uint32_t d;
         asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));

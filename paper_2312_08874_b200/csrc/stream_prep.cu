@@ -3,8 +3,8 @@
 //   * agents A = Pooling(Q) (text under Eq. 6): one warp per (slab, agent) window, 16-byte loads with sixteen in
 //     flight per lane, fp32 sums in a fixed order; written as A and as scale1 * A, scale2 * A (each rounded
 //     once from the fp32 mean), the operands of the logit products of Eq. 3.  A caller's agents are only scaled.
-//   * agent biases (Eq. 5): B1 clamped to finite values, transposed to [N][64] (pad columns zero); B2 clamped
-//     and padded to 64 columns with a large negative value.  The attention kernels add the bias inside the
+//   * agent biases (Eq. 5): B1 clamped to +-30000, transposed to [N][64] (pad columns zero); B2 clamped and
+//     padded to 64 columns with -60000.  The attention kernels add the bias inside the
 //     tensor-core contraction (a product with an identity block), where an infinite entry would turn 0 * inf into NaN for every other agent; and the pad
 //     columns make the agents past n drop out of the broadcast softmax without any masking instructions.
 //   * the depthwise filter as diagonal operand slices: the broadcast kernel evaluates the 3x3 term on the tensor
@@ -129,7 +129,7 @@ __global__ void __launch_bounds__(NT) stream_prep_kernel(const StreamArgs p, int
 #pragma unroll
             for (int k = 0; k < 8; ++k) {
                 const int col = c0 + k;
-                float v = -Pair<T>::kBig;
+                float v = -Pair<T>::kPad;
                 if (col < n) v = src ? fminf(fmaxf(Elem<T>::to_f32(src[rowi * n + col]), -Pair<T>::kBig), Pair<T>::kBig) : 0.f;
                 f[k] = v;
             }

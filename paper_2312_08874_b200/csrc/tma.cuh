@@ -52,6 +52,11 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
 __device__ __forceinline__ void fence_proxy_async() {
     asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
 }
+// Orders this thread's earlier generic-proxy accesses (here: the acquire that observed other blocks' plain global
+// stores) before its later async-proxy accesses (TMA reads of that global memory).
+__device__ __forceinline__ void fence_proxy_async_all() {
+    asm volatile("fence.proxy.async;\n" ::: "memory");
+}
 // 2-D tiled load: box at (x = innermost coordinate, y) of the tensor map -> shared memory.
 // x * element size must be a multiple of 16 bytes.
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {

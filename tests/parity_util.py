@@ -67,9 +67,14 @@ def oracle_forward(w: Workload, inp, threads: int = 0, slabs=None, **kw):
     return outs
 
 
-def gpu_forward(mod: AgentAttention, w: Workload, inp) -> torch.Tensor:
-    out = mod.forward(to_dev(inp["q"]), to_dev(inp["k"]), to_dev(inp["v"]), w.grid_h, w.grid_w, w.agents,
-                      b1=to_dev(inp["b1"]), b2=to_dev(inp["b2"]), dwc_weight=to_dev(inp["dwc"]))
+def gpu_forward(mod: AgentAttention, w: Workload, inp, agents=None, return_workspace: bool = False):
+    """One forward call through the C ABI on poisoned buffers: `out` starts as NaN and the workspace as 0xFF bytes
+    (NaN in every element type), so an element the kernels do not write, or read before writing, shows."""
+    dev = {k: to_dev(v) for k, v in inp.items()}
+    out = torch.full_like(dev["q"], float("nan"))
+    ws = torch.full((mod.workspace_bytes(w.grid_h, w.grid_w, w.agents),), 0xFF, dtype=torch.uint8, device="cuda")
+    mod.forward(dev["q"], dev["k"], dev["v"], w.grid_h, w.grid_w, w.agents, agents=agents,
+                b1=dev["b1"], b2=dev["b2"], dwc_weight=dev["dwc"], out=out, workspace=ws)
     torch.cuda.synchronize()
     assert mod.query_status() == 0, "a device-side bounded wait expired"
-    return out
+    return (out, ws) if return_workspace else out

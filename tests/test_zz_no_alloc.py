@@ -7,11 +7,13 @@ a fixed array inside the library instead of a caller-provided workspace.  It mus
 `agent_attn_aggregate` returns, on consecutive calls that reuse the array, and must refuse
 shapes that do not fit the array.
 """
+import numpy as np
 import pytest
 import torch
 
 from paper_2312_08874_b200 import WORKLOADS, AgentAttnError, make_inputs
-from tests.parity_util import TOL, make_module, to_dev
+from oracle import agent_attention_oracle as orc
+from tests.parity_util import TOL, assert_close, make_module, to_dev, to_np
 
 pytestmark = pytest.mark.gpu
 
@@ -36,6 +38,12 @@ def test_static_scratch_aggregation_matches_workspace_aggregation_twice_in_a_row
         torch.cuda.synchronize()
         assert torch.isfinite(got.float()).all(), f"call {call}"
         _close(got, expect, w.dtype)
+        # and against the oracle's aggregation (Eq. 3 with the bias of Eq. 5) on the same agents
+        a_np, k_np, v_np, b_np = to_np(agents.cpu()), to_np(inp["k"]), to_np(inp["v"]), to_np(inp["b1"])
+        ref = np.stack([np.stack([orc.softmax_attention(a_np[b, h], k_np[b, h], v_np[b, h], bias=b_np[h],
+                                                        scale=w.head_dim ** -0.5)
+                                  for h in range(w.heads)]) for b in range(w.batch)])
+        assert_close(got, ref, w.dtype, f"static-scratch aggregation, call {call}")
     # same inputs again: the array keeps the previous call's contents and that must not matter
     again = mod.aggregate_static(agents, k, v, b1=b1)
     torch.cuda.synchronize()
