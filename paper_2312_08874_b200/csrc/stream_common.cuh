@@ -122,13 +122,15 @@ __device__ __forceinline__ void wait_par(Pipe& pp, int i, uint32_t parity, int c
     if (pp.status) atomicCAS(pp.status, 0, code);
 }
 
-// Spinning wait of a single-lane role on the critical path (no back-off: a hand-off costs tens of cycles);
-// bounded like every other wait.
+// Wait of an issuing role (producer, MMA issuers).  The thread is parked by the suspended form of try_wait and
+// woken by the phase completion: a tight polling loop here would take issue slots from the compute warp that
+// shares the scheduler.  Bounded like every other wait.
 __device__ __forceinline__ void wait_spin(Pipe& pp, int i, uint32_t parity, int code) {
     const uint32_t bar = pipe_bar(pp, i);
-    for (unsigned tries = 0; tries < (1u << 24); ++tries) {
-        if (mbar_try_wait(bar, parity & 1u)) return;
-        if ((tries & 1023u) == 1023u && pipe_dead(pp)) return;
+    if (mbar_try_wait(bar, parity & 1u)) return;
+    for (unsigned tries = 0; tries < (1u << 22); ++tries) {
+        if (mbar_try_wait_suspend(bar, parity & 1u, 4000u)) return;
+        if ((tries & 63u) == 63u && pipe_dead(pp)) return;
     }
     *reinterpret_cast<volatile int*>(pp.dead) = 1;
     if (pp.status) atomicCAS(pp.status, 0, code);

@@ -1,6 +1,6 @@
 // First kernel of the streaming path for small agent counts: everything the two attention kernels need
 // besides Q, K and V themselves.
-//   * agents A = Pooling(Q) (text under Eq. 6): one warp per (slab, agent) window, 16-byte loads with sixteen in
+//   * agents A = Pooling(Q) (text under Eq. 6): one warp per (slab, agent) window, 16-byte loads with eight in
 //     flight per lane, fp32 sums in a fixed order; written as A and as scale1 * A, scale2 * A (each rounded
 //     once from the fp32 mean), the operands of the logit products of Eq. 3.  A caller's agents are only scaled.
 //   * agent biases (Eq. 5): B1 clamped to +-30000, transposed to [N][64] (pad columns zero); B2 clamped and
@@ -18,7 +18,7 @@ namespace {
 constexpr int NT = 256;
 
 template <typename T>
-__global__ void __launch_bounds__(NT) stream_prep_kernel(const StreamArgs p, int bias_blocks) {
+__global__ void __launch_bounds__(NT, 4) stream_prep_kernel(const StreamArgs p, int bias_blocks) {
     pdl_launch_dependents();          // the aggregation kernel may set itself up while this one runs
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int N = p.H * p.W, n = p.n;
@@ -40,24 +40,24 @@ __global__ void __launch_bounds__(NT) stream_prep_kernel(const StreamArgs p, int
             const int win_h = p.H / p.p, win_w = p.W / p.p, cnt = win_h * win_w;
             const int y0 = (a / p.p) * win_h, x0 = (a % p.p) * win_w;
             // lane (c, ts) walks the window's tokens ts, ts + 4, ... in row-major order; (wy, wx) is kept
-            // incrementally, so the sixteen loads of a batch cost an add and a compare each
+            // incrementally, so the loads of a batch cost an add and a compare each
             const uint4* gq = reinterpret_cast<const uint4*>(static_cast<const T*>(p.q) + ((size_t)slab * N + (size_t)y0 * p.W + x0) * 64) + c;
             inv = 1.f / (float)cnt;
             int wy = ts / win_w, wx = ts - wy * win_w;
             float2 acc2[4];
 #pragma unroll
             for (int k = 0; k < 4; ++k) acc2[k] = make_float2(0.f, 0.f);
-            for (int ib = ts; ib < cnt; ib += 64) {
-                uint4 raw[16];
+            for (int ib = ts; ib < cnt; ib += 32) {          // eight loads in flight per lane, four blocks per SM
+                uint4 raw[8];
 #pragma unroll
-                for (int u = 0; u < 16; ++u) {
+                for (int u = 0; u < 8; ++u) {
                     raw[u] = make_uint4(0u, 0u, 0u, 0u);
                     if (ib + 4 * u < cnt) raw[u] = __ldg(gq + ((size_t)wy * p.W + wx) * 8);
                     wx += 4;
                     while (wx >= win_w) { wx -= win_w; ++wy; }
                 }
 #pragma unroll
-                for (int u = 0; u < 16; ++u) {
+                for (int u = 0; u < 8; ++u) {
                     acc2[0] = fadd2(acc2[0], unpack2<T>(raw[u].x));
                     acc2[1] = fadd2(acc2[1], unpack2<T>(raw[u].y));
                     acc2[2] = fadd2(acc2[2], unpack2<T>(raw[u].z));
