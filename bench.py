@@ -33,7 +33,7 @@ DEFAULT_WORKLOAD = "cfg3_pvt_bf16"
 # dram__bytes_read.sum + dram__bytes_write.sum per forward pass of the streaming path (three launches), from the ncu
 # capture summarised under profiles/, with the digest of the kernel sources it was taken from: the figure is
 # reported only while those sources are unchanged
-NCU_TRAFFIC = {"cfg3_pvt_bf16": {"bytes": None, "sources_sha256": None}}
+NCU_TRAFFIC = {"cfg3_pvt_bf16": {"bytes": 117.3e6, "sources_sha256": "59cc6ac0f570fe83"}}
 TRAFFIC_SOURCES = ("stream_prep.cu", "stream_aggregate.cu", "stream_broadcast.cu", "stream_common.cuh")
 
 
@@ -333,8 +333,13 @@ def main():
     ap.add_argument("--direction", choices=["forward", "backward"], default="forward",
                     help="backward: time agent_attn_backward (fp32 gradients of Q, K, V, both biases and the filter) "
                          "instead of the forward pass; prints a line with \"pass\": \"backward\"")
+    ap.add_argument("--path", choices=["auto", "queue", "unfused", "simt"], default="auto",
+                    help="kernel family: auto (the library's choice), queue (the persistent task-queue kernel wherever it "
+                         "applies), unfused (one kernel per step), simt (fp32 FMA kernels)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-configs", action="store_true", help="skip the short runs of the other configurations")
+    ap.add_argument("--no-kernel-split", action="store_true",
+                    help="skip the per-kernel timing of the streaming path (for short runs under a profiler)")
     ap.add_argument("--min-warmup-seconds", type=float, default=0.2)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
@@ -356,7 +361,8 @@ def main():
     set_bytes = w.algorithmic_bytes()
     n_sets = n_sets_for(w, l2_bytes)
     host, sets = make_sets(w, dev, n_sets, rank, args.layout)
-    mod = AgentAttention(w.batch, w.heads, w.head_dim, w.tokens, w.agents, dt, device=local_rank)
+    path = {"auto": 0, "simt": 1, "unfused": 2, "queue": 3}[args.path]
+    mod = AgentAttention(w.batch, w.heads, w.head_dim, w.tokens, w.agents, dt, device=local_rank, path=path)
     ws = mod.workspace(w.grid_h, w.grid_w, w.agents)
     stream = torch.cuda.current_stream()
     if args.direction == "backward":
@@ -398,7 +404,7 @@ def main():
     peak, tensor_peak, peak_src = measured_peaks()
     kb_steps = min(args.steps, 200)
     kern_note = None
-    if launches_per_step == 3 and args.layout == "dense":
+    if launches_per_step == 3 and args.layout == "dense" and not args.no_kernel_split:
         # three streaming kernels per forward call: each timed by itself between events through the stage mask
         # (a later stage alone reads what the last full call left in the workspace)
         names = ("prep", "aggregate", "broadcast_dwc")
@@ -415,7 +421,7 @@ def main():
                      "programmatic dependent launch gives the path); kernel_algorithmic_bytes counts what a kernel "
                      "touches, second reads of Q and V included, so it sums to more than the path's bytes")
         dominant = "forward_path"
-    elif launches_per_step == 1 or args.layout != "dense":
+    elif launches_per_step in (1, 3) or args.layout != "dense":
         dominant = "fused_kernel" if launches_per_step == 1 else "forward_path"
         kern_ms = {dominant: ms_step}
         kern_bytes = {dominant: set_bytes}
@@ -537,7 +543,7 @@ def main():
             "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
             "config": {"workload": w.name, "batch_per_gpu": w.batch, "heads": w.heads, "tokens": w.tokens,
                        "grid": [w.grid_h, w.grid_w], "head_dim": w.head_dim, "agents": w.agents,
-                       "bias": w.bias, "dwc": w.dwc, "layout": args.layout,
+                       "bias": w.bias, "dwc": w.dwc, "layout": args.layout, "path": args.path,
                        "l2": f"{n_sets} rotating buffer sets of {set_bytes / 1e6:.1f} MB (> 4x the {l2_bytes / 2**20:.0f} MiB L2)",
                        "timing": f"median of {len(times)} regions of {args.steps} forward calls each, CUDA events",
                        "parallelism": f"batch-sharded x{world}, no collective"},
