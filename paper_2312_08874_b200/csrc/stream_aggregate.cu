@@ -53,7 +53,8 @@ constexpr int BAR_P_FULL = 10;    // [2]       row threads    MMA issuer
 constexpr int BAR_PV = 12;        // [2]       commit         row warps (only when a reference moves, and at the end)
 constexpr int BAR_A = 14;         //           row threads    MMA issuer      the agent operand is in tensor memory
 constexpr int BAR_S_EMPTY = 15;   // [2]       row threads    MMA issuer      the logits have been read
-constexpr int kBars = 17;
+constexpr int BAR_DRAIN = 17;     // [2]       commit         each MMA issuer, once, at its end
+constexpr int kBars = 19;
 
 // tensor memory columns: logits 2 x 128, probabilities 2 x 64 (16-bit pairs), accumulator 64,
 // agent operand 32 (64 channels) + 32 (identity, 64 agents)
@@ -133,7 +134,7 @@ __global__ void __launch_bounds__(NT, 1) stream_aggregate_kernel(const __grid_co
     if (tid == 0) {
         s_dead = 0;
         for (int i = 0; i < kBars; ++i)
-            mbar_init(pp.bars + 8 * i, ((i >= BAR_P_FULL && i < BAR_PV) || i >= BAR_A) ? (uint32_t)NROW : 1u);
+            mbar_init(pp.bars + 8 * i, ((i >= BAR_P_FULL && i < BAR_PV) || (i >= BAR_A && i < BAR_DRAIN)) ? (uint32_t)NROW : 1u);
         mbar_fence_init();
     }
     if (warp == 0) tmem_alloc<512>(smem_u32(&s_tmem));
@@ -161,7 +162,7 @@ __global__ void __launch_bounds__(NT, 1) stream_aggregate_kernel(const __grid_co
             if (has_bias)
                 for (int i = 0; i < first; ++i)
                     tma_load_3d(ring + i * kStage + 2 * kTile, &p.tm_b1, 0, (t0 + i) * TK, head, pipe_bar(pp, BAR_FULL + i));
-            for (int i = first; i < tiles; ++i) {
+            for (int i = first; i < tiles && !pipe_dead(pp); ++i) {
                 const int s = i % STAGES, c0 = (t0 + i) * TK;
                 wait_spin(pp, BAR_EMPTY + s, (i / STAGES) - 1, kTimeoutRole);
                 const uint32_t bar = pipe_bar(pp, BAR_FULL + s), dst = ring + s * kStage;
@@ -182,7 +183,7 @@ __global__ void __launch_bounds__(NT, 1) stream_aggregate_kernel(const __grid_co
             // descriptor start addresses count 16-byte units: + 2 per K-step of a K-major operand (32 bytes).
             // `u` is a compile-time constant (the tile loop is unrolled over the ring).
             wait_spin(pp, BAR_A, 0, kTimeoutLoads);
-            for (int i0 = 0; i0 < tiles; i0 += STAGES) {
+            for (int i0 = 0; i0 < tiles && !pipe_dead(pp); i0 += STAGES) {
 #pragma unroll
                 for (int u = 0; u < STAGES; ++u) {
                     const int i = i0 + u;
@@ -205,6 +206,7 @@ __global__ void __launch_bounds__(NT, 1) stream_aggregate_kernel(const __grid_co
                     }
                 }
             }
+            umma_drain_w(pp, BAR_DRAIN);
         }
         __syncwarp();
     } else if (warp == 6) {
@@ -214,7 +216,7 @@ __global__ void __launch_bounds__(NT, 1) stream_aggregate_kernel(const __grid_co
             const uint64_t dRing = umma_desc_sw128(ring);
             const uint32_t tD = pp.tmem + TM_D, tPb = pp.tmem + TM_P;
             // + 128 per K-step of an MN-major operand (16 rows of 128 bytes)
-            for (int i0 = 0; i0 < tiles; i0 += STAGES) {
+            for (int i0 = 0; i0 < tiles && !pipe_dead(pp); i0 += STAGES) {
 #pragma unroll
                 for (int u = 0; u < STAGES; ++u) {
                     const int i = i0 + u;
@@ -231,6 +233,7 @@ __global__ void __launch_bounds__(NT, 1) stream_aggregate_kernel(const __grid_co
                     }
                 }
             }
+            umma_drain_w(pp, BAR_DRAIN + 1);
         }
         __syncwarp();
     } else {

@@ -71,7 +71,8 @@ constexpr int BAR_P_FULL = 12;    // [2]       softmax threads attention issuer
 constexpr int BAR_O_FULL = 14;    // [2]       commit          output warps
 constexpr int BAR_D_FULL = 16;    // [2]       2 commits       output warps
 constexpr int BAR_O_EMPTY = 18;   // [2]       output threads  both MMA issuers, softmax warps (the row sums' buffer)
-constexpr int kBars = 20;
+constexpr int BAR_DRAIN = 20;     // [3]       commit          each MMA issuer, once, at its end
+constexpr int kBars = 23;
 
 // tensor memory columns: logits 2 x 64 (the probabilities overwrite the first 32), output 2 x 64,
 // depthwise 2 issuers x 2 x 64
@@ -114,7 +115,7 @@ __global__ void __launch_bounds__(NT, 1) stream_broadcast_kernel(const __grid_co
     if (tid == 0) {
         s_dead = 0;
         for (int i = 0; i < kBars; ++i)
-            mbar_init(pp.bars + 8 * i, ((i >= BAR_P_FULL && i < BAR_O_FULL) || i >= BAR_O_EMPTY) ? (uint32_t)NROW
+            mbar_init(pp.bars + 8 * i, ((i >= BAR_P_FULL && i < BAR_O_FULL) || (i >= BAR_O_EMPTY && i < BAR_DRAIN)) ? (uint32_t)NROW
                                        : ((i >= BAR_H_EMPTY && i < BAR_S_FULL) || (i >= BAR_D_FULL && i < BAR_O_EMPTY)) ? 2u : 1u);
         mbar_fence_init();
     }
@@ -156,7 +157,7 @@ __global__ void __launch_bounds__(NT, 1) stream_broadcast_kernel(const __grid_co
             pdl_wait();      // A, V_A, the padded B2 and the weight slices come from the preceding kernels
             int cur = -1, ord = -1;
             const uint32_t qb_tx = 2u * (uint32_t)L.tq * 128u;
-            for (int i = 0; i < T_; ++i, it.next()) {
+            for (int i = 0; i < T_ && !pipe_dead(pp); ++i, it.next()) {
                 if (it.slab != cur) {
                     // (a buffer is reused two slabs later: every product that read it is long done, since the
                     // stage waits below already cover the tiles of the slab in between)
@@ -220,7 +221,7 @@ __global__ void __launch_bounds__(NT, 1) stream_broadcast_kernel(const __grid_co
                 umma_commit_w(pipe_bar(pp, BAR_S_FULL + b));
             };
             if (T_ > 0) issue_S(0, 0);
-            for (int i0 = 0; i0 < T_; i0 += 2) {
+            for (int i0 = 0; i0 < T_ && !pipe_dead(pp); i0 += 2) {
 #pragma unroll
                 for (int b = 0; b < 2; ++b) {
                     const int i = i0 + b;
@@ -240,6 +241,7 @@ __global__ void __launch_bounds__(NT, 1) stream_broadcast_kernel(const __grid_co
                     }
                 }
             }
+            umma_drain_w(pp, BAR_DRAIN);
         }
         __syncwarp();
     } else if (warp == 10 || warp == 11) {
@@ -252,7 +254,7 @@ __global__ void __launch_bounds__(NT, 1) stream_broadcast_kernel(const __grid_co
             const uint32_t tD = pp.tmem + TM_D + 128 * half;
             const int wp8 = L.wp * 8;                        // one grid row of the V tile, in 16-byte descriptor units
             int cur = -1, ord = -1;
-            for (int i0 = 0; i0 < T_; i0 += 2) {
+            for (int i0 = 0; i0 < T_ && !pipe_dead(pp); i0 += 2) {
 #pragma unroll
                 for (int b = 0; b < 2; ++b) {
                     const int i = i0 + b;
@@ -285,6 +287,7 @@ __global__ void __launch_bounds__(NT, 1) stream_broadcast_kernel(const __grid_co
                     }
                 }
             }
+            umma_drain_w(pp, BAR_DRAIN + 1 + half);
         }
         __syncwarp();
     } else if (warp < 4) {

@@ -136,6 +136,15 @@ __device__ __forceinline__ void wait_spin(Pipe& pp, int i, uint32_t parity, int 
     if (pp.status) atomicCAS(pp.status, 0, code);
 }
 
+// End of an MMA-issuing warp: commit to a barrier of its own and wait (bounded, whatever the block's state) until
+// every instruction it has issued is complete, so that the block never frees its tensor memory under a running one.
+__device__ __forceinline__ void umma_drain_w(Pipe& pp, int i) {
+    umma_commit_w(pipe_bar(pp, i));
+    const uint32_t bar = pipe_bar(pp, i);
+    for (unsigned tries = 0; tries < (1u << 16); ++tries)
+        if (mbar_try_wait_suspend(bar, 0u, 4000u)) return;
+}
+
 // 3-D tiled load: box at (0, row, z) of a map whose dimensions are (64 channels or columns, rows, slabs or
 // heads).  Rows outside [0, rows) are zero-filled, so a tile never runs into the next slab.
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
