@@ -130,7 +130,7 @@ __global__ void __launch_bounds__(NT, 1) aggregate_umma_kernel(const __grid_cons
     } else if (warp == 17 || warp == 18) {
         // ------------------------------------------------------------------ MMA issuer of chain m = agent block m
         const int m = warp - 17;
-        if (lane == 0 && m < MB) {
+        if (m < MB) {     // (the whole warp runs the loop; one elected lane issues)
             const uint32_t idK = umma_idesc(fmt, 128, 64, 0), idMN = umma_idesc(fmt, 128, 64, 1);
             const uint64_t dA = umma_desc_sw128(sA) + 1024 * m, dRing = umma_desc_sw128(ring);
             // descriptor start addresses count 16-byte units: + 2 per K-step of a K-major operand (32 bytes),
@@ -142,11 +142,11 @@ __global__ void __launch_bounds__(NT, 1) aggregate_umma_kernel(const __grid_cons
                 tc_fence_after_sync();
                 const uint64_t dK = dRing + (uint64_t)(s * (kStage >> 4));
                 const uint32_t dd = pp.tmem + TM_S + 128 * b + 64 * m;
-                umma_f16_c<0>(dd, dA, dK, idK);
-                umma_f16_c<1>(dd, dA + 2, dK + 2, idK);
-                umma_f16_c<1>(dd, dA + 4, dK + 4, idK);
-                umma_f16_c<1>(dd, dA + 6, dK + 6, idK);
-                umma_commit(pipe_bar(pp, BAR_S_FULL + 2 * m + b));
+                umma_ss_w(dd, dA, dK, idK, 0u);
+                umma_ss_w(dd, dA + 2, dK + 2, idK, 1u);
+                umma_ss_w(dd, dA + 4, dK + 4, idK, 1u);
+                umma_ss_w(dd, dA + 6, dK + 6, idK, 1u);
+                umma_commit_w(pipe_bar(pp, BAR_S_FULL + 2 * m + b));
             };
             pipe_wait_one(pp, BAR_AG, kTimeoutLoads);
             issue_S(0);
@@ -162,11 +162,11 @@ __global__ void __launch_bounds__(NT, 1) aggregate_umma_kernel(const __grid_cons
                     if (32 * c >= ntok) break;
                     const uint32_t dd = pp.tmem + TM_O + 64 * (2 * m + c);
                     const uint64_t da = dP + 4 * c, db = dV + 256 * c;
-                    if (t > 0) umma_f16_c<1>(dd, da, db, idMN); else umma_f16_c<0>(dd, da, db, idMN);
-                    umma_f16_c<1>(dd, da + 2, db + 128, idMN);
+                    if (t > 0) umma_ss_w(dd, da, db, idMN, 1u); else umma_ss_w(dd, da, db, idMN, 0u);
+                    umma_ss_w(dd, da + 2, db + 128, idMN, 1u);
                 }
-                umma_commit(pipe_bar(pp, BAR_EMPTY + s));
-                umma_commit(pipe_bar(pp, BAR_PV + m));
+                umma_commit_w(pipe_bar(pp, BAR_EMPTY + s));
+                umma_commit_w(pipe_bar(pp, BAR_PV + m));
             }
             for (int t = max(0, tiles - 2); t < tiles; ++t) pipe_wait_one(pp, BAR_S_EMPTY + 2 * m + (t & 1), kTimeoutRole);
         }

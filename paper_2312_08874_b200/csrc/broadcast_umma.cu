@@ -155,7 +155,7 @@ __global__ void __launch_bounds__(NT, 1) broadcast_umma_kernel(const __grid_cons
         __syncwarp();
     } else if (warp == 17) {
         // ------------------------------------------------------------------ MMA issuer: logits, one step ahead
-        if (lane == 0) {
+        {     // (the whole warp runs the loop; one elected lane issues)
             const uint32_t idS = umma_idesc(fmt, 128, 128, 0);
             const uint64_t dA = umma_desc_sw128(sA), dQ = umma_desc_sw128(sQ);
             // descriptor start addresses count 16-byte units: + 2 per K-step of a K-major operand (32 bytes),
@@ -168,19 +168,19 @@ __global__ void __launch_bounds__(NT, 1) broadcast_umma_kernel(const __grid_cons
                 tc_fence_after_sync();
                 const uint32_t dd = pp.tmem + TM_S + 128 * b;
                 const uint64_t da = dQ + 1024 * (i & 1), db = dA + 1024 * a;
-                umma_f16_c<0>(dd, da, db, idS);
-                umma_f16_c<1>(dd, da + 2, db + 2, idS);
-                umma_f16_c<1>(dd, da + 4, db + 4, idS);
-                umma_f16_c<1>(dd, da + 6, db + 6, idS);
-                if (a == MB - 1) umma_commit(pipe_bar(pp, BAR_Q_EMPTY + (i & 1)));
-                umma_commit(pipe_bar(pp, BAR_S_FULL + b));
+                umma_ss_w(dd, da, db, idS, 0u);
+                umma_ss_w(dd, da + 2, db + 2, idS, 1u);
+                umma_ss_w(dd, da + 4, db + 4, idS, 1u);
+                umma_ss_w(dd, da + 6, db + 6, idS, 1u);
+                if (a == MB - 1) umma_commit_w(pipe_bar(pp, BAR_Q_EMPTY + (i & 1)));
+                umma_commit_w(pipe_bar(pp, BAR_S_FULL + b));
             }
             for (int j = max(0, steps - 2); j < steps; ++j) pipe_wait_one(pp, BAR_S_EMPTY + (j & 1), kTimeoutRole);
         }
         __syncwarp();
     } else if (warp == 18) {
         // ------------------------------------------------------------------ MMA issuer: products P V_A
-        if (lane == 0) {
+        {     // (the whole warp runs the loop; one elected lane issues)
             const uint32_t idMN = umma_idesc(fmt, 128, 64, 1);
             const uint64_t dVA = umma_desc_sw128(sVA), dP0 = umma_desc_sw128(sB2);
             // + 128 per K-step of an MN-major operand (16 rows of 128 bytes)
@@ -196,12 +196,12 @@ __global__ void __launch_bounds__(NT, 1) broadcast_umma_kernel(const __grid_cons
                     if (128 * a + 32 * gq >= n) break;
                     const uint32_t dd = pp.tmem + TM_O + 64 * gq;
                     const uint64_t da = dP + 1024 * (gq >> 1) + 4 * (gq & 1), db = dVA + 128 * (8 * a + 2 * gq);
-                    if ((started >> gq) & 1u) umma_f16_c<1>(dd, da, db, idMN); else umma_f16_c<0>(dd, da, db, idMN);
-                    umma_f16_c<1>(dd, da + 2, db + 128, idMN);
+                    if ((started >> gq) & 1u) umma_ss_w(dd, da, db, idMN, 1u); else umma_ss_w(dd, da, db, idMN, 0u);
+                    umma_ss_w(dd, da + 2, db + 128, idMN, 1u);
                     started |= 1u << gq;
                 }
-                if (has_b2) umma_commit(pipe_bar(pp, BAR_B_EMPTY + (j & 1)));     // the stage may take the bias of step j + 2
-                umma_commit(pipe_bar(pp, BAR_PV));
+                if (has_b2) umma_commit_w(pipe_bar(pp, BAR_B_EMPTY + (j & 1)));     // the stage may take the bias of step j + 2
+                umma_commit_w(pipe_bar(pp, BAR_PV));
             }
         }
         __syncwarp();
